@@ -1,0 +1,163 @@
+/*
+ * director.h - C ABI of libdirector.so
+ *
+ * The expert-parallel Mixture-of-Experts layer forward under a given expert placement, on one
+ * GPU, with the expert-parallel "ranks" as logical partitions of that GPU (no inter-GPU
+ * traffic).  This is the computation whose latency the paper's proactive expert placement
+ * reduces: gate -> all-to-all dispatch -> expert FFNs -> all-to-all aggregate (Section II-A,
+ * Section II-B), together with the quantities its placement optimiser trades off (Section VI-A,
+ * Eq. 1-4).
+ *
+ * Notation (paper, Section VI-A; indices are 0-based here, the paper counts from 1):
+ *   T  tokens in the batch            H  hidden size            F  expert FFN width
+ *   E  routed experts per layer       K  experts chosen per token (top-k)
+ *   S  always-on shared experts       R  logical ranks (the GPU set G of the paper)
+ *   C_max  expert slots per rank (the paper's per-GPU capacity C_max)
+ *   X[E][R]  placement matrix, X[i][j] = 1 iff expert i is hosted on rank j (the variable
+ *            x_{i,j} of Eq. 6: sum_j x_{i,j} >= 1, sum_i x_{i,j} <= C_max); an expert hosted on
+ *            several ranks is replicated, all replicas use the same weight array.
+ *   A = T*K  (token, choice) assignments;   G = R*C_max  slots.
+ *   Slot g = j*C_max + p holds the p-th smallest expert id hosted on rank j (or nothing).
+ *
+ * Conventions
+ *   - Every pointer marked "dev" is caller-owned device memory on the context's device,
+ *     16-byte aligned, valid until the stream has reached the call.  "host" pointers are
+ *     ordinary host memory.  The context owns only its internal workspace, sized at create
+ *     time; no entry point allocates after director_create.
+ *   - bf16 tensors are passed as void* (raw 16-bit patterns), row-major, innermost last.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Calls are asynchronous on `stream` and never synchronise unless stated.  Every function
+ *     returns a director_status; nothing throws across the boundary.  Argument errors are
+ *     detected on the host before anything is launched.  Faults only visible on the device
+ *     (an expert id outside [0,E), a non-finite logit, a bounded wait that expired) set a
+ *     sticky status word that director_last_status reads; the offending element is skipped,
+ *     kernels never trap.
+ *   - Supported ranges: 1 <= K <= 8, K <= E <= 256, 1 <= R <= 64, 1 <= C_max <= 16,
+ *     E <= R*C_max, H % 256 == 0, F % 128 == 0, S >= 0, T_max*K < 2^31.
+ */
+#ifndef DIRECTOR_H
+#define DIRECTOR_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct director_ctx director_ctx;
+
+typedef enum {
+    DIRECTOR_OK = 0,
+    DIRECTOR_ERR_INVALID_ARG = 1,   /* NULL / misaligned pointer, size out of range            */
+    DIRECTOR_ERR_PLACEMENT = 2,     /* an expert has no host, or a rank exceeds C_max, or unset */
+    DIRECTOR_ERR_WORKSPACE = 3,     /* device allocation failed at create time                  */
+    DIRECTOR_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed                        */
+    DIRECTOR_ERR_UNSUPPORTED = 5,   /* shape outside the supported ranges, or not an sm_100 GPU */
+    DIRECTOR_ERR_TIMEOUT = 6,       /* device: a bounded wait inside a kernel expired           */
+    DIRECTOR_ERR_BAD_INDEX = 7,     /* device: expert id outside [0,E) met (element skipped)    */
+    DIRECTOR_ERR_NONFINITE = 8      /* device: NaN/Inf router logit met                         */
+} director_status;
+
+typedef struct {
+    int32_t T_max;   /* largest batch any call will pass */
+    int32_t H, F, E, K, S, R, C_max;
+} director_shape;
+
+/* Life cycle.  director_create allocates the workspace on the current device (it is the only
+ * call that allocates) and binds the context to that device. */
+int director_create(const director_shape* shape, director_ctx** out);
+int director_destroy(director_ctx* ctx);
+
+/* Expert placement (Section VI-A placement map; Eq. 6 assignment and capacity constraints).
+ * X_host: host, uint8 [E][R] row-major, entries 0/1.  Validates that every expert has at
+ * least one host and no rank hosts more than C_max experts (DIRECTOR_ERR_PLACEMENT
+ * otherwise, previous placement kept), builds the slot tables and uploads them on `stream`.
+ * X_host may be reused as soon as the call returns. */
+int director_set_placement(director_ctx* ctx, const uint8_t* X_host, void* stream);
+
+/* (a1) Gating (Section II-A: relevance scores, top-k selection, scores used as weights).
+ * logits: dev fp32 [T,E].  topk_idx: dev int32 [T,K], the K experts with the largest logits in
+ * descending order, ties to the lower expert id.  topk_w: dev fp32 [T,K], softmax scores of
+ * the chosen experts renormalised to sum to one. */
+int director_route(director_ctx* ctx, int32_t T, const float* logits,
+                   int32_t* topk_idx, float* topk_w, void* stream);
+
+/* (a2) Dispatch (Section II-B: tokens are packaged and sent to the ranks hosting their experts;
+ * here an on-device permutation, the bytes that would cross ranks are counted by
+ * director_placement_cost).  The n-th assignment of expert e in ascending token order goes to
+ * replica n mod r_e of e (replicas ordered by rank) and becomes row n div r_e of that replica's
+ * segment; segments lie in slot order.
+ * x: dev bf16 [T,H].  topk_idx: dev int32 [T,K].
+ * xp: dev bf16 [T*K,H] permuted copies of the rows of x.   row_token: dev int32 [T*K], token of
+ * each row.  inv_row: dev int32 [T,K], row of each assignment.  dest_rank: dev int32 [T,K].
+ * seg_offsets: dev int32 [R*C_max+1], first row of each slot's segment, last entry T*K. */
+int director_dispatch(director_ctx* ctx, int32_t T, const void* x, const int32_t* topk_idx,
+                      void* xp, int32_t* row_token, int32_t* inv_row, int32_t* dest_rank,
+                      int32_t* seg_offsets, void* stream);
+
+/* (a3) Expert FFNs (Section II-A: each expert is an FFN sub-network), SwiGLU, bf16 operands,
+ * fp32 accumulation on the tensor cores:  for every row i of the segment of slot g (expert e)
+ *   yp[i,:] = ( silu(xp[i,:] . w_gate[e]^T) * (xp[i,:] . w_up[e]^T) ) . w_down[e]^T
+ * xp: dev bf16 [T*K,H].  seg_offsets: dev int32 [R*C_max+1] as written by director_dispatch under
+ * the current placement.  w_gate, w_up: dev bf16 [E,F,H].  w_down: dev bf16 [E,H,F].
+ * yp: dev bf16 [T*K,H].
+ * Shared experts (only if the context has S > 0 and x != NULL): the S always-on FFNs applied
+ * to every token's own row, summed: x: dev bf16 [T,H]; ws_gate, ws_up: dev bf16 [S*F,H] (the S
+ * experts stacked); ws_down: dev bf16 [H,S*F] (the S experts side by side);
+ * y_shared: dev bf16 [T,H]. */
+int director_expert_ffn(director_ctx* ctx, int32_t T, const void* xp, const int32_t* seg_offsets,
+                        const void* w_gate, const void* w_up, const void* w_down, void* yp,
+                        const void* x, const void* ws_gate, const void* ws_up, const void* ws_down,
+                        void* y_shared, void* stream);
+
+/* (a4) Combine (Section II-A weighted summation; Section II-B second all-to-all):
+ *   y[t,:] = bf16( sum_s topk_w[t,s] * yp[inv_row[t,s],:]  (+ y_shared[t,:]) ), fp32 accumulation
+ * in slot order.  yp: dev bf16 [T*K,H].  inv_row: dev int32 [T,K].  topk_w: dev fp32 [T,K].
+ * y_shared: dev bf16 [T,H] or NULL.  y: dev bf16 [T,H]. */
+int director_combine(director_ctx* ctx, int32_t T, const void* yp, const int32_t* inv_row,
+                     const float* topk_w, const void* y_shared, void* y, void* stream);
+
+/* (a5) Placement cost (Section VI-A): workload matrix W, per-rank load of Eq. 1 and dispatch
+ * volume of Eq. 3 for the current placement, counted per executed assignment.
+ * topk_idx: dev int32 [T,K].  token_src_rank: dev int32 [T] home rank of each token, or NULL for
+ * the block partition src(t) = floor(t*R/T).
+ * workload: dev int64 [R,E], W[j][i] = tokens of rank j routed to expert i.
+ * rank_load: dev int64 [R], assignments executed on rank j (lambda_j).
+ * dispatch_tokens: dev int64 [R,R], [j][k] = assignments of tokens of rank j executed on rank k
+ * (the diagonal is local traffic, which Eq. 4 leaves out).
+ * dispatch_bytes: dev uint64 [R,R] = dispatch_tokens * d with d = 2*H bytes per token (Eq. 3). */
+int director_placement_cost(director_ctx* ctx, int32_t T, const int32_t* topk_idx,
+                            const int32_t* token_src_rank, int64_t* workload, int64_t* rank_load,
+                            int64_t* dispatch_tokens, uint64_t* dispatch_bytes, void* stream);
+
+/* The whole layer for callers that hold their batch in host memory: copies logits and x to the
+ * device, runs (a1)-(a5) on context-owned buffers and copies y and the histograms back, all
+ * on `stream`; synchronises `stream` before returning.
+ * logits: host fp32 [T,E].  x: host bf16 [T,H].  Weights: dev, as for director_expert_ffn
+ * (ws_* may be NULL when S == 0).  y: host bf16 [T,H].  rank_load: host int64 [R] or NULL.
+ * dispatch_bytes: host uint64 [R,R] or NULL.  Pinned host buffers make the copies asynchronous. */
+int director_layer_forward_host(director_ctx* ctx, int32_t T, const float* logits, const void* x,
+                                const void* w_gate, const void* w_up, const void* w_down,
+                                const void* ws_gate, const void* ws_up, const void* ws_down,
+                                void* y, int64_t* rank_load, uint64_t* dispatch_bytes, void* stream);
+
+/* Synchronises `stream`, returns the sticky device status word (DIRECTOR_OK if clean) and
+ * clears it. */
+int director_last_status(director_ctx* ctx, void* stream);
+
+/* Number of kernels this context has launched since it was created. */
+int64_t director_launch_count(const director_ctx* ctx);
+
+/* Per-kernel device timing.  While enabled, every launch is bracketed by CUDA events on its
+ * stream.  director_kernel_time synchronises the device, then returns the summed duration in
+ * milliseconds and the number of launches of the kernels whose name contains `name_substr`
+ * since profiling was last enabled; returns a negative value on error. */
+int director_set_profiling(director_ctx* ctx, int32_t enabled);
+double director_kernel_time(director_ctx* ctx, const char* name_substr, int64_t* launches);
+
+const char* director_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DIRECTOR_H */

@@ -1,0 +1,179 @@
+"""Thin ctypes binding of ``libdirector.so`` (see ``include/director.h``).
+
+Argument marshalling only: torch tensors supply device memory and the current CUDA stream; every
+step of the layer runs in the library's own kernels.  There is no fallback: if the library is
+missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+from ctypes import POINTER, c_char_p, c_double, c_float, c_int, c_int32, c_int64, c_uint8, c_uint64, c_void_p
+
+from . import build as _build
+
+STATUS_NAMES = {
+    0: "DIRECTOR_OK", 1: "DIRECTOR_ERR_INVALID_ARG", 2: "DIRECTOR_ERR_PLACEMENT", 3: "DIRECTOR_ERR_WORKSPACE",
+    4: "DIRECTOR_ERR_CUDA", 5: "DIRECTOR_ERR_UNSUPPORTED", 6: "DIRECTOR_ERR_TIMEOUT", 7: "DIRECTOR_ERR_BAD_INDEX",
+    8: "DIRECTOR_ERR_NONFINITE",
+}
+
+# every symbol include/director.h declares
+EXPORTED = (
+    "director_create", "director_destroy", "director_set_placement", "director_route", "director_dispatch",
+    "director_expert_ffn", "director_combine", "director_placement_cost", "director_layer_forward_host",
+    "director_last_status", "director_launch_count", "director_set_profiling", "director_kernel_time",
+    "director_status_string",
+)
+
+
+class DirectorShape(ctypes.Structure):
+    _fields_ = [(n, c_int32) for n in ("T_max", "H", "F", "E", "K", "S", "R", "C_max")]
+
+
+class DirectorError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+
+
+_lib = None
+
+
+def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
+    """Loads libdirector.so from the package directory (building it first if the sources are newer).
+    Raises if it cannot be built or loaded - there is no other implementation to fall back to."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.build_director() if rebuild_if_stale else _build.DIRECTOR_LIB
+    lib = ctypes.CDLL(str(path))
+    vp = c_void_p
+    lib.director_create.argtypes = [POINTER(DirectorShape), POINTER(vp)]
+    lib.director_destroy.argtypes = [vp]
+    lib.director_set_placement.argtypes = [vp, vp, vp]
+    lib.director_route.argtypes = [vp, c_int32, vp, vp, vp, vp]
+    lib.director_dispatch.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.director_expert_ffn.argtypes = [vp, c_int32] + [vp] * 12
+    lib.director_combine.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp]
+    lib.director_placement_cost.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp, vp]
+    lib.director_layer_forward_host.argtypes = [vp, c_int32] + [vp] * 12
+    lib.director_last_status.argtypes = [vp, vp]
+    lib.director_launch_count.argtypes = [vp]
+    lib.director_launch_count.restype = c_int64
+    lib.director_set_profiling.argtypes = [vp, c_int32]
+    lib.director_kernel_time.argtypes = [vp, c_char_p, POINTER(c_int64)]
+    lib.director_kernel_time.restype = c_double
+    lib.director_status_string.argtypes = [c_int]
+    lib.director_status_string.restype = c_char_p
+    for name in EXPORTED:
+        if name not in ("director_launch_count", "director_kernel_time", "director_status_string"):
+            getattr(lib, name).restype = c_int
+    _lib = lib
+    return lib
+
+
+def _ptr(t):
+    """Device (or host) address of a torch tensor / numpy array / None."""
+    if t is None:
+        return None
+    if hasattr(t, "data_ptr"):
+        return t.data_ptr()
+    return t.ctypes.data
+
+
+def _stream():
+    import torch
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise DirectorError(status, where)
+
+
+class Director:
+    """One MoE layer context: shape, placement and workspace.  Methods mirror the C entry points and
+    take torch CUDA tensors (bf16 tensors as torch.bfloat16).  One context serves one stream at a time."""
+
+    def __init__(self, T_max: int, H: int, F: int, E: int, K: int, S: int, R: int, C_max: int):
+        self.lib = load_library()
+        self.shape = DirectorShape(T_max, H, F, E, K, S, R, C_max)
+        self._ctx = c_void_p()
+        _check(self.lib.director_create(ctypes.byref(self.shape), ctypes.byref(self._ctx)), "director_create")
+
+    def close(self):
+        if getattr(self, "_ctx", None) is not None and self._ctx.value:
+            self.lib.director_destroy(self._ctx)
+            self._ctx = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- placement -----------------------------------------------------------------------------
+    def set_placement(self, X):
+        """X: numpy uint8 [E, R] (C-contiguous)."""
+        import numpy as np
+        X = np.ascontiguousarray(X, dtype=np.uint8)
+        assert X.shape == (self.shape.E, self.shape.R)
+        _check(self.lib.director_set_placement(self._ctx, X.ctypes.data, _stream()), "director_set_placement")
+
+    # -- stages --------------------------------------------------------------------------------
+    def route(self, T, logits, topk_idx, topk_w):
+        _check(self.lib.director_route(self._ctx, T, _ptr(logits), _ptr(topk_idx), _ptr(topk_w), _stream()),
+               "director_route")
+
+    def dispatch(self, T, x, topk_idx, xp, row_token, inv_row, dest_rank, seg_offsets):
+        _check(self.lib.director_dispatch(self._ctx, T, _ptr(x), _ptr(topk_idx), _ptr(xp), _ptr(row_token),
+                                          _ptr(inv_row), _ptr(dest_rank), _ptr(seg_offsets), _stream()),
+               "director_dispatch")
+
+    def expert_ffn(self, T, xp, seg_offsets, w_gate, w_up, w_down, yp, x=None, ws_gate=None, ws_up=None,
+                   ws_down=None, y_shared=None):
+        _check(self.lib.director_expert_ffn(self._ctx, T, _ptr(xp), _ptr(seg_offsets), _ptr(w_gate), _ptr(w_up),
+                                            _ptr(w_down), _ptr(yp), _ptr(x), _ptr(ws_gate), _ptr(ws_up),
+                                            _ptr(ws_down), _ptr(y_shared), _stream()), "director_expert_ffn")
+
+    def combine(self, T, yp, inv_row, topk_w, y_shared, y):
+        _check(self.lib.director_combine(self._ctx, T, _ptr(yp), _ptr(inv_row), _ptr(topk_w), _ptr(y_shared),
+                                         _ptr(y), _stream()), "director_combine")
+
+    def placement_cost(self, T, topk_idx, token_src_rank, workload, rank_load, dispatch_tokens, dispatch_bytes):
+        _check(self.lib.director_placement_cost(self._ctx, T, _ptr(topk_idx), _ptr(token_src_rank), _ptr(workload),
+                                                _ptr(rank_load), _ptr(dispatch_tokens), _ptr(dispatch_bytes),
+                                                _stream()), "director_placement_cost")
+
+    def layer_forward_host(self, T, logits, x, w_gate, w_up, w_down, ws_gate, ws_up, ws_down, y,
+                           rank_load=None, dispatch_bytes=None):
+        """logits, x, y, rank_load, dispatch_bytes: host (pinned torch CPU tensors or numpy); weights: device."""
+        _check(self.lib.director_layer_forward_host(self._ctx, T, _ptr(logits), _ptr(x), _ptr(w_gate), _ptr(w_up),
+                                                    _ptr(w_down), _ptr(ws_gate), _ptr(ws_up), _ptr(ws_down), _ptr(y),
+                                                    _ptr(rank_load), _ptr(dispatch_bytes), _stream()),
+               "director_layer_forward_host")
+
+    # -- status / instrumentation --------------------------------------------------------------
+    def last_status(self) -> int:
+        return int(self.lib.director_last_status(self._ctx, _stream()))
+
+    def check_device_status(self):
+        _check(self.last_status(), "device status")
+
+    def launch_count(self) -> int:
+        return int(self.lib.director_launch_count(self._ctx))
+
+    def set_profiling(self, enabled: bool):
+        _check(self.lib.director_set_profiling(self._ctx, 1 if enabled else 0), "director_set_profiling")
+
+    def kernel_time(self, name_substr: str):
+        """(total milliseconds, launches) of kernels whose name contains name_substr since profiling was enabled."""
+        n = c_int64(0)
+        ms = float(self.lib.director_kernel_time(self._ctx, name_substr.encode(), ctypes.byref(n)))
+        if ms < 0:
+            raise DirectorError(4, "director_kernel_time")
+        return ms, int(n.value)
+
+
+def status_string(status: int) -> str:
+    return load_library().director_status_string(status).decode()

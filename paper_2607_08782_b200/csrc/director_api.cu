@@ -1,0 +1,352 @@
+// C-ABI entry points of libdirector.so: argument checks, context life cycle, placement tables,
+// the host-buffer convenience call and the per-kernel timing hooks.  The kernels live in the
+// director_<stage>.cu files.
+#include "director_common.cuh"
+
+#include <cstring>
+#include <new>
+
+using namespace director;
+
+namespace director {
+int ffn_init(director_ctx* ctx);   // director_ffn.cu: shared-memory opt-in for the GEMM kernels
+}
+
+namespace {
+
+template <typename T>
+bool dev_alloc(T** p, size_t count) {
+    if (count == 0) count = 1;
+    return cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T)) == cudaSuccess;
+}
+
+bool shape_supported(const director_shape& s) {
+    if (s.T_max < 1 || s.H < 256 || s.F < 128 || s.E < 1 || s.K < 1 || s.S < 0 || s.R < 1 || s.C_max < 1) return false;
+    if (s.K > kMaxK || s.K > s.E || s.E > kMaxE || s.R > kMaxR || s.C_max > kMaxC) return false;
+    if ((long long)s.E > (long long)s.R * s.C_max) return false;
+    if (s.H % 256 != 0 || s.F % 128 != 0) return false;
+    if ((long long)s.T_max * s.K >= (1ll << 31)) return false;
+    if ((long long)s.E * s.F >= (1ll << 31) || (long long)s.E * s.H >= (1ll << 31)) return false;
+    return true;
+}
+
+void free_all(director_ctx* c) {
+    void* ptrs[] = {c->d_rep_start, c->d_rep_slot, c->d_slot_expert, c->d_tile_counts, c->d_seg_offsets, c->d_ticket,
+                    c->d_status, c->d_hidden, c->d_hidden_shared, c->d_one_seg,
+                    c->d_zero_expert, c->e_logits, c->e_x, c->e_topk_idx, c->e_topk_w, c->e_xp, c->e_yp, c->e_y,
+                    c->e_y_shared, c->e_row_token, c->e_inv_row, c->e_dest_rank, c->e_cost};
+    for (void* p : ptrs)
+        if (p) cudaFree(p);
+    for (auto& ev : c->events) { cudaEventDestroy(ev.start); cudaEventDestroy(ev.stop); }
+    for (auto& ev : c->free_events) { cudaEventDestroy(ev.start); cudaEventDestroy(ev.stop); }
+}
+
+inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
+
+#define REQUIRE_CTX(ctx)                              \
+    do {                                              \
+        if ((ctx) == nullptr) return DIRECTOR_ERR_INVALID_ARG; \
+    } while (0)
+#define REQUIRE_T(ctx, T)                                                   \
+    do {                                                                    \
+        if ((T) < 1 || (T) > (ctx)->shape.T_max) return DIRECTOR_ERR_INVALID_ARG; \
+    } while (0)
+#define REQUIRE_PTR(p)                                                      \
+    do {                                                                    \
+        if ((p) == nullptr || !aligned16(p)) return DIRECTOR_ERR_INVALID_ARG; \
+    } while (0)
+#define REQUIRE_PLACEMENT(ctx)                                   \
+    do {                                                         \
+        if (!(ctx)->placement_set) return DIRECTOR_ERR_PLACEMENT; \
+    } while (0)
+
+}  // namespace
+
+extern "C" {
+
+int director_create(const director_shape* shape, director_ctx** out) {
+    if (shape == nullptr || out == nullptr) return DIRECTOR_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!shape_supported(*shape)) return DIRECTOR_ERR_UNSUPPORTED;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    if (prop.major != 10) return DIRECTOR_ERR_UNSUPPORTED;   // tcgen05 / TMEM kernels: sm_100 only
+
+    director_ctx* c = new (std::nothrow) director_ctx();
+    if (c == nullptr) return DIRECTOR_ERR_WORKSPACE;
+    c->shape = *shape;
+    c->device = dev;
+    c->sm_count = prop.multiProcessorCount;
+    c->G = shape->R * shape->C_max;
+    c->n_tiles_max = (shape->T_max + kTokenTile - 1) / kTokenTile;
+    const director_shape& s = c->shape;
+    const size_t A = (size_t)s.T_max * s.K, T = (size_t)s.T_max;
+    const size_t cost_words = (size_t)s.R * s.E + s.R + 2 * (size_t)s.R * s.R;
+
+    bool ok = dev_alloc(&c->d_rep_start, s.E + 1) && dev_alloc(&c->d_rep_slot, (size_t)s.E * s.R) &&
+              dev_alloc(&c->d_slot_expert, c->G) && dev_alloc(&c->d_tile_counts, (size_t)c->n_tiles_max * s.E) &&
+              dev_alloc(&c->d_seg_offsets, c->G + 1) && dev_alloc(&c->d_ticket, 1) && dev_alloc(&c->d_status, 1) &&
+              dev_alloc(&c->d_one_seg, 2) &&
+              dev_alloc(&c->d_zero_expert, 1) &&
+              dev_alloc(reinterpret_cast<uint16_t**>(&c->d_hidden), A * s.F) &&
+              dev_alloc(reinterpret_cast<uint16_t**>(&c->d_hidden_shared), T * s.S * s.F) &&
+              dev_alloc(&c->e_logits, T * s.E) && dev_alloc(reinterpret_cast<uint16_t**>(&c->e_x), T * s.H) &&
+              dev_alloc(&c->e_topk_idx, A) && dev_alloc(&c->e_topk_w, A) &&
+              dev_alloc(reinterpret_cast<uint16_t**>(&c->e_xp), A * s.H) &&
+              dev_alloc(reinterpret_cast<uint16_t**>(&c->e_yp), A * s.H) &&
+              dev_alloc(reinterpret_cast<uint16_t**>(&c->e_y), T * s.H) &&
+              dev_alloc(reinterpret_cast<uint16_t**>(&c->e_y_shared), s.S > 0 ? T * s.H : 0) &&
+              dev_alloc(&c->e_row_token, A) && dev_alloc(&c->e_inv_row, A) && dev_alloc(&c->e_dest_rank, A) &&
+              dev_alloc(&c->e_cost, cost_words);
+    if (!ok) {
+        cudaGetLastError();
+        free_all(c);
+        delete c;
+        return DIRECTOR_ERR_WORKSPACE;
+    }
+    ok = cudaMemset(c->d_ticket, 0, sizeof(unsigned int)) == cudaSuccess &&
+         cudaMemset(c->d_status, 0, sizeof(int32_t)) == cudaSuccess &&
+         cudaMemset(c->d_zero_expert, 0, sizeof(int32_t)) == cudaSuccess;
+
+    cudaDriverEntryPointQueryResult qres;
+    if (ok) {
+        ok = cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &c->encode_tiled, 12000, cudaEnableDefault,
+                                              &qres) == cudaSuccess &&
+             qres == cudaDriverEntryPointSuccess && c->encode_tiled != nullptr;
+    }
+    if (ok) ok = ffn_init(c) == DIRECTOR_OK;
+    if (!ok) {
+        cudaGetLastError();
+        free_all(c);
+        delete c;
+        return DIRECTOR_ERR_CUDA;
+    }
+    *out = c;
+    return DIRECTOR_OK;
+}
+
+int director_destroy(director_ctx* ctx) {
+    REQUIRE_CTX(ctx);
+    cudaSetDevice(ctx->device);
+    cudaDeviceSynchronize();
+    free_all(ctx);
+    delete ctx;
+    return DIRECTOR_OK;
+}
+
+int director_set_placement(director_ctx* ctx, const uint8_t* X, void* stream) {
+    REQUIRE_CTX(ctx);
+    if (X == nullptr) return DIRECTOR_ERR_INVALID_ARG;
+    const director_shape& s = ctx->shape;
+    const int E = s.E, R = s.R, C = s.C_max;
+    std::vector<int32_t> rep_start(E + 1, 0), rep_slot, slot_expert((size_t)R * C, -1), slot_of((size_t)E * R, -1);
+    // hosted(j): experts on rank j in ascending id -> slots j*C + 0,1,...   (capacity: sum_i x_ij <= C_max)
+    for (int j = 0; j < R; ++j) {
+        int p = 0;
+        for (int e = 0; e < E; ++e) {
+            const uint8_t v = X[(size_t)e * R + j];
+            if (v > 1) return DIRECTOR_ERR_PLACEMENT;
+            if (v == 1) {
+                if (p >= C) return DIRECTOR_ERR_PLACEMENT;
+                slot_expert[(size_t)j * C + p] = e;
+                slot_of[(size_t)e * R + j] = j * C + p;
+                ++p;
+            }
+        }
+    }
+    // reps(e): hosting ranks in ascending order                          (assignment: sum_j x_ij >= 1)
+    for (int e = 0; e < E; ++e) {
+        rep_start[e] = (int32_t)rep_slot.size();
+        for (int j = 0; j < R; ++j)
+            if (slot_of[(size_t)e * R + j] >= 0) rep_slot.push_back(slot_of[(size_t)e * R + j]);
+        if ((int32_t)rep_slot.size() == rep_start[e]) return DIRECTOR_ERR_PLACEMENT;
+    }
+    rep_start[E] = (int32_t)rep_slot.size();
+    cudaStream_t st = as_stream(stream);
+    // pageable sources: the runtime stages them before returning, so the vectors may die here
+    if (cudaMemcpyAsync(ctx->d_rep_start, rep_start.data(), rep_start.size() * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(ctx->d_rep_slot, rep_slot.data(), rep_slot.size() * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(ctx->d_slot_expert, slot_expert.data(), slot_expert.size() * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return DIRECTOR_ERR_CUDA;
+    ctx->h_slot_expert = slot_expert;
+    ctx->placement_set = true;
+    return DIRECTOR_OK;
+}
+
+int director_route(director_ctx* ctx, int32_t T, const float* logits, int32_t* topk_idx, float* topk_w, void* stream) {
+    REQUIRE_CTX(ctx);
+    REQUIRE_T(ctx, T);
+    REQUIRE_PTR(logits);
+    REQUIRE_PTR(topk_idx);
+    REQUIRE_PTR(topk_w);
+    return launch_route(ctx, T, logits, topk_idx, topk_w, as_stream(stream));
+}
+
+int director_dispatch(director_ctx* ctx, int32_t T, const void* x, const int32_t* topk_idx, void* xp, int32_t* row_token,
+                      int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, void* stream) {
+    REQUIRE_CTX(ctx);
+    REQUIRE_T(ctx, T);
+    REQUIRE_PLACEMENT(ctx);
+    REQUIRE_PTR(x);
+    REQUIRE_PTR(topk_idx);
+    REQUIRE_PTR(xp);
+    REQUIRE_PTR(row_token);
+    REQUIRE_PTR(inv_row);
+    REQUIRE_PTR(dest_rank);
+    REQUIRE_PTR(seg_offsets);
+    return launch_dispatch(ctx, T, x, topk_idx, xp, row_token, inv_row, dest_rank, seg_offsets, as_stream(stream));
+}
+
+int director_expert_ffn(director_ctx* ctx, int32_t T, const void* xp, const int32_t* seg_offsets, const void* w_gate,
+                        const void* w_up, const void* w_down, void* yp, const void* x, const void* ws_gate,
+                        const void* ws_up, const void* ws_down, void* y_shared, void* stream) {
+    REQUIRE_CTX(ctx);
+    REQUIRE_T(ctx, T);
+    REQUIRE_PLACEMENT(ctx);
+    REQUIRE_PTR(xp);
+    REQUIRE_PTR(seg_offsets);
+    REQUIRE_PTR(w_gate);
+    REQUIRE_PTR(w_up);
+    REQUIRE_PTR(w_down);
+    REQUIRE_PTR(yp);
+    if (ctx->shape.S > 0 && x != nullptr) {
+        REQUIRE_PTR(x);
+        REQUIRE_PTR(ws_gate);
+        REQUIRE_PTR(ws_up);
+        REQUIRE_PTR(ws_down);
+        REQUIRE_PTR(y_shared);
+    }
+    return launch_expert_ffn(ctx, T, xp, seg_offsets, w_gate, w_up, w_down, yp, x, ws_gate, ws_up, ws_down, y_shared,
+                             as_stream(stream));
+}
+
+int director_combine(director_ctx* ctx, int32_t T, const void* yp, const int32_t* inv_row, const float* topk_w,
+                     const void* y_shared, void* y, void* stream) {
+    REQUIRE_CTX(ctx);
+    REQUIRE_T(ctx, T);
+    REQUIRE_PTR(yp);
+    REQUIRE_PTR(inv_row);
+    REQUIRE_PTR(topk_w);
+    REQUIRE_PTR(y);
+    if (y_shared != nullptr && !aligned16(y_shared)) return DIRECTOR_ERR_INVALID_ARG;
+    return launch_combine(ctx, T, yp, inv_row, topk_w, y_shared, y, as_stream(stream));
+}
+
+int director_placement_cost(director_ctx* ctx, int32_t T, const int32_t* topk_idx, const int32_t* token_src_rank,
+                            int64_t* workload, int64_t* rank_load, int64_t* dispatch_tokens, uint64_t* dispatch_bytes,
+                            void* stream) {
+    REQUIRE_CTX(ctx);
+    REQUIRE_T(ctx, T);
+    REQUIRE_PLACEMENT(ctx);
+    REQUIRE_PTR(topk_idx);
+    if (token_src_rank != nullptr && (reinterpret_cast<uintptr_t>(token_src_rank) & 3u)) return DIRECTOR_ERR_INVALID_ARG;
+    if (!workload || !rank_load || !dispatch_tokens || !dispatch_bytes) return DIRECTOR_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(workload) | reinterpret_cast<uintptr_t>(rank_load) |
+         reinterpret_cast<uintptr_t>(dispatch_tokens) | reinterpret_cast<uintptr_t>(dispatch_bytes)) & 7u)
+        return DIRECTOR_ERR_INVALID_ARG;
+    return launch_cost(ctx, T, topk_idx, token_src_rank, workload, rank_load, dispatch_tokens, dispatch_bytes,
+                       as_stream(stream));
+}
+
+int director_layer_forward_host(director_ctx* ctx, int32_t T, const float* logits, const void* x, const void* w_gate,
+                                const void* w_up, const void* w_down, const void* ws_gate, const void* ws_up,
+                                const void* ws_down, void* y, int64_t* rank_load, uint64_t* dispatch_bytes, void* stream) {
+    REQUIRE_CTX(ctx);
+    REQUIRE_T(ctx, T);
+    REQUIRE_PLACEMENT(ctx);
+    if (!logits || !x || !y) return DIRECTOR_ERR_INVALID_ARG;
+    REQUIRE_PTR(w_gate);
+    REQUIRE_PTR(w_up);
+    REQUIRE_PTR(w_down);
+    const director_shape& s = ctx->shape;
+    const bool shared = s.S > 0;
+    if (shared) {
+        REQUIRE_PTR(ws_gate);
+        REQUIRE_PTR(ws_up);
+        REQUIRE_PTR(ws_down);
+    }
+    cudaStream_t st = as_stream(stream);
+    int64_t* c_w = ctx->e_cost;
+    int64_t* c_load = c_w + (size_t)s.R * s.E;
+    int64_t* c_tok = c_load + s.R;
+    uint64_t* c_bytes = reinterpret_cast<uint64_t*>(c_tok + (size_t)s.R * s.R);
+
+    if (cudaMemcpyAsync(ctx->e_logits, logits, sizeof(float) * (size_t)T * s.E, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(ctx->e_x, x, 2 * (size_t)T * s.H, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return DIRECTOR_ERR_CUDA;
+    int rc = launch_route(ctx, T, ctx->e_logits, ctx->e_topk_idx, ctx->e_topk_w, st);
+    if (rc == DIRECTOR_OK)
+        rc = launch_dispatch(ctx, T, ctx->e_x, ctx->e_topk_idx, ctx->e_xp, ctx->e_row_token, ctx->e_inv_row,
+                             ctx->e_dest_rank, ctx->d_seg_offsets, st);
+    if (rc == DIRECTOR_OK)
+        rc = launch_expert_ffn(ctx, T, ctx->e_xp, ctx->d_seg_offsets, w_gate, w_up, w_down, ctx->e_yp,
+                               shared ? ctx->e_x : nullptr, ws_gate, ws_up, ws_down, ctx->e_y_shared, st);
+    if (rc == DIRECTOR_OK)
+        rc = launch_combine(ctx, T, ctx->e_yp, ctx->e_inv_row, ctx->e_topk_w, shared ? ctx->e_y_shared : nullptr,
+                            ctx->e_y, st);
+    if (rc == DIRECTOR_OK) rc = launch_cost(ctx, T, ctx->e_topk_idx, nullptr, c_w, c_load, c_tok, c_bytes, st);
+    if (rc != DIRECTOR_OK) return rc;
+    if (cudaMemcpyAsync(y, ctx->e_y, 2 * (size_t)T * s.H, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    if (rank_load && cudaMemcpyAsync(rank_load, c_load, sizeof(int64_t) * s.R, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return DIRECTOR_ERR_CUDA;
+    if (dispatch_bytes &&
+        cudaMemcpyAsync(dispatch_bytes, c_bytes, sizeof(uint64_t) * s.R * s.R, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return DIRECTOR_ERR_CUDA;
+    return cuda_status(cudaStreamSynchronize(st));
+}
+
+int director_last_status(director_ctx* ctx, void* stream) {
+    REQUIRE_CTX(ctx);
+    cudaStream_t st = as_stream(stream);
+    int32_t h = 0;
+    if (cudaMemcpyAsync(&h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    if (cudaMemsetAsync(ctx->d_status, 0, sizeof(h), st) != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    return h;
+}
+
+int64_t director_launch_count(const director_ctx* ctx) { return ctx ? ctx->launches : -1; }
+
+int director_set_profiling(director_ctx* ctx, int32_t enabled) {
+    REQUIRE_CTX(ctx);
+    if (cudaDeviceSynchronize() != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    for (auto& ev : ctx->events) ctx->free_events.push_back(ev);
+    ctx->events.clear();
+    ctx->profiling = enabled != 0;
+    return DIRECTOR_OK;
+}
+
+double director_kernel_time(director_ctx* ctx, const char* name_substr, int64_t* launches) {
+    if (ctx == nullptr || name_substr == nullptr) return -1.0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return -1.0;
+    double total = 0.0;
+    int64_t n = 0;
+    for (const auto& ev : ctx->events) {
+        if (std::strstr(ev.name, name_substr) == nullptr) continue;
+        float ms = 0.0f;
+        if (cudaEventElapsedTime(&ms, ev.start, ev.stop) != cudaSuccess) return -1.0;
+        total += ms;
+        ++n;
+    }
+    if (launches) *launches = n;
+    return total;
+}
+
+const char* director_status_string(int status) {
+    switch (status) {
+        case DIRECTOR_OK: return "ok";
+        case DIRECTOR_ERR_INVALID_ARG: return "invalid argument";
+        case DIRECTOR_ERR_PLACEMENT: return "invalid or missing expert placement";
+        case DIRECTOR_ERR_WORKSPACE: return "workspace allocation failed";
+        case DIRECTOR_ERR_CUDA: return "CUDA call failed";
+        case DIRECTOR_ERR_UNSUPPORTED: return "unsupported shape or device";
+        case DIRECTOR_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        case DIRECTOR_ERR_BAD_INDEX: return "expert or rank index out of range on the device";
+        case DIRECTOR_ERR_NONFINITE: return "non-finite router logit";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

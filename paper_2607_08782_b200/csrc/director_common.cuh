@@ -1,0 +1,129 @@
+// Internal definitions shared by the translation units of libdirector.so.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "director.h"
+
+namespace director {
+
+constexpr int kTokenTile = 256;   // tokens per CTA in the count / index kernels (8 warps)
+constexpr int kMaxE = 256;
+constexpr int kMaxK = 8;
+constexpr int kMaxR = 64;
+constexpr int kMaxC = 16;
+constexpr int kMaxG = kMaxR * kMaxC;
+
+struct KernelEvent {
+    const char* name;
+    cudaEvent_t start, stop;
+};
+
+}  // namespace director
+
+struct director_ctx {
+    director_shape shape{};
+    int device = 0;
+    int sm_count = 0;
+    int G = 0;            // R * C_max
+    int n_tiles_max = 0;  // ceil(T_max / kTokenTile)
+
+    // placement tables (device): replicas of expert e are rep_slot[rep_start[e] .. rep_start[e+1])
+    bool placement_set = false;
+    int32_t* d_rep_start = nullptr;    // [E+1]
+    int32_t* d_rep_slot = nullptr;     // [E*R] slot id of each replica, replicas by ascending rank
+    int32_t* d_slot_expert = nullptr;  // [G] expert of each slot or -1
+    std::vector<int32_t> h_slot_expert;
+
+    // dispatch / cost workspace
+    int32_t* d_tile_counts = nullptr;   // [n_tiles_max, E] per-tile expert counts -> exclusive prefix
+    int32_t* d_seg_offsets = nullptr;   // [G+1] internal copy (placement-cost path, host forward)
+    unsigned int* d_ticket = nullptr;   // last-CTA-done counter, self-resetting
+    int32_t* d_status = nullptr;        // sticky device status word
+
+    // expert FFN workspace
+    void* d_hidden = nullptr;          // bf16 [T_max*K, F]   SwiGLU activations of the routed experts
+    void* d_hidden_shared = nullptr;   // bf16 [T_max, S*F]
+    int32_t* d_one_seg = nullptr;      // [2] segment table {0, T} used for the shared experts
+    int32_t* d_zero_expert = nullptr;  // [1] = {0}
+
+    // buffers of director_layer_forward_host
+    float* e_logits = nullptr;
+    void* e_x = nullptr;
+    int32_t* e_topk_idx = nullptr;
+    float* e_topk_w = nullptr;
+    void* e_xp = nullptr;
+    void* e_yp = nullptr;
+    void* e_y = nullptr;
+    void* e_y_shared = nullptr;
+    int32_t* e_row_token = nullptr;
+    int32_t* e_inv_row = nullptr;
+    int32_t* e_dest_rank = nullptr;
+    int64_t* e_cost = nullptr;          // workload [R,E] | rank_load [R] | dispatch_tokens [R,R] | bytes [R,R]
+
+    void* encode_tiled = nullptr;       // cuTensorMapEncodeTiled, resolved through the runtime
+
+    int64_t launches = 0;
+    bool profiling = false;
+    std::vector<director::KernelEvent> events;
+    std::vector<director::KernelEvent> free_events;
+};
+
+namespace director {
+
+// Brackets one kernel launch: counts it and, when profiling is on, records events around it.
+struct LaunchScope {
+    director_ctx* ctx;
+    cudaStream_t stream;
+    KernelEvent ev{};
+    bool timed = false;
+    LaunchScope(director_ctx* c, cudaStream_t s, const char* name) : ctx(c), stream(s) {
+        ctx->launches++;
+        if (ctx->profiling) {
+            if (!ctx->free_events.empty()) {
+                ev = ctx->free_events.back();
+                ctx->free_events.pop_back();
+                timed = true;
+            } else {
+                timed = cudaEventCreate(&ev.start) == cudaSuccess && cudaEventCreate(&ev.stop) == cudaSuccess;
+            }
+            ev.name = name;
+            if (timed) cudaEventRecord(ev.start, stream);
+        }
+    }
+    ~LaunchScope() {
+        if (timed) {
+            cudaEventRecord(ev.stop, stream);
+            ctx->events.push_back(ev);
+        }
+    }
+};
+
+inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? DIRECTOR_OK : DIRECTOR_ERR_CUDA; }
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Stage launchers implemented in the individual translation units.  All validate nothing:
+// the extern "C" wrappers in director_api.cu check arguments first.
+int launch_route(director_ctx*, int T, const float* logits, int32_t* topk_idx, float* topk_w, cudaStream_t);
+int launch_dispatch(director_ctx*, int T, const void* x, const int32_t* topk_idx, void* xp, int32_t* row_token,
+                    int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, cudaStream_t);
+int launch_cost(director_ctx*, int T, const int32_t* topk_idx, const int32_t* src_rank, int64_t* workload,
+                int64_t* rank_load, int64_t* dispatch_tokens, uint64_t* dispatch_bytes, cudaStream_t);
+int launch_expert_ffn(director_ctx*, int T, const void* xp, const int32_t* seg_offsets, const void* w_gate,
+                      const void* w_up, const void* w_down, void* yp, const void* x, const void* ws_gate,
+                      const void* ws_up, const void* ws_down, void* y_shared, cudaStream_t);
+int launch_combine(director_ctx*, int T, const void* yp, const int32_t* inv_row, const float* topk_w,
+                   const void* y_shared, void* y, cudaStream_t);
+
+}  // namespace director
+
+// Device-side sticky status: keep the first error.
+__device__ __forceinline__ void director_set_status(int32_t* status, int32_t code) {
+    atomicCAS(status, 0, code);
+}

@@ -1,0 +1,296 @@
+// (a2) Placement-aware dispatch and (a5) placement cost.
+//
+// Dispatch (Section II-B: tokens are packaged and sent to the ranks hosting their experts) is an
+// on-device stable counting sort of the T*K (token, choice) assignments by (destination rank,
+// expert id, token id), followed by the row copies.  The same counting front-end feeds the
+// placement-cost histograms (Section VI-A: workload matrix W, Eq. 1 load, Eq. 3 dispatch volume).
+//
+// Kernels
+//   count_scan_kernel  per 256-token tile: per-expert counts from lane bitmasks; the last CTA to
+//                      finish (atomic ticket, no spinning) turns them into exclusive per-tile
+//                      prefixes, splits every expert's total over its replicas and scans the
+//                      slot lengths into seg_offsets.
+//   index_kernel       recomputes each assignment's stable rank inside its tile from the bitmasks,
+//                      adds the tile prefix, applies the round-robin replica rule and writes
+//                      inv_row / dest_rank / row_token.
+//   scatter_rows_kernel  one warp per (token, 2 KB column slice): one coalesced 16-byte-per-lane read
+//                      of x, K writes into xp.  HBM-bound: 2H + 2HK bytes per token.
+//   cost_kernel        same ranks -> destination rank; shared-memory histograms flushed with
+//                      integer atomics (order independent, hence deterministic).
+#include "director_common.cuh"
+
+namespace director {
+
+namespace {
+
+constexpr int kTileWarps = kTokenTile / 32;
+
+// Lane bitmasks: mask[e][w] has bit l set iff token (tile*256 + w*32 + l) chose expert e.
+__device__ __forceinline__ void build_masks(uint32_t (*mask)[kTileWarps], const int32_t* __restrict__ topk_idx,
+                                            int tile, int T, int E, int K, int32_t* status) {
+    for (int i = threadIdx.x; i < E * kTileWarps; i += blockDim.x) (&mask[0][0])[i] = 0u;
+    __syncthreads();
+    const int t = tile * kTokenTile + threadIdx.x;
+    if (t < T) {
+        const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        for (int s = 0; s < K; ++s) {
+            const int e = __ldg(topk_idx + (size_t)t * K + s);
+            if ((unsigned)e < (unsigned)E) atomicOr(&mask[e][w], 1u << lane);
+            else director_set_status(status, DIRECTOR_ERR_BAD_INDEX);
+        }
+    }
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(kTokenTile)
+count_scan_kernel(const int32_t* __restrict__ topk_idx, int T, int E, int K, int G, int n_tiles,
+                  const int32_t* __restrict__ rep_start, const int32_t* __restrict__ rep_slot,
+                  int32_t* __restrict__ tile_counts, int32_t* __restrict__ seg_offsets_a,
+                  int32_t* __restrict__ seg_offsets_b, unsigned int* __restrict__ ticket,
+                  int32_t* __restrict__ status) {
+    __shared__ uint32_t mask[kMaxE][kTileWarps];
+    __shared__ int32_t slot_len[kMaxG];
+    __shared__ int32_t warp_sum[kTileWarps];
+    __shared__ bool is_last;
+
+    const int tile = blockIdx.x;
+    build_masks(mask, topk_idx, tile, T, E, K, status);
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
+        int c = 0;
+#pragma unroll
+        for (int w = 0; w < kTileWarps; ++w) c += __popc(mask[e][w]);
+        tile_counts[(size_t)tile * E + e] = c;
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1u) == (unsigned)(n_tiles - 1));
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+
+    // ---- last CTA: per-expert exclusive scan over tiles, replica split, slot scan ----
+    for (int g = threadIdx.x; g < G; g += blockDim.x) slot_len[g] = 0;
+    __syncthreads();
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
+        int run = 0;
+        for (int i = 0; i < n_tiles; ++i) {
+            const int c = __ldcg(tile_counts + (size_t)i * E + e);
+            tile_counts[(size_t)i * E + e] = run;
+            run += c;
+        }
+        const int r0 = rep_start[e], r_e = rep_start[e + 1] - r0;
+        for (int q = 0; q < r_e; ++q)               // replica q gets ceil((N_e - q) / r_e) rows
+            slot_len[rep_slot[r0 + q]] = (run > q) ? (run - q + r_e - 1) / r_e : 0;
+    }
+    __syncthreads();
+    // exclusive scan of slot_len[0..G): each thread owns a contiguous chunk
+    const int per = (G + blockDim.x - 1) / blockDim.x;
+    const int lo = min(threadIdx.x * per, G), hi = min(lo + per, G);
+    int local = 0;
+    for (int g = lo; g < hi; ++g) local += slot_len[g];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_sum[w] = incl;
+    __syncthreads();
+    int base = incl - local;
+    for (int i = 0; i < w; ++i) base += warp_sum[i];
+    for (int g = lo; g < hi; ++g) {
+        seg_offsets_a[g] = base;
+        if (seg_offsets_b) seg_offsets_b[g] = base;
+        base += slot_len[g];
+    }
+    if (threadIdx.x == blockDim.x - 1) {
+        // the last thread's running total is the grand total T*K (minus skipped bad indices)
+        seg_offsets_a[G] = base;
+        if (seg_offsets_b) seg_offsets_b[G] = base;
+        *ticket = 0u;                                 // ready for the next call on this stream
+    }
+}
+
+// Stable rank of (token, expert e) among the tile's tokens that chose e.
+__device__ __forceinline__ int tile_rank(const uint32_t (*mask)[kTileWarps], const uint16_t (*warp_prefix)[kTileWarps],
+                                         int e, int w, int lane) {
+    return warp_prefix[e][w] + __popc(mask[e][w] & ((1u << lane) - 1u));
+}
+
+__device__ __forceinline__ void build_warp_prefix(const uint32_t (*mask)[kTileWarps], uint16_t (*warp_prefix)[kTileWarps], int E) {
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
+        int run = 0;
+#pragma unroll
+        for (int w = 0; w < kTileWarps; ++w) { warp_prefix[e][w] = (uint16_t)run; run += __popc(mask[e][w]); }
+    }
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(kTokenTile)
+index_kernel(const int32_t* __restrict__ topk_idx, int T, int E, int K, int C_max,
+             const int32_t* __restrict__ rep_start, const int32_t* __restrict__ rep_slot,
+             const int32_t* __restrict__ tile_prefix, const int32_t* __restrict__ seg_offsets,
+             int32_t* __restrict__ row_token, int32_t* __restrict__ inv_row, int32_t* __restrict__ dest_rank,
+             int32_t* __restrict__ status) {
+    __shared__ uint32_t mask[kMaxE][kTileWarps];
+    __shared__ uint16_t warp_prefix[kMaxE][kTileWarps];
+    const int tile = blockIdx.x;
+    build_masks(mask, topk_idx, tile, T, E, K, status);
+    build_warp_prefix(mask, warp_prefix, E);
+    const int t = tile * kTokenTile + threadIdx.x;
+    if (t >= T) return;
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int s = 0; s < K; ++s) {
+        const int e = __ldg(topk_idx + (size_t)t * K + s);
+        int row = -1, dest = -1;
+        if ((unsigned)e < (unsigned)E) {
+            const int n = __ldg(tile_prefix + (size_t)tile * E + e) + tile_rank(mask, warp_prefix, e, w, lane);
+            const int r0 = __ldg(rep_start + e), r_e = __ldg(rep_start + e + 1) - r0;
+            const int q = n % r_e, p = n / r_e;
+            const int slot = __ldg(rep_slot + r0 + q);
+            row = __ldg(seg_offsets + slot) + p;
+            dest = slot / C_max;
+            row_token[row] = t;
+        }
+        inv_row[(size_t)t * K + s] = row;
+        dest_rank[(size_t)t * K + s] = dest;
+    }
+}
+
+// One warp copies a 2 KB slice (4 x 16 bytes per lane) of row t of x to its K destination rows.
+constexpr int kSliceVec = 4;                       // uint4 per lane
+constexpr int kSliceBytes = 32 * 16 * kSliceVec;   // 2048
+constexpr int kScatterWarps = 8;
+
+__global__ void __launch_bounds__(kScatterWarps * 32)
+scatter_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ inv_row, uint4* __restrict__ xp,
+                    int T, int K, int row_vec /* uint4 per row */, int slices_per_row) {
+    const int lane = threadIdx.x & 31;
+    const long long item = (long long)blockIdx.x * kScatterWarps + (threadIdx.x >> 5);
+    if (item >= (long long)T * slices_per_row) return;
+    const int t = (int)(item / slices_per_row);
+    const int v0 = (int)(item % slices_per_row) * (32 * kSliceVec) + lane;
+    const uint4* src = x + (size_t)t * row_vec;
+    uint4 v[kSliceVec];
+#pragma unroll
+    for (int i = 0; i < kSliceVec; ++i)
+        if (v0 + 32 * i < row_vec) v[i] = __ldcs(src + v0 + 32 * i);
+    int my_row = (lane < K) ? __ldg(inv_row + (size_t)t * K + lane) : -1;
+    for (int s = 0; s < K; ++s) {
+        const int row = __shfl_sync(0xFFFFFFFFu, my_row, s);
+        if (row < 0) continue;
+        uint4* dst = xp + (size_t)row * row_vec;
+#pragma unroll
+        for (int i = 0; i < kSliceVec; ++i)
+            if (v0 + 32 * i < row_vec) dst[v0 + 32 * i] = v[i];
+    }
+}
+
+// Placement cost: per assignment (src rank j, expert e, destination rank k).
+__global__ void __launch_bounds__(kTokenTile)
+cost_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ src_rank, int T, int E, int K, int R,
+            int C_max, const int32_t* __restrict__ rep_start, const int32_t* __restrict__ rep_slot,
+            const int32_t* __restrict__ tile_prefix, unsigned long long* __restrict__ workload,
+            unsigned long long* __restrict__ rank_load, unsigned long long* __restrict__ dispatch_tokens,
+            unsigned long long* __restrict__ dispatch_bytes, unsigned long long bytes_per_token,
+            int32_t* __restrict__ status) {
+    __shared__ uint32_t mask[kMaxE][kTileWarps];
+    __shared__ uint16_t warp_prefix[kMaxE][kTileWarps];
+    __shared__ uint32_t h_rr[kMaxR * kMaxR];        // [src][dest]
+    __shared__ uint32_t h_load[kMaxR];
+    const int tile = blockIdx.x;
+    for (int i = threadIdx.x; i < R * R; i += blockDim.x) h_rr[i] = 0u;
+    for (int i = threadIdx.x; i < R; i += blockDim.x) h_load[i] = 0u;
+    build_masks(mask, topk_idx, tile, T, E, K, status);
+    build_warp_prefix(mask, warp_prefix, E);
+    const int t = tile * kTokenTile + threadIdx.x;
+    if (t < T) {
+        const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        int src = src_rank ? __ldg(src_rank + t) : (int)(((long long)t * R) / T);
+        if ((unsigned)src >= (unsigned)R) { director_set_status(status, DIRECTOR_ERR_BAD_INDEX); src = -1; }
+        for (int s = 0; s < K && src >= 0; ++s) {
+            const int e = __ldg(topk_idx + (size_t)t * K + s);
+            if ((unsigned)e >= (unsigned)E) continue;
+            const int n = __ldg(tile_prefix + (size_t)tile * E + e) + tile_rank(mask, warp_prefix, e, w, lane);
+            const int r0 = __ldg(rep_start + e), r_e = __ldg(rep_start + e + 1) - r0;
+            const int dest = __ldg(rep_slot + r0 + n % r_e) / C_max;
+            atomicAdd(&h_rr[src * R + dest], 1u);
+            atomicAdd(&h_load[dest], 1u);
+            atomicAdd(workload + (size_t)src * E + e, 1ull);
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < R * R; i += blockDim.x) {
+        const uint32_t c = h_rr[i];
+        if (c) {
+            atomicAdd(dispatch_tokens + i, (unsigned long long)c);
+            atomicAdd(dispatch_bytes + i, (unsigned long long)c * bytes_per_token);
+        }
+    }
+    for (int i = threadIdx.x; i < R; i += blockDim.x)
+        if (h_load[i]) atomicAdd(rank_load + i, (unsigned long long)h_load[i]);
+}
+
+int launch_count_scan(director_ctx* ctx, int T, const int32_t* topk_idx, int32_t* seg_a, int32_t* seg_b, cudaStream_t st) {
+    const director_shape& s = ctx->shape;
+    const int n_tiles = (T + kTokenTile - 1) / kTokenTile;
+    LaunchScope scope(ctx, st, "count_scan_kernel");
+    count_scan_kernel<<<n_tiles, kTokenTile, 0, st>>>(topk_idx, T, s.E, s.K, ctx->G, n_tiles, ctx->d_rep_start,
+                                                      ctx->d_rep_slot, ctx->d_tile_counts, seg_a, seg_b,
+                                                      ctx->d_ticket, ctx->d_status);
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace
+
+int launch_dispatch(director_ctx* ctx, int T, const void* x, const int32_t* topk_idx, void* xp, int32_t* row_token,
+                    int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, cudaStream_t st) {
+    const director_shape& s = ctx->shape;
+    const int n_tiles = (T + kTokenTile - 1) / kTokenTile;
+    int rc = launch_count_scan(ctx, T, topk_idx, seg_offsets, ctx->d_seg_offsets, st);
+    if (rc != DIRECTOR_OK) return rc;
+    {
+        LaunchScope scope(ctx, st, "index_kernel");
+        index_kernel<<<n_tiles, kTokenTile, 0, st>>>(topk_idx, T, s.E, s.K, s.C_max, ctx->d_rep_start, ctx->d_rep_slot,
+                                                     ctx->d_tile_counts, seg_offsets, row_token, inv_row, dest_rank,
+                                                     ctx->d_status);
+        rc = cuda_status(cudaGetLastError());
+        if (rc != DIRECTOR_OK) return rc;
+    }
+    {
+        const int row_vec = s.H * 2 / 16;
+        const int slices = (s.H * 2 + kSliceBytes - 1) / kSliceBytes;
+        const long long items = (long long)T * slices;
+        const unsigned grid = (unsigned)((items + kScatterWarps - 1) / kScatterWarps);
+        LaunchScope scope(ctx, st, "scatter_rows_kernel");
+        scatter_rows_kernel<<<grid, kScatterWarps * 32, 0, st>>>(static_cast<const uint4*>(x), inv_row,
+                                                                 static_cast<uint4*>(xp), T, s.K, row_vec, slices);
+        rc = cuda_status(cudaGetLastError());
+    }
+    return rc;
+}
+
+int launch_cost(director_ctx* ctx, int T, const int32_t* topk_idx, const int32_t* src_rank, int64_t* workload,
+                int64_t* rank_load, int64_t* dispatch_tokens, uint64_t* dispatch_bytes, cudaStream_t st) {
+    const director_shape& s = ctx->shape;
+    const int n_tiles = (T + kTokenTile - 1) / kTokenTile;
+    cudaError_t e;
+    if ((e = cudaMemsetAsync(workload, 0, sizeof(int64_t) * s.R * s.E, st)) != cudaSuccess) return cuda_status(e);
+    if ((e = cudaMemsetAsync(rank_load, 0, sizeof(int64_t) * s.R, st)) != cudaSuccess) return cuda_status(e);
+    if ((e = cudaMemsetAsync(dispatch_tokens, 0, sizeof(int64_t) * s.R * s.R, st)) != cudaSuccess) return cuda_status(e);
+    if ((e = cudaMemsetAsync(dispatch_bytes, 0, sizeof(uint64_t) * s.R * s.R, st)) != cudaSuccess) return cuda_status(e);
+    int rc = launch_count_scan(ctx, T, topk_idx, ctx->d_seg_offsets, nullptr, st);
+    if (rc != DIRECTOR_OK) return rc;
+    LaunchScope scope(ctx, st, "cost_kernel");
+    cost_kernel<<<n_tiles, kTokenTile, 0, st>>>(topk_idx, src_rank, T, s.E, s.K, s.R, s.C_max, ctx->d_rep_start,
+                                                ctx->d_rep_slot, ctx->d_tile_counts,
+                                                reinterpret_cast<unsigned long long*>(workload),
+                                                reinterpret_cast<unsigned long long*>(rank_load),
+                                                reinterpret_cast<unsigned long long*>(dispatch_tokens),
+                                                reinterpret_cast<unsigned long long*>(dispatch_bytes),
+                                                (unsigned long long)s.H * 2ull, ctx->d_status);
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace director

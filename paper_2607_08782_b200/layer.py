@@ -1,0 +1,79 @@
+"""Device-tensor convenience around the C entry points: owns the output tensors of one MoE layer
+and calls the five stages in order on the current stream.  Allocation and marshalling only."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from .binding import Director
+
+
+def bf16_bits_to_tensor(bits: np.ndarray, device="cuda") -> torch.Tensor:
+    """uint16 bf16 bit patterns (numpy) -> torch.bfloat16 tensor on `device` (bit-exact)."""
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16))
+    return t.to(device).view(torch.bfloat16)
+
+
+def tensor_to_bf16_bits(t: torch.Tensor) -> np.ndarray:
+    return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+class MoELayer:
+    """Routed experts w_gate/w_up [E,F,H], w_down [E,H,F]; optional shared experts ws_gate/ws_up [S*F,H],
+    ws_down [H,S*F] (all torch.bfloat16 CUDA tensors, kept by reference)."""
+
+    def __init__(self, T_max, H, F, E, K, S, R, C_max, w_gate, w_up, w_down, ws_gate=None, ws_up=None,
+                 ws_down=None, device="cuda"):
+        self.dims = dict(T_max=T_max, H=H, F=F, E=E, K=K, S=S, R=R, C_max=C_max)
+        self.d = Director(T_max, H, F, E, K, S, R, C_max)
+        self.w = (w_gate, w_up, w_down)
+        self.ws = (ws_gate, ws_up, ws_down)
+        A, G = T_max * K, R * C_max
+        i32 = dict(dtype=torch.int32, device=device)
+        self.topk_idx = torch.empty((T_max, K), **i32)
+        self.topk_w = torch.empty((T_max, K), dtype=torch.float32, device=device)
+        self.xp = torch.empty((A, H), dtype=torch.bfloat16, device=device)
+        self.yp = torch.empty((A, H), dtype=torch.bfloat16, device=device)
+        self.row_token = torch.empty((A,), **i32)
+        self.inv_row = torch.empty((T_max, K), **i32)
+        self.dest_rank = torch.empty((T_max, K), **i32)
+        self.seg_offsets = torch.empty((G + 1,), **i32)
+        self.y = torch.empty((T_max, H), dtype=torch.bfloat16, device=device)
+        self.y_shared = torch.empty((T_max, H), dtype=torch.bfloat16, device=device) if S > 0 else None
+        i64 = dict(dtype=torch.int64, device=device)
+        self.workload = torch.empty((R, E), **i64)
+        self.rank_load = torch.empty((R,), **i64)
+        self.dispatch_tokens = torch.empty((R, R), **i64)
+        self.dispatch_bytes = torch.empty((R, R), **i64)     # bit pattern of uint64
+
+    def set_placement(self, X: np.ndarray):
+        self.d.set_placement(X)
+
+    def route(self, T, logits):
+        self.d.route(T, logits, self.topk_idx, self.topk_w)
+
+    def dispatch(self, T, x):
+        self.d.dispatch(T, x, self.topk_idx, self.xp, self.row_token, self.inv_row, self.dest_rank, self.seg_offsets)
+
+    def expert_ffn(self, T, x=None):
+        S = self.dims["S"]
+        self.d.expert_ffn(T, self.xp, self.seg_offsets, *self.w, self.yp,
+                          x if S > 0 else None, *(self.ws if S > 0 else (None, None, None)),
+                          self.y_shared if S > 0 else None)
+
+    def combine(self, T):
+        self.d.combine(T, self.yp, self.inv_row, self.topk_w, self.y_shared, self.y)
+
+    def placement_cost(self, T, token_src_rank=None):
+        self.d.placement_cost(T, self.topk_idx, token_src_rank, self.workload, self.rank_load,
+                              self.dispatch_tokens, self.dispatch_bytes)
+
+    def forward(self, T, logits, x, with_cost=True):
+        """One pass of the whole layer on device tensors; returns y[:T] (a view of the owned buffer)."""
+        self.route(T, logits)
+        self.dispatch(T, x)
+        self.expert_ffn(T, x)
+        self.combine(T)
+        if with_cost:
+            self.placement_cost(T)
+        return self.y[:T]

@@ -1,0 +1,230 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Integer outputs (routing indices, permutation, segment offsets, histograms) must be
+bit-exact; weights within 1e-6; bf16 layer outputs within relative L2 <= 1e-2 and max abs <= 5e-2."""
+import numpy as np
+import pytest
+
+from oracle import director_oracle as orc
+from paper_2607_08782_b200 import synth
+
+from gpu_harness import (GpuCase, check_integer_parity, max_abs, oracle_layer_tokens, rel_l2, sample_tokens)
+
+pytestmark = pytest.mark.gpu
+
+REL_L2_TOL = 1e-2      # relative L2 error of bf16 outputs against the fp64 oracle
+MAX_ABS_TOL = 5e-2     # max abs error
+W_TOL = 1e-6           # gating weights, absolute
+
+
+def _oracle_front(shape, logits, x_bits, X, C_max, src=None):
+    idx, w, w64 = orc.route(logits, shape.K)
+    d = orc.dispatch(idx, X, C_max, x_bits)
+    c = orc.placement_cost(idx, X, C_max, shape.H, src)
+    return idx, w, w64, d, c
+
+
+def _check_outputs(shape, g, x_bits, weights, idx, w, w64, d, c, tokens, label):
+    assert g.status == 0, f"{label}: device status {g.status}"
+    check_integer_parity(g, idx, d, c, label)
+    assert np.max(np.abs(g.topk_w.astype(np.float64) - w64)) <= W_TOL, f"{label}: gating weights"
+    assert np.max(np.abs(g.topk_w.astype(np.float64).sum(axis=1) - 1.0)) <= W_TOL
+    assert np.array_equal(g.xp, d["xp"]), f"{label}: permuted rows are not exact copies"
+    y_o, rows, yp_o, ysh_o = oracle_layer_tokens(shape, x_bits, weights, idx, w64, d, tokens)
+    yp_g = orc.bf16_to_f64(g.yp[rows])
+    y_g = orc.bf16_to_f64(g.y[tokens])
+    e = dict(yp_rel=rel_l2(yp_g, yp_o), yp_max=max_abs(yp_g, yp_o), y_rel=rel_l2(y_g, y_o), y_max=max_abs(y_g, y_o))
+    if ysh_o is not None:
+        ys_g = orc.bf16_to_f64(g.y_shared[tokens])
+        e.update(ysh_rel=rel_l2(ys_g, ysh_o), ysh_max=max_abs(ys_g, ysh_o))
+    print(label, {k: f"{v:.3e}" for k, v in e.items()})
+    for k, v in e.items():
+        assert v <= (REL_L2_TOL if k.endswith("rel") else MAX_ABS_TOL), f"{label}: {k} = {v:.3e}"
+    return e
+
+
+def test_c1_tiny_full_tensor_parity():
+    wl = synth.make_workload("c1_tiny")
+    s = wl.shape
+    case = GpuCase(s, wl.logits, wl.x, wl.weights)
+    g = case.run(wl.X_primary)
+    idx, w, w64, d, c = _oracle_front(s, wl.logits, wl.x, wl.X_primary, s.C_max)
+    _check_outputs(s, g, wl.x, wl.weights, idx, w, w64, d, c, np.arange(s.T), "c1")
+
+
+def _custom(seed, T, H, E, K, F, S, R, C, zipf=1.2):
+    shape = synth.Shape(f"custom{seed}", T, H, E, K, F, S, R, C, zipf, seed)
+    return shape, synth.make_logits(shape), synth.make_x(shape), synth.make_weights(shape)
+
+
+def _random_placement(seed, E, R, C, extra):
+    rng = np.random.default_rng(seed)
+    X = np.zeros((E, R), dtype=np.uint8)
+    slots = [j for j in range(R) for _ in range(C)]
+    rng.shuffle(slots)
+    for e in range(E):
+        X[e, slots[e]] = 1
+    for _ in range(extra):
+        free = [(e, j) for e in range(E) for j in range(R) if not X[e, j] and X[:, j].sum() < C]
+        if not free:
+            break
+        e, j = free[rng.integers(len(free))]
+        X[e, j] = 1
+    return X
+
+
+@pytest.mark.parametrize("seed,T,H,E,K,F,S,R,C,extra", [
+    (11, 777, 256, 12, 3, 384, 0, 4, 4, 4),      # several 256-token tiles and a ragged tail, replicas
+    (12, 1000, 512, 60, 4, 256, 2, 8, 8, 4),     # E not a multiple of 32, shared experts
+    (13, 300, 256, 5, 5, 128, 0, 2, 5, 5),       # K == E, every expert replicated everywhere
+    (14, 1, 256, 8, 2, 128, 1, 4, 2, 0),         # a single token
+    (15, 513, 768, 128, 8, 256, 0, 16, 9, 16),   # Qwen3-like routing sizes, many empty segments
+    (16, 260, 256, 256, 8, 128, 0, 64, 4, 0),    # the largest supported E and R
+])
+def test_small_cases_full_tensor_parity(seed, T, H, E, K, F, S, R, C, extra):
+    shape, logits, x, weights = _custom(seed, T, H, E, K, F, S, R, C)
+    X = _random_placement(seed, E, R, C, extra)
+    src = (synth.raw_u64(seed, 50, 0, T) % np.uint64(R)).astype(np.int32) if seed % 2 else None
+    case = GpuCase(shape, logits, x, weights)
+    g = case.run(X, src=src)
+    idx, w, w64, d, c = _oracle_front(shape, logits, x, X, C, src)
+    _check_outputs(shape, g, x, weights, idx, w, w64, d, c, np.arange(T), f"custom{seed}")
+
+
+def test_degenerate_routing_all_tokens_to_the_same_experts():
+    shape, logits, x, weights = _custom(21, 600, 256, 8, 2, 256, 0, 4, 3, 1.2)
+    logits[:] = 0.0                       # all ties: every token picks experts 0 and 1, weights 1/2
+    X = synth.placement_from_ranks(np.arange(8) // 2, 4)
+    X[0, 2] = X[0, 3] = 1                 # expert 0 on three ranks: its 600 rows split 200/200/200
+    case = GpuCase(shape, logits, x, weights)
+    g = case.run(X)
+    idx, w, w64, d, c = _oracle_front(shape, logits, x, X, 3)
+    assert np.array_equal(g.topk_idx, np.tile(np.array([0, 1], dtype=np.int32), (600, 1)))
+    _check_outputs(shape, g, x, weights, idx, w, w64, d, c, np.arange(600), "degenerate")
+
+
+def test_identity_round_trip_dispatch_then_combine():
+    """combine(dispatch(x)) == x bit-exactly when the experts are the identity (yp := xp)."""
+    wl = synth.make_workload("c1_tiny")
+    s = wl.shape
+    case = GpuCase(s, wl.logits, wl.x, wl.weights)
+    L, T = case.layer, s.T
+    L.set_placement(wl.X_primary)
+    L.route(T, case.logits)
+    L.dispatch(T, case.x)
+    L.d.combine(T, L.xp, L.inv_row, L.topk_w, None, L.y)
+    case.torch.cuda.synchronize()
+    from paper_2607_08782_b200.layer import tensor_to_bf16_bits
+    assert np.array_equal(tensor_to_bf16_bits(L.y[:T]), wl.x)
+
+
+def test_tie_breaks_and_signed_zero():
+    shape, logits, x, weights = _custom(31, 64, 256, 8, 3, 128, 0, 4, 2, 1.2)
+    logits[:] = np.round(logits)          # many exact ties
+    logits[0] = [-0.0, 0.0, -1.0, 0.0, -5, -5, -5, -5]
+    X = synth.placement_from_ranks(np.arange(8) // 2, 4)
+    case = GpuCase(shape, logits, x, weights)
+    g = case.run(X, stages="front")
+    idx, w, w64 = orc.route(logits, 3)
+    assert np.array_equal(g.topk_idx, idx)
+    assert g.topk_idx[0].tolist() == [0, 1, 3]
+    assert np.max(np.abs(g.topk_w - w64)) <= W_TOL
+
+
+def test_layer_output_is_bitwise_invariant_to_placement():
+    """Placement moves experts between ranks, never changes what a token computes."""
+    wl = synth.make_workload("c1_tiny")
+    s = wl.shape
+    case = GpuCase(s, wl.logits, wl.x, wl.weights, C_max=4)
+    y0 = case.run(wl.X_primary).y
+    for seed in (1, 2, 3):
+        X = _random_placement(seed, s.E, s.R, 4, 2 * seed)
+        assert np.array_equal(case.run(X).y, y0)
+
+
+def test_results_are_reproducible_run_to_run():
+    shape, logits, x, weights = _custom(41, 2000, 256, 64, 6, 128, 0, 8, 9, 1.2)
+    X = _random_placement(41, 64, 8, 9, 8)
+    case = GpuCase(shape, logits, x, weights)
+    a, b = case.run(X), case.run(X)
+    for name in ("topk_idx", "row_token", "inv_row", "dest_rank", "seg_offsets", "workload", "rank_load",
+                 "dispatch_tokens", "dispatch_bytes", "y"):
+        assert np.array_equal(getattr(a, name), getattr(b, name)), name
+
+
+def test_device_side_faults_set_the_sticky_status_without_trapping():
+    import torch
+    shape, logits, x, weights = _custom(51, 64, 256, 8, 2, 128, 0, 4, 2, 1.2)
+    case = GpuCase(shape, logits, x, weights)
+    L = case.layer
+    L.set_placement(synth.placement_from_ranks(np.arange(8) // 2, 4))
+    bad = case.logits.clone()
+    bad[3, 1] = float("nan")
+    L.route(64, bad)
+    assert L.d.last_status() == 8          # DIRECTOR_ERR_NONFINITE, then cleared
+    assert L.d.last_status() == 0
+    L.route(64, case.logits)
+    L.topk_idx[5, 0] = 99                  # expert id outside [0, E): assignment skipped, flag raised
+    L.dispatch(64, case.x)
+    assert L.d.last_status() == 7          # DIRECTOR_ERR_BAD_INDEX
+    torch.cuda.synchronize()
+    assert int(L.inv_row[5, 0]) == -1 and int(L.seg_offsets[-1]) == 64 * 2 - 1
+
+
+# ---------------------------------------------------------------------------------------------
+# the paper-shaped workloads at full size: integer parity on the whole batch, floating-point
+# parity on the first/last token of every segment plus seeded random tokens (all their K
+# assignments and the shared experts), placement invariance on the whole output tensor.
+# ---------------------------------------------------------------------------------------------
+
+def _full_size(name, T, placements, n_random=48):
+    wl = synth.make_workload(name, T)
+    s = wl.shape
+    case = GpuCase(s, wl.logits, wl.x, wl.weights)
+    idx, w, w64 = orc.route(wl.logits, s.K)
+    N = np.bincount(idx.ravel(), minlength=s.E)
+    y_first = None
+    for pname, make in placements:
+        X = make(N, wl, s)
+        g = case.run(X)
+        d = orc.dispatch(idx, X, s.C_max, wl.x)
+        c = orc.placement_cost(idx, X, s.C_max, s.H)
+        tokens = sample_tokens(d, s.T, n_random, s.seed)
+        _check_outputs(s, g, wl.x, wl.weights, idx, w, w64, d, c, tokens, f"{name}/T={s.T}/{pname}")
+        assert c["rank_load"].sum() == s.T * s.K
+        if y_first is None:
+            y_first = g.y
+        else:
+            assert np.array_equal(g.y, y_first), f"{name}: output depends on placement"
+
+
+def _primary(N, wl, s):
+    return wl.X_primary
+
+
+def _hot2(N, wl, s):
+    return orc.replicate_hottest(N, wl.X_primary, 2)
+
+
+def _fill_spare(N, wl, s):
+    return orc.balanced_placement(N, s.R, s.C_max, synth.primary_ranks(s))
+
+
+def _balanced(N, wl, s):
+    return orc.balanced_placement(N, s.R, s.C_max)
+
+
+def test_c2_mixtral_shaped():
+    _full_size("c2_mixtral", None, [("one-per-rank", _primary), ("hot2-replicated", _hot2)], n_random=24)
+
+
+def test_c3_deepseek_v2_lite_shaped():
+    _full_size("c3_dsv2lite", None, [("primaries", _primary), ("spare-filled", _fill_spare)])
+
+
+def test_c4_qwen15_shaped():
+    _full_size("c4_qwen15", None, [("primaries", _primary), ("spare-filled", _fill_spare)])
+
+
+@pytest.mark.parametrize("T", synth.C5_SWEEP)
+def test_c5_qwen3_shaped_sweep(T):
+    _full_size("c5_qwen3", T, [("round-robin", _primary), ("load-balanced", _balanced)])
