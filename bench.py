@@ -1,0 +1,483 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE layer forward under an expert placement (route -> dispatch -> grouped SwiGLU
+expert FFN -> combine -> placement cost) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c2_mixtral] [--impl ours|reference]
+
+One "step" is one pass of the whole layer over one batch of seeded synthetic input.  The default
+workload is the Mixtral-8x7B-shaped layer (4096 tokens, hidden 4096, 8 experts top-2, FFN 14336, 8
+logical ranks, the two hottest experts replicated).  Prints ONE JSON line (rank 0).
+
+With N > 1 (launched under torch.distributed.run) every rank runs an independent replica of the layer on
+its own GPU - the path has no inter-GPU exchange - and the value is the aggregate over ranks divided by
+the slowest rank's time ("weak" scaling).
+
+--impl reference times the CPU oracle (the plain fp64 restatement of the method) on the host cores, on a
+bounded sample of the same workload per step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import signal
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "moe_layer_tokens_per_s"
+UNIT = "tokens/s"
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
+# from the ncu captures summarised under profiles/ (None until a capture for that workload exists).
+NCU_TRAFFIC_BYTES = {}
+
+
+# ------------------------------------------------------------------------------------------------
+# clock sampling (child process; NVML, read only)
+# ------------------------------------------------------------------------------------------------
+
+REASON_BITS = {
+    0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+    0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+    0x100: "display_clock_setting",
+}
+
+
+def _sample_clocks_main(uuid: str, out_path: str, period_s: float = 0.02):
+    """Child process: polls SM clock, power and clock-event reasons of one GPU until SIGTERM."""
+    import pynvml
+    pynvml.nvmlInit()
+    h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if isinstance(uuid, str) else uuid)
+    stop = {"now": False}
+    signal.signal(signal.SIGTERM, lambda *_: stop.__setitem__("now", True))
+    max_sm = pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM)
+    with open(out_path, "w") as f:
+        f.write(f"max {max_sm}\n")
+        while not stop["now"]:
+            sm = pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)
+            try:
+                reasons = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
+            except Exception:
+                reasons = pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+            try:
+                power = pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0
+            except Exception:
+                power = -1.0
+            f.write(f"{time.time():.4f} {sm} {reasons} {power:.1f}\n")
+            f.flush()
+            time.sleep(period_s)
+
+
+class ClockSampler:
+    def __init__(self, uuid: str):
+        self.path = tempfile.mktemp(prefix="director_clocks_", suffix=".txt")
+        self.proc = subprocess.Popen([sys.executable, os.path.abspath(__file__), "--sample-clocks", uuid, self.path],
+                                     stdout=subprocess.DEVNULL, stderr=subprocess.DEVNULL)
+        for _ in range(200):                      # wait until the child has written its header
+            if os.path.exists(self.path) and os.path.getsize(self.path) > 0:
+                break
+            time.sleep(0.02)
+
+    def stop(self, t0: float, t1: float) -> dict:
+        self.proc.send_signal(signal.SIGTERM)
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        try:
+            lines = open(self.path).read().split("\n")
+            os.unlink(self.path)
+        except OSError:
+            return out
+        sm, bits, power = [], 0, []
+        for ln in lines:
+            p = ln.split()
+            if len(p) == 2 and p[0] == "max":
+                out["sm_max_mhz"] = int(p[1])
+            elif len(p) == 4 and t0 <= float(p[0]) <= t1:
+                sm.append(int(p[1]))
+                bits |= int(p[2])
+                power.append(float(p[3]))
+        if sm:
+            out["sm_mhz"] = statistics.median(sm)
+            out["samples"] = len(sm)
+            out["power_w_max"] = max(power)
+            out["reasons"] = [name for bit, name in REASON_BITS.items() if bits & bit and name != "gpu_idle"]
+        return out
+
+
+# ------------------------------------------------------------------------------------------------
+# workload
+# ------------------------------------------------------------------------------------------------
+
+WORKLOAD_TEXT = {
+    "c1_tiny": "tiny MoE layer: 64 tokens, hidden 256, 8 experts top-2, FFN 512, 4 ranks x 2 slots, seeded random placement",
+    "c2_mixtral": "Mixtral-8x7B-shaped layer: 4096 tokens, hidden 4096, 8 experts top-2, SwiGLU FFN 14336, "
+                  "8 logical ranks, 2 hottest experts replicated",
+    "c3_dsv2lite": "DeepSeek-V2-Lite-shaped layer: 8192 tokens, hidden 2048, 64 experts top-6 + 2 shared, FFN 1408, "
+                   "8 ranks x 9 slots, spare slots filled by greedy replication",
+    "c4_qwen15": "Qwen1.5-MoE-A2.7B-shaped layer: 16384 tokens, hidden 2048, 60 experts top-4 + 4 shared, FFN 1408, "
+                 "8 ranks x 8 slots, popularity shifting every 512 tokens",
+    "c5_qwen3": "Qwen3-30B-A3B-shaped layer: hidden 2048, 128 experts top-8, FFN 768, 16 ranks x 9 slots, "
+                "greedy load-balanced placement",
+}
+
+
+def algorithmic_work(s, T):
+    """Bytes / FLOP the method itself must move or compute for one batch (per-token figures times T)."""
+    A = T * s.K
+    return {
+        "route_bytes": T * (4 * s.E + 8 * s.K),
+        "dispatch_bytes": T * (2 * s.H + 2 * s.H * s.K + 16 * s.K),
+        "combine_bytes": T * (2 * s.H * s.K + 8 * s.K + 2 * s.H + (2 * s.H if s.S > 0 else 0)),
+        "cost_bytes": T * 8 * s.K,
+        "gemm1_flop": 4 * s.H * s.F * A,            # gate and up projections
+        "gemm2_flop": 2 * s.H * s.F * A,            # down projection
+        "shared_flop": 6 * s.H * s.F * s.S * T,
+        "ffn_flop": 6 * s.H * s.F * (A + T * s.S),
+    }
+
+
+def build_layer(args, device):
+    """Generates the workload on the host, uploads it, derives the placement through the product path
+    (route -> placement-cost histogram -> greedy helper) and returns everything the timed loops need."""
+    import numpy as np
+    import torch
+    from paper_2607_08782_b200 import placement, synth
+    from paper_2607_08782_b200.layer import MoELayer, bf16_bits_to_tensor
+
+    wl = synth.make_workload(args.config, args.tokens)
+    s, w = wl.shape, wl.weights
+    wg, wu, wd = (bf16_bits_to_tensor(a, device) for a in (w.w_gate, w.w_up, w.w_down))
+    sg = su = sd = None
+    if s.S > 0:
+        sg = bf16_bits_to_tensor(w.ws_gate.reshape(s.S * s.F, s.H), device)
+        su = bf16_bits_to_tensor(w.ws_up.reshape(s.S * s.F, s.H), device)
+        sd = bf16_bits_to_tensor(synth.concat_shared_down(w.ws_down), device)
+    layer = MoELayer(s.T, s.H, s.F, s.E, s.K, s.S, s.R, s.C_max, wg, wu, wd, sg, su, sd, device)
+    logits = torch.from_numpy(wl.logits).to(device)
+    x = bf16_bits_to_tensor(wl.x, device)
+
+    # placement from the layer's own histograms of this batch (ground-truth routing)
+    layer.set_placement(wl.X_primary)
+    layer.route(s.T, logits)
+    layer.placement_cost(s.T)
+    torch.cuda.synchronize()
+    N = placement.expert_counts(layer.workload.cpu().numpy())
+    if args.placement == "primary" or s.name == "c1_tiny":
+        X, pname = wl.X_primary, "primary"
+    elif s.name == "c2_mixtral":
+        X, pname = placement.replicate_hottest(N, wl.X_primary, 2), "2 hottest experts replicated"
+    elif s.name == "c5_qwen3":
+        X, pname = placement.greedy_balanced(N, s.R, s.C_max), "greedy load-balanced"
+    else:
+        X, pname = placement.greedy_balanced(N, s.R, s.C_max, synth.primary_ranks(s)), "primaries + greedy replicas"
+    layer.set_placement(X)
+    return wl, layer, logits, x, X, pname
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs (cpu_baseline and --impl reference)
+# ------------------------------------------------------------------------------------------------
+
+def oracle_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return 1
+
+
+def oracle_weights(wl):
+    """The oracle's parameters decoded once into its compute precision (fp64), the counterpart of the
+    GPU path's weights being resident in HBM before the timed region."""
+    from oracle import director_oracle as orc
+    from paper_2607_08782_b200.synth import Weights
+    w = wl.weights
+    dec = lambda a: None if a is None else orc.bf16_to_f64(a)
+    return Weights(dec(w.w_gate), dec(w.w_up), dec(w.w_down), dec(w.ws_gate), dec(w.ws_up), dec(w.ws_down))
+
+
+def oracle_step(wl, w, X, n_tokens):
+    """The oracle, as it stands, on the first n_tokens tokens of the batch as a batch of their own."""
+    from oracle import director_oracle as orc
+    s = wl.shape
+    logits, x = wl.logits[:n_tokens], wl.x[:n_tokens]
+    idx, _, w64 = orc.route(logits, s.K)
+    d = orc.dispatch(idx, X, s.C_max, x)
+    yp = orc.expert_ffn(d["xp"], d["seg_offsets"], d["slot_expert"], w.w_gate, w.w_up, w.w_down)
+    ysh = orc.shared_ffn(x, w.ws_gate, w.ws_up, w.ws_down) if s.S > 0 else None
+    y = orc.combine(yp, d["inv_row"], w64, ysh)
+    orc.placement_cost(idx, X, s.C_max, s.H)
+    return y
+
+
+def oracle_sample_tokens(s, target_flop):
+    """Sub-batch size whose fp64 FFN work is about target_flop (a few seconds on a many-core host)."""
+    per_token = 6.0 * s.H * s.F * (s.K + s.S)
+    n = int(max(1, min(s.T, target_flop // per_token)))
+    return n
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    from paper_2607_08782_b200 import synth
+    from oracle import director_oracle as orc
+    wl = synth.make_workload(args.config, args.tokens)
+    s = wl.shape
+    idx, _, _ = orc.route(wl.logits, s.K)
+    N = np.bincount(idx.ravel(), minlength=s.E)
+    if s.name == "c2_mixtral":
+        X = orc.replicate_hottest(N, wl.X_primary, 2)
+    elif s.name == "c5_qwen3":
+        X = orc.balanced_placement(N, s.R, s.C_max)
+    elif s.name == "c1_tiny":
+        X = wl.X_primary
+    else:
+        X = orc.balanced_placement(N, s.R, s.C_max, synth.primary_ranks(s))
+    n = oracle_sample_tokens(s, 2.0e11)
+    w64 = oracle_weights(wl)
+    for _ in range(args.warmup):
+        oracle_step(wl, w64, X, n)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(wl, w64, X, n)
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt
+    cores = oracle_threads()
+    sample = f"each step = the oracle on the first {n} of {s.T} tokens as a batch of their own (all stages, fp64)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD_TEXT[args.config], "tokens": s.T, "sample_tokens_per_step": n},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------------------------
+# main (CUDA arm)
+# ------------------------------------------------------------------------------------------------
+
+STAGE_KERNELS = {
+    "route": ["route_topk_kernel"],
+    "dispatch": ["dispatch_count_scan_kernel", "dispatch_index_kernel", "dispatch_scatter_rows_kernel"],
+    "expert_ffn": ["grouped_gemm_swiglu_kernel", "grouped_gemm_down_kernel", "one_segment_kernel"],
+    "combine": ["combine_kernel"],
+    "placement_cost": ["cost_count_scan_kernel", "cost_kernel"],
+}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="c2_mixtral", choices=sorted(WORKLOAD_TEXT))
+    ap.add_argument("--tokens", type=int, default=None, help="batch size override (c5_qwen3 sweep: 1, 64, 1024, 32768)")
+    ap.add_argument("--placement", default="auto", choices=["auto", "primary"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sample-clocks", nargs=2, metavar=("UUID", "PATH"), help=argparse.SUPPRESS)
+    args = ap.parse_args()
+    if args.sample_clocks:
+        _sample_clocks_main(*args.sample_clocks)
+        return
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the layer has no CPU implementation")
+    torch.cuda.set_device(local_rank)
+    device = f"cuda:{local_rank}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(device))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    wl, layer, logits, x, X, pname = build_layer(args, device)
+    s = wl.shape
+    T = s.T
+    peaks = measured_peaks()
+
+    # ---- device-resident throughput ----
+    for _ in range(max(args.warmup, 3)):
+        layer.forward(T, logits, x)
+    torch.cuda.synchronize()
+    layer.d.check_device_status()
+
+    sampler = None
+    if rank == 0:
+        try:
+            uuid = str(torch.cuda.get_device_properties(local_rank).uuid)
+            sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+        except Exception:
+            sampler = None
+    # keep the GPU busy while the sampler starts so that the first samples see load clocks
+    for _ in range(3):
+        layer.forward(T, logits, x)
+    barrier()
+    torch.cuda.synchronize()
+    layer.d.set_profiling(True)
+    n0 = layer.d.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wall0 = time.time()
+    ev0.record()
+    for _ in range(args.steps):
+        layer.forward(T, logits, x)
+    ev1.record()
+    torch.cuda.synchronize()
+    wall1 = time.time()
+    barrier()
+    launches = layer.d.launch_count() - n0
+    ms_total = ev0.elapsed_time(ev1)
+    clocks = sampler.stop(wall0, wall1) if sampler else {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+    kernel_ms = {}
+    for names in STAGE_KERNELS.values():
+        for k in names:
+            ms, n = layer.d.kernel_time(k)
+            if n:
+                kernel_ms[k] = (ms / n, n // args.steps)
+    layer.d.set_profiling(False)
+    layer.d.check_device_status()
+    if world > 1:
+        t = torch.tensor([ms_total], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = world * T * args.steps / (ms_total * 1e-3)
+
+    # ---- end to end through the host-buffer entry point ----
+    h_logits = torch.from_numpy(wl.logits).pin_memory()
+    h_x = torch.from_numpy(wl.x.view(np.int16)).pin_memory()
+    h_y = torch.empty((T, s.H), dtype=torch.int16).pin_memory()
+    h_load = torch.empty((s.R,), dtype=torch.int64).pin_memory()
+    h_bytes = torch.empty((s.R, s.R), dtype=torch.int64).pin_memory()
+
+    def e2e_step():
+        layer.d.layer_forward_host(T, h_logits, h_x, *layer.w, *layer.ws, h_y, h_load, h_bytes)
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    layer.d.check_device_status()
+    # the host-path result must be the same bits as the device-path result
+    same = bool(torch.equal(h_y.cuda().view(torch.bfloat16), layer.y[:T]))
+    e2e = {"value": world * T * args.steps / (e2e_ms * 1e-3), "unit": UNIT,
+           "h2d_bytes_per_step": int(h_logits.numel() * 4 + h_x.numel() * 2),
+           "d2h_bytes_per_step": int(h_y.numel() * 2 + h_load.numel() * 8 + h_bytes.numel() * 8),
+           "ms_per_step": e2e_ms / args.steps, "matches_device_path": same,
+           "api": "director_layer_forward_host (pinned host logits/x in, y + histograms out)"}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel and per-stage figures ----
+    work = algorithmic_work(s, T)
+    dom = "grouped_gemm_swiglu_kernel"
+    dom_ms, dom_per_step = kernel_ms.get(dom, (None, 0))
+    shared_frac = work["shared_flop"] / work["ffn_flop"] if work["ffn_flop"] else 0.0
+    # with shared experts the kernel is launched twice per step (routed + shared); flops per launch averaged
+    gemm1_flop_per_launch = (work["gemm1_flop"] + work["shared_flop"] * 2 / 3) / max(dom_per_step, 1)
+    achieved = gemm1_flop_per_launch / (dom_ms * 1e-3) / 1e12 if dom_ms else None
+    peak = peaks["bf16_tflops_sustained"]
+    roofline = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": (achieved / peak) if achieved else None,
+                "traffic": NCU_TRAFFIC_BYTES.get(args.config),
+                "peak_source": f"{peaks['source']} cuBLAS bf16, sustained (kernel timed inside the step)",
+                "flop_per_launch": gemm1_flop_per_launch, "ms_per_launch": dom_ms,
+                "frac_of_burst_peak": (achieved / peaks["bf16_tflops"]) if achieved else None}
+
+    def stage_ms(stage):
+        return sum(kernel_ms[k][0] * kernel_ms[k][1] for k in STAGE_KERNELS[stage] if k in kernel_ms)
+
+    stages = {}
+    for stage, key, unit in (("route", "route_bytes", "GB/s"), ("dispatch", "dispatch_bytes", "GB/s"),
+                             ("combine", "combine_bytes", "GB/s"), ("placement_cost", "cost_bytes", "GB/s"),
+                             ("expert_ffn", "ffn_flop", "TFLOP/s")):
+        ms = stage_ms(stage)
+        if ms <= 0:
+            continue
+        rate = work[key] / (ms * 1e-3) / (1e9 if unit == "GB/s" else 1e12)
+        pk = peaks["hbm_gbs"] if unit == "GB/s" else peaks["bf16_tflops_sustained"]
+        stages[stage] = {"ms": round(ms, 4), "rate": round(rate, 2), "unit": unit, "frac_of_measured_peak": round(rate / pk, 4)}
+    kernels = {k: {"ms_per_launch": round(v[0], 4), "launches_per_step": v[1]} for k, v in kernel_ms.items()}
+
+    # ---- CPU baseline: the oracle on a bounded sample, on this machine's host cores ----
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        n = oracle_sample_tokens(s, 2.0e12)
+        w64 = oracle_weights(wl)
+        t0 = time.perf_counter()
+        oracle_step(wl, w64, X, n)
+        dt = time.perf_counter() - t0
+        cpu_baseline = {"value": n / dt, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                        "sample": f"the oracle (all stages, fp64, weights pre-decoded to fp64) on the first {n} of {T} "
+                                  f"tokens as a batch of their own, one run, {dt:.1f} s", "host_cpus": os.cpu_count()}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD_TEXT[args.config], "tokens": T, "placement": pname,
+                   "l2": "inputs larger than L2: every step streams the expert weights "
+                         f"({3 * s.E * s.F * s.H * 2 / 1e9:.2f} GB) and activations through HBM",
+                   "parallelism": "single GPU, logical ranks" if world == 1 else f"{world} independent replicas"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+        "cpu_baseline": cpu_baseline, "stages": stages, "kernels": kernels,
+        "ffn_tflops": round(work["ffn_flop"] / (stage_ms("expert_ffn") * 1e-3) / 1e12, 1) if stage_ms("expert_ffn") else None,
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -27,8 +27,13 @@ import numpy as np
 # ----------------------------------------------------------------------------------------------
 
 def bf16_to_f64(bits: np.ndarray) -> np.ndarray:
-    """Exact value of bf16 bit patterns (uint16) as fp64."""
-    return (np.asarray(bits).astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    """Exact value of bf16 bit patterns (uint16) as fp64.  Arrays that are already fp64 pass through,
+    so callers may decode their weights once and keep them resident in the compute precision."""
+    bits = np.asarray(bits)
+    if bits.dtype == np.float64:
+        return bits
+    assert bits.dtype == np.uint16
+    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
 
 
 def f64_to_bf16_bits(v: np.ndarray) -> np.ndarray:
@@ -177,7 +182,7 @@ def dispatch(topk_idx: np.ndarray, X: np.ndarray, C_max: int, x_bits: np.ndarray
 def swiglu_ffn_rows(rows_f64: np.ndarray, wg_bits, wu_bits, wd_bits) -> np.ndarray:
     """One expert on a block of rows, fp64 throughout, no intermediate rounding:
     g = rows . Wg^T, u = rows . Wu^T, a = g/(1+exp(-g)) * u, out = a . Wd^T.
-    wg, wu: [F,H] bf16 bits; wd: [H,F] bf16 bits."""
+    wg, wu: [F,H]; wd: [H,F]; bf16 bits or already-decoded fp64."""
     wg, wu, wd = bf16_to_f64(wg_bits), bf16_to_f64(wu_bits), bf16_to_f64(wd_bits)
     g = rows_f64 @ wg.T
     u = rows_f64 @ wu.T

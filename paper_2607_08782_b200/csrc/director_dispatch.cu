@@ -232,10 +232,11 @@ cost_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ sr
         if (h_load[i]) atomicAdd(rank_load + i, (unsigned long long)h_load[i]);
 }
 
-int launch_count_scan(director_ctx* ctx, int T, const int32_t* topk_idx, int32_t* seg_a, int32_t* seg_b, cudaStream_t st) {
+int launch_count_scan(director_ctx* ctx, const char* name, int T, const int32_t* topk_idx, int32_t* seg_a, int32_t* seg_b,
+                      cudaStream_t st) {
     const director_shape& s = ctx->shape;
     const int n_tiles = (T + kTokenTile - 1) / kTokenTile;
-    LaunchScope scope(ctx, st, "count_scan_kernel");
+    LaunchScope scope(ctx, st, name);
     count_scan_kernel<<<n_tiles, kTokenTile, 0, st>>>(topk_idx, T, s.E, s.K, ctx->G, n_tiles, ctx->d_rep_start,
                                                       ctx->d_rep_slot, ctx->d_tile_counts, seg_a, seg_b,
                                                       ctx->d_ticket, ctx->d_status);
@@ -248,10 +249,10 @@ int launch_dispatch(director_ctx* ctx, int T, const void* x, const int32_t* topk
                     int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, cudaStream_t st) {
     const director_shape& s = ctx->shape;
     const int n_tiles = (T + kTokenTile - 1) / kTokenTile;
-    int rc = launch_count_scan(ctx, T, topk_idx, seg_offsets, ctx->d_seg_offsets, st);
+    int rc = launch_count_scan(ctx, "dispatch_count_scan_kernel", T, topk_idx, seg_offsets, ctx->d_seg_offsets, st);
     if (rc != DIRECTOR_OK) return rc;
     {
-        LaunchScope scope(ctx, st, "index_kernel");
+        LaunchScope scope(ctx, st, "dispatch_index_kernel");
         index_kernel<<<n_tiles, kTokenTile, 0, st>>>(topk_idx, T, s.E, s.K, s.C_max, ctx->d_rep_start, ctx->d_rep_slot,
                                                      ctx->d_tile_counts, seg_offsets, row_token, inv_row, dest_rank,
                                                      ctx->d_status);
@@ -263,7 +264,7 @@ int launch_dispatch(director_ctx* ctx, int T, const void* x, const int32_t* topk
         const int slices = (s.H * 2 + kSliceBytes - 1) / kSliceBytes;
         const long long items = (long long)T * slices;
         const unsigned grid = (unsigned)((items + kScatterWarps - 1) / kScatterWarps);
-        LaunchScope scope(ctx, st, "scatter_rows_kernel");
+        LaunchScope scope(ctx, st, "dispatch_scatter_rows_kernel");
         scatter_rows_kernel<<<grid, kScatterWarps * 32, 0, st>>>(static_cast<const uint4*>(x), inv_row,
                                                                  static_cast<uint4*>(xp), T, s.K, row_vec, slices);
         rc = cuda_status(cudaGetLastError());
@@ -280,7 +281,7 @@ int launch_cost(director_ctx* ctx, int T, const int32_t* topk_idx, const int32_t
     if ((e = cudaMemsetAsync(rank_load, 0, sizeof(int64_t) * s.R, st)) != cudaSuccess) return cuda_status(e);
     if ((e = cudaMemsetAsync(dispatch_tokens, 0, sizeof(int64_t) * s.R * s.R, st)) != cudaSuccess) return cuda_status(e);
     if ((e = cudaMemsetAsync(dispatch_bytes, 0, sizeof(uint64_t) * s.R * s.R, st)) != cudaSuccess) return cuda_status(e);
-    int rc = launch_count_scan(ctx, T, topk_idx, ctx->d_seg_offsets, nullptr, st);
+    int rc = launch_count_scan(ctx, "cost_count_scan_kernel", T, topk_idx, ctx->d_seg_offsets, nullptr, st);
     if (rc != DIRECTOR_OK) return rc;
     LaunchScope scope(ctx, st, "cost_kernel");
     cost_kernel<<<n_tiles, kTokenTile, 0, st>>>(topk_idx, src_rank, T, s.E, s.K, s.R, s.C_max, ctx->d_rep_start,
