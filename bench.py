@@ -36,7 +36,10 @@ UNIT = "tokens/s"
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
 # from the ncu captures summarised under profiles/ (None until a capture for that workload exists).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/grouped_gemm_dram_c2_mixtral.md: gate||up GEMM, full-size workload, 2 435 702 016 B read + 227 459 584 B written
+    "c2_mixtral": 2663161600,
+}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -293,8 +296,8 @@ def measured_peaks():
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c2_mixtral", choices=sorted(WORKLOAD_TEXT))
     ap.add_argument("--tokens", type=int, default=None, help="batch size override (c5_qwen3 sweep: 1, 64, 1024, 32768)")
@@ -453,7 +456,7 @@ def main():
     # ---- CPU baseline: the oracle on a bounded sample, on this machine's host cores ----
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
-        n = oracle_sample_tokens(s, 2.0e12)
+        n = oracle_sample_tokens(s, 1.5e13)
         w64 = oracle_weights(wl)
         t0 = time.perf_counter()
         oracle_step(wl, w64, X, n)
