@@ -55,7 +55,8 @@ typedef enum {
     DIRECTOR_ERR_UNSUPPORTED = 5,   /* shape outside the supported ranges, or not an sm_100 GPU */
     DIRECTOR_ERR_TIMEOUT = 6,       /* device: a bounded wait inside a kernel expired           */
     DIRECTOR_ERR_BAD_INDEX = 7,     /* device: expert id outside [0,E) met (element skipped)    */
-    DIRECTOR_ERR_NONFINITE = 8      /* device: NaN/Inf router logit met                         */
+    DIRECTOR_ERR_NONFINITE = 8,     /* device: NaN/Inf router logit met                         */
+    DIRECTOR_ERR_STATIC_LIMIT = 9   /* problem larger than the fixed scratch of a *_static call */
 } director_status;
 
 typedef struct {
@@ -129,6 +130,36 @@ int director_combine(director_ctx* ctx, int32_t T, const void* yp, const int32_t
 int director_placement_cost(director_ctx* ctx, int32_t T, const int32_t* topk_idx,
                             const int32_t* token_src_rank, int64_t* workload, int64_t* rank_load,
                             int64_t* dispatch_tokens, uint64_t* dispatch_bytes, void* stream);
+
+/* Dispatch indices without a context and without any allocation.  (The paper has no counterpart:
+ * this entry point exists for the library's users, not for the method.)
+ *
+ * director_create allocates its workspace, so it is closed to callers that must never call
+ * cudaMalloc: code embedded in a host application that owns the device heap, latency-critical loops
+ * that may not block on the allocator, processes running under a fixed memory reservation.  This
+ * call computes the same permutation as director_dispatch (everything except the row copies) and
+ * performs no cudaMalloc, cudaFree or other allocating call, on any invocation.  Its scratch (launch
+ * ticket, status word, per-tile expert counts) is a fixed 1 MiB array inside the library image that
+ * each device holds from library load to process exit.
+ *
+ * Inputs, all dev: topk_idx int32 [T,K]; the placement as replica tables: rep_start int32 [E+1]
+ * (exclusive prefix of replica counts, rep_start[0] = 0) and rep_slot int32 [rep_start[E]], the slot
+ * g = rank*C_max + p of each replica, an expert's replicas in ascending rank order (slot numbering as
+ * in the header comment; the caller builds the tables, they are not validated).
+ * Outputs, all dev: row_token int32 [T*K], inv_row int32 [T,K], dest_rank int32 [T,K], seg_offsets
+ * int32 [R*C_max+1], exactly as director_dispatch writes them.  device_status: dev int32 [1] that the
+ * caller has zeroed, receives DIRECTOR_ERR_BAD_INDEX if an expert id outside [0,E) was skipped; may be
+ * NULL (the flag is then kept in the scratch and lost).
+ * Limits: ceil(T/256) * E <= 262080 (e.g. T <= 524032 at E = 128), otherwise DIRECTOR_ERR_STATIC_LIMIT
+ * is returned and nothing is launched; K, E, R, C_max within the ranges of the header comment.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress); make
+ * that first call outside any stream capture.  All calls on a device share the one array and it
+ * keeps the previous call's contents: the call clears what must start at zero itself, but two calls
+ * whose kernels overlap on the GPU (different streams, no dependency) race on it - serialise them. */
+int director_dispatch_index_static(int32_t T, int32_t K, int32_t E, int32_t R, int32_t C_max,
+                                   const int32_t* topk_idx, const int32_t* rep_start, const int32_t* rep_slot,
+                                   int32_t* row_token, int32_t* inv_row, int32_t* dest_rank,
+                                   int32_t* seg_offsets, int32_t* device_status, void* stream);
 
 /* The whole layer for callers that hold their batch in host memory: copies logits and x to the
  * device, runs (a1)-(a5) on context-owned buffers and copies y and the histograms back, all

@@ -14,7 +14,7 @@ from . import build as _build
 STATUS_NAMES = {
     0: "DIRECTOR_OK", 1: "DIRECTOR_ERR_INVALID_ARG", 2: "DIRECTOR_ERR_PLACEMENT", 3: "DIRECTOR_ERR_WORKSPACE",
     4: "DIRECTOR_ERR_CUDA", 5: "DIRECTOR_ERR_UNSUPPORTED", 6: "DIRECTOR_ERR_TIMEOUT", 7: "DIRECTOR_ERR_BAD_INDEX",
-    8: "DIRECTOR_ERR_NONFINITE",
+    8: "DIRECTOR_ERR_NONFINITE", 9: "DIRECTOR_ERR_STATIC_LIMIT",
 }
 
 # every symbol include/director.h declares
@@ -22,7 +22,7 @@ EXPORTED = (
     "director_create", "director_destroy", "director_set_placement", "director_route", "director_dispatch",
     "director_expert_ffn", "director_combine", "director_placement_cost", "director_layer_forward_host",
     "director_last_status", "director_launch_count", "director_set_profiling", "director_kernel_time",
-    "director_status_string",
+    "director_status_string", "director_dispatch_index_static",
 )
 
 
@@ -57,6 +57,7 @@ def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.director_combine.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp]
     lib.director_placement_cost.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp, vp]
     lib.director_layer_forward_host.argtypes = [vp, c_int32] + [vp] * 12
+    lib.director_dispatch_index_static.argtypes = [c_int32] * 5 + [vp] * 9
     lib.director_last_status.argtypes = [vp, vp]
     lib.director_launch_count.argtypes = [vp]
     lib.director_launch_count.restype = c_int64
@@ -177,3 +178,13 @@ class Director:
 
 def status_string(status: int) -> str:
     return load_library().director_status_string(status).decode()
+
+
+def dispatch_index_static(T, K, E, R, C_max, topk_idx, rep_start, rep_slot, row_token, inv_row, dest_rank,
+                          seg_offsets, device_status=None):
+    """Context-free, allocation-free dispatch indices (director_dispatch_index_static): for callers
+    that may not allocate device memory.  All tensor arguments are caller-owned CUDA int32 tensors."""
+    st = load_library().director_dispatch_index_static(
+        T, K, E, R, C_max, _ptr(topk_idx), _ptr(rep_start), _ptr(rep_slot), _ptr(row_token), _ptr(inv_row),
+        _ptr(dest_rank), _ptr(seg_offsets), _ptr(device_status), _stream())
+    _check(st, "director_dispatch_index_static")

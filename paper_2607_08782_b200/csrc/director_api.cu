@@ -345,6 +345,7 @@ const char* director_status_string(int status) {
         case DIRECTOR_ERR_TIMEOUT: return "a bounded device-side wait expired";
         case DIRECTOR_ERR_BAD_INDEX: return "expert or rank index out of range on the device";
         case DIRECTOR_ERR_NONFINITE: return "non-finite router logit";
+        case DIRECTOR_ERR_STATIC_LIMIT: return "problem exceeds the fixed scratch of an allocation-free call";
         default: return "unknown status";
     }
 }

@@ -295,3 +295,66 @@ int launch_cost(director_ctx* ctx, int T, const int32_t* topk_idx, const int32_t
 }
 
 }  // namespace director
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant of the dispatch index computation.
+//
+// Some hosts of this library may not call cudaMalloc at all: a plugin running inside an engine
+// that owns the whole device heap, a real-time loop that must not take the allocator lock, a
+// process whose memory budget was handed out up front.  Such callers cannot create a
+// director_ctx (creation allocates the workspace).  For them the counting sort keeps its
+// scratch - the launch ticket, a status word and the per-tile expert counts - in the fixed
+// array below, which every device that loads the library carries until the process exits.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticScratchInts = 262144;   // 1 MiB
+constexpr int kStaticHeaderInts = 64;        // [0] launch ticket, [1] status word, rest reserved
+static __device__ __align__(256) int32_t g_static_scratch[kStaticScratchInts];
+
+constexpr int kStaticMaxDevices = 64;
+int32_t* g_static_scratch_addr[kStaticMaxDevices] = {};   // device address of the array, per device
+
+}  // namespace
+
+extern "C" int director_dispatch_index_static(int32_t T, int32_t K, int32_t E, int32_t R, int32_t C_max,
+                                              const int32_t* topk_idx, const int32_t* rep_start,
+                                              const int32_t* rep_slot, int32_t* row_token, int32_t* inv_row,
+                                              int32_t* dest_rank, int32_t* seg_offsets, int32_t* device_status,
+                                              void* stream) {
+    using namespace director;
+    if (T < 1 || K < 1 || K > kMaxK || E < K || E > kMaxE || R < 1 || R > kMaxR || C_max < 1 || C_max > kMaxC)
+        return DIRECTOR_ERR_INVALID_ARG;
+    if ((long long)T * K >= (1ll << 31)) return DIRECTOR_ERR_INVALID_ARG;
+    if (!topk_idx || !rep_start || !rep_slot || !row_token || !inv_row || !dest_rank || !seg_offsets)
+        return DIRECTOR_ERR_INVALID_ARG;
+    const int n_tiles = (T + kTokenTile - 1) / kTokenTile;
+    if ((long long)n_tiles * E > kStaticScratchInts - kStaticHeaderInts) return DIRECTOR_ERR_STATIC_LIMIT;
+
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    if (dev < 0 || dev >= kStaticMaxDevices) return DIRECTOR_ERR_UNSUPPORTED;
+    if (g_static_scratch_addr[dev] == nullptr) {
+        // One-time set-up on this device (the first call on a device should precede any stream capture).
+        // In host code the array's name is only a handle; the kernels need its device address.
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return DIRECTOR_ERR_CUDA;
+        g_static_scratch_addr[dev] = static_cast<int32_t*>(p);
+    }
+    int32_t* scratch = g_static_scratch_addr[dev];
+    unsigned int* ticket = reinterpret_cast<unsigned int*>(scratch);
+    int32_t* status = device_status ? device_status : scratch + 1;
+    int32_t* tile_counts = scratch + kStaticHeaderInts;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    // The array keeps whatever the previous call left: the ticket must start at zero (the tile
+    // counts are fully rewritten by the first kernel before they are read).
+    if (cudaMemsetAsync(scratch, 0, kStaticHeaderInts * sizeof(int32_t), st) != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    const int G = R * C_max;
+    count_scan_kernel<<<n_tiles, kTokenTile, 0, st>>>(topk_idx, T, E, K, G, n_tiles, rep_start, rep_slot, tile_counts,
+                                                      seg_offsets, nullptr, ticket, status);
+    if (cudaGetLastError() != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    index_kernel<<<n_tiles, kTokenTile, 0, st>>>(topk_idx, T, E, K, C_max, rep_start, rep_slot, tile_counts, seg_offsets,
+                                                 row_token, inv_row, dest_rank, status);
+    return cuda_status(cudaGetLastError());
+}

@@ -1,0 +1,88 @@
+"""The allocation-free dispatch-index entry point (director_dispatch_index_static).
+
+Callers that are not allowed to allocate device memory - code living inside an engine that owns the
+device heap, loops that must never wait on the allocator, processes with a fixed memory reservation -
+cannot create a context, because creating one allocates its workspace.  This entry point keeps its
+scratch in a fixed array inside the library instead.  The test calls it through the C ABI twice in a
+row, on two different batches, and requires bit-identical results to director_dispatch (the existing,
+context-based entry point), and that the device's free memory does not change across the calls.
+
+The file name makes pytest collect it after every other test file."""
+import numpy as np
+import pytest
+
+from paper_2607_08782_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _replica_tables(X, C_max):
+    """rep_start [E+1], rep_slot [sum of replicas]: slot = rank*C_max + position of the expert among the
+    rank's hosted experts (ascending id); an expert's replicas in ascending rank order."""
+    E, R = X.shape
+    pos = np.cumsum(X, axis=0) - 1                 # position of expert e among the experts of rank j
+    rep_start, rep_slot = [0], []
+    for e in range(E):
+        for j in range(R):
+            if X[e, j]:
+                rep_slot.append(j * C_max + int(pos[e, j]))
+        rep_start.append(len(rep_slot))
+    return np.array(rep_start, dtype=np.int32), np.array(rep_slot, dtype=np.int32)
+
+
+def test_static_entry_point_matches_director_dispatch_on_two_calls_in_a_row():
+    import torch
+    from paper_2607_08782_b200 import binding
+    from paper_2607_08782_b200.layer import MoELayer
+
+    E, K, R, C, H, F = 60, 4, 8, 9, 256, 128
+    X = synth.placement_from_ranks(np.arange(E) % R, R)
+    X[3, 5] = X[3, 6] = X[17, 0] = X[59, 2] = 1           # a few replicas
+    rep_start, rep_slot = _replica_tables(X, C)
+    dev = "cuda"
+    w = torch.zeros((E, F, H), dtype=torch.bfloat16, device=dev)
+    wd = torch.zeros((E, H, F), dtype=torch.bfloat16, device=dev)
+    layer = MoELayer(3000, H, F, E, K, 0, R, C, w, w, wd, device=dev)
+    layer.set_placement(X)
+    d_start = torch.from_numpy(rep_start).to(dev)
+    d_slot = torch.from_numpy(rep_slot).to(dev)
+
+    for call, (T, seed) in enumerate([(3000, 71), (1237, 72)]):
+        shape = synth.Shape("na", T, H, E, K, F, 0, R, C, 1.3, seed)
+        logits = torch.from_numpy(synth.make_logits(shape)).to(dev)
+        x = torch.zeros((T, H), dtype=torch.bfloat16, device=dev)
+        layer.route(T, logits)
+        layer.dispatch(T, x)                                   # existing entry point
+        A = T * K
+        row_token = torch.full((A,), -7, dtype=torch.int32, device=dev)
+        inv_row = torch.full((T, K), -7, dtype=torch.int32, device=dev)
+        dest_rank = torch.full((T, K), -7, dtype=torch.int32, device=dev)
+        seg_offsets = torch.full((R * C + 1,), -7, dtype=torch.int32, device=dev)
+        status = torch.zeros((1,), dtype=torch.int32, device=dev)
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
+        binding.dispatch_index_static(T, K, E, R, C, layer.topk_idx, d_start, d_slot, row_token, inv_row,
+                                      dest_rank, seg_offsets, status)
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        if call > 0:                                           # the first call may load the module's image
+            assert free_after == free_before, "the allocation-free entry point changed the free device memory"
+        assert int(status.item()) == 0
+        assert torch.equal(seg_offsets, layer.seg_offsets), f"call {call}: seg_offsets"
+        assert torch.equal(row_token, layer.row_token[:A]), f"call {call}: row_token"
+        assert torch.equal(inv_row, layer.inv_row[:T]), f"call {call}: inv_row"
+        assert torch.equal(dest_rank, layer.dest_rank[:T]), f"call {call}: dest_rank"
+        assert int(seg_offsets[-1]) == A
+
+
+def test_static_entry_point_rejects_problems_beyond_its_fixed_scratch():
+    import torch
+    from paper_2607_08782_b200 import binding
+    lib = binding.load_library()
+    t = torch.zeros((16,), dtype=torch.int32, device="cuda")
+    p = t.data_ptr()
+    # ceil(T/256) * E must fit the 1 MiB array: 600000 tokens at E = 128 do not
+    rc = lib.director_dispatch_index_static(600000, 2, 128, 16, 9, p, p, p, p, p, p, p, None, None)
+    assert rc == 9 and "fixed scratch" in binding.status_string(rc)
+    assert lib.director_dispatch_index_static(0, 2, 128, 16, 9, p, p, p, p, p, p, p, None, None) == 1
+    assert lib.director_dispatch_index_static(64, 2, 128, 16, 9, None, p, p, p, p, p, p, None, None) == 1
