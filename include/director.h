@@ -162,8 +162,8 @@ int director_dispatch_index_static(int32_t T, int32_t K, int32_t E, int32_t R, i
                                    int32_t* seg_offsets, int32_t* device_status, void* stream);
 
 /* The whole layer for callers that hold their batch in host memory: copies logits and x to the
- * device, runs (a1)-(a5) on context-owned buffers and copies y and the histograms back, all
- * on `stream`; synchronises `stream` before returning.
+ * device, runs (a1)-(a5) on context-owned buffers and copies y and the histograms back; returns
+ * when the results are in the host buffers (director_layer_submit_host + director_layer_wait_host).
  * logits: host fp32 [T,E].  x: host bf16 [T,H].  Weights: dev, as for director_expert_ffn
  * (ws_* may be NULL when S == 0).  y: host bf16 [T,H].  rank_load: host int64 [R] or NULL.
  * dispatch_bytes: host uint64 [R,R] or NULL.  Pinned host buffers make the copies asynchronous. */
@@ -171,6 +171,22 @@ int director_layer_forward_host(director_ctx* ctx, int32_t T, const float* logit
                                 const void* w_gate, const void* w_up, const void* w_down,
                                 const void* ws_gate, const void* ws_up, const void* ws_down,
                                 void* y, int64_t* rank_load, uint64_t* dispatch_bytes, void* stream);
+
+/* The same, split in two so that a stream of batches overlaps its transfers with its kernels (the
+ * serving loop of Section IV feeds one batch after another): submit enqueues the host->device copies
+ * on an internal copy stream, the kernels on `stream` and the device->host copies on a second internal
+ * copy stream, chained by events, and returns at once with a ticket; wait blocks until that batch's
+ * results are in its host buffers.  Inputs, y and the histograms are double-buffered on the device, so
+ * the copies of batch i+1 and of batch i-1 run while the kernels of batch i do.  At most two batches
+ * may be in flight: wait for ticket i-1 (at the latest) before submitting batch i+1.  The host buffers
+ * of a batch (pinned, for real overlap) must stay valid and untouched until its wait returns.
+ * Arguments as for director_layer_forward_host; ticket: host, receives the batch's sequence number. */
+int director_layer_submit_host(director_ctx* ctx, int32_t T, const float* logits, const void* x,
+                               const void* w_gate, const void* w_up, const void* w_down,
+                               const void* ws_gate, const void* ws_up, const void* ws_down,
+                               void* y, int64_t* rank_load, uint64_t* dispatch_bytes, void* stream,
+                               int64_t* ticket);
+int director_layer_wait_host(director_ctx* ctx, int64_t ticket);
 
 /* Synchronises `stream`, returns the sticky device status word (DIRECTOR_OK if clean) and
  * clears it. */

@@ -22,7 +22,8 @@ EXPORTED = (
     "director_create", "director_destroy", "director_set_placement", "director_route", "director_dispatch",
     "director_expert_ffn", "director_combine", "director_placement_cost", "director_layer_forward_host",
     "director_last_status", "director_launch_count", "director_set_profiling", "director_kernel_time",
-    "director_status_string", "director_dispatch_index_static",
+    "director_status_string", "director_dispatch_index_static", "director_layer_submit_host",
+    "director_layer_wait_host",
 )
 
 
@@ -57,6 +58,8 @@ def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.director_combine.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp]
     lib.director_placement_cost.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp, vp]
     lib.director_layer_forward_host.argtypes = [vp, c_int32] + [vp] * 12
+    lib.director_layer_submit_host.argtypes = [vp, c_int32] + [vp] * 13
+    lib.director_layer_wait_host.argtypes = [vp, c_int64]
     lib.director_dispatch_index_static.argtypes = [c_int32] * 5 + [vp] * 9
     lib.director_last_status.argtypes = [vp, vp]
     lib.director_launch_count.argtypes = [vp]
@@ -153,6 +156,20 @@ class Director:
                                                     _ptr(w_down), _ptr(ws_gate), _ptr(ws_up), _ptr(ws_down), _ptr(y),
                                                     _ptr(rank_load), _ptr(dispatch_bytes), _stream()),
                "director_layer_forward_host")
+
+    def layer_submit_host(self, T, logits, x, w_gate, w_up, w_down, ws_gate, ws_up, ws_down, y,
+                          rank_load=None, dispatch_bytes=None) -> int:
+        """Enqueues one batch (host buffers as for layer_forward_host) and returns its ticket; at most two
+        batches may be in flight."""
+        ticket = c_int64(-1)
+        _check(self.lib.director_layer_submit_host(self._ctx, T, _ptr(logits), _ptr(x), _ptr(w_gate), _ptr(w_up),
+                                                   _ptr(w_down), _ptr(ws_gate), _ptr(ws_up), _ptr(ws_down), _ptr(y),
+                                                   _ptr(rank_load), _ptr(dispatch_bytes), _stream(),
+                                                   ctypes.byref(ticket)), "director_layer_submit_host")
+        return int(ticket.value)
+
+    def layer_wait_host(self, ticket: int):
+        _check(self.lib.director_layer_wait_host(self._ctx, ticket), "director_layer_wait_host")
 
     # -- status / instrumentation --------------------------------------------------------------
     def last_status(self) -> int:

@@ -33,10 +33,18 @@ bool shape_supported(const director_shape& s) {
 void free_all(director_ctx* c) {
     void* ptrs[] = {c->d_rep_start, c->d_rep_slot, c->d_slot_expert, c->d_tile_counts, c->d_seg_offsets, c->d_ticket,
                     c->d_status, c->d_hidden, c->d_hidden_shared, c->d_one_seg,
-                    c->d_zero_expert, c->e_logits, c->e_x, c->e_topk_idx, c->e_topk_w, c->e_xp, c->e_yp, c->e_y,
-                    c->e_y_shared, c->e_row_token, c->e_inv_row, c->e_dest_rank, c->e_cost};
+                    c->d_zero_expert, c->e_logits2[0], c->e_logits2[1], c->e_x2[0], c->e_x2[1], c->e_topk_idx,
+                    c->e_topk_w, c->e_xp, c->e_yp, c->e_y2[0], c->e_y2[1], c->e_y_shared, c->e_row_token, c->e_inv_row,
+                    c->e_dest_rank, c->e_cost2[0], c->e_cost2[1]};
     for (void* p : ptrs)
         if (p) cudaFree(p);
+    for (int i = 0; i < 2; ++i) {
+        if (c->ev_h2d_done[i]) cudaEventDestroy(c->ev_h2d_done[i]);
+        if (c->ev_compute_done[i]) cudaEventDestroy(c->ev_compute_done[i]);
+        if (c->ev_d2h_done[i]) cudaEventDestroy(c->ev_d2h_done[i]);
+    }
+    if (c->h2d_stream) cudaStreamDestroy(c->h2d_stream);
+    if (c->d2h_stream) cudaStreamDestroy(c->d2h_stream);
     for (auto& ev : c->events) { cudaEventDestroy(ev.start); cudaEventDestroy(ev.stop); }
     for (auto& ev : c->free_events) { cudaEventDestroy(ev.start); cudaEventDestroy(ev.stop); }
 }
@@ -92,14 +100,17 @@ int director_create(const director_shape* shape, director_ctx** out) {
               dev_alloc(&c->d_zero_expert, 1) &&
               dev_alloc(reinterpret_cast<uint16_t**>(&c->d_hidden), A * s.F) &&
               dev_alloc(reinterpret_cast<uint16_t**>(&c->d_hidden_shared), T * s.S * s.F) &&
-              dev_alloc(&c->e_logits, T * s.E) && dev_alloc(reinterpret_cast<uint16_t**>(&c->e_x), T * s.H) &&
+              dev_alloc(&c->e_logits2[0], T * s.E) && dev_alloc(&c->e_logits2[1], T * s.E) &&
+              dev_alloc(reinterpret_cast<uint16_t**>(&c->e_x2[0]), T * s.H) &&
+              dev_alloc(reinterpret_cast<uint16_t**>(&c->e_x2[1]), T * s.H) &&
               dev_alloc(&c->e_topk_idx, A) && dev_alloc(&c->e_topk_w, A) &&
               dev_alloc(reinterpret_cast<uint16_t**>(&c->e_xp), A * s.H) &&
               dev_alloc(reinterpret_cast<uint16_t**>(&c->e_yp), A * s.H) &&
-              dev_alloc(reinterpret_cast<uint16_t**>(&c->e_y), T * s.H) &&
+              dev_alloc(reinterpret_cast<uint16_t**>(&c->e_y2[0]), T * s.H) &&
+              dev_alloc(reinterpret_cast<uint16_t**>(&c->e_y2[1]), T * s.H) &&
               dev_alloc(reinterpret_cast<uint16_t**>(&c->e_y_shared), s.S > 0 ? T * s.H : 0) &&
               dev_alloc(&c->e_row_token, A) && dev_alloc(&c->e_inv_row, A) && dev_alloc(&c->e_dest_rank, A) &&
-              dev_alloc(&c->e_cost, cost_words);
+              dev_alloc(&c->e_cost2[0], cost_words) && dev_alloc(&c->e_cost2[1], cost_words);
     if (!ok) {
         cudaGetLastError();
         free_all(c);
@@ -117,6 +128,14 @@ int director_create(const director_shape* shape, director_ctx** out) {
              qres == cudaDriverEntryPointSuccess && c->encode_tiled != nullptr;
     }
     if (ok) ok = ffn_init(c) == DIRECTOR_OK;
+    if (ok) {
+        ok = cudaStreamCreateWithFlags(&c->h2d_stream, cudaStreamNonBlocking) == cudaSuccess &&
+             cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking) == cudaSuccess;
+        for (int i = 0; i < 2 && ok; ++i)
+            ok = cudaEventCreateWithFlags(&c->ev_h2d_done[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&c->ev_compute_done[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&c->ev_d2h_done[i], cudaEventDisableTiming) == cudaSuccess;
+    }
     if (!ok) {
         cudaGetLastError();
         free_all(c);
@@ -250,13 +269,14 @@ int director_placement_cost(director_ctx* ctx, int32_t T, const int32_t* topk_id
                        as_stream(stream));
 }
 
-int director_layer_forward_host(director_ctx* ctx, int32_t T, const float* logits, const void* x, const void* w_gate,
-                                const void* w_up, const void* w_down, const void* ws_gate, const void* ws_up,
-                                const void* ws_down, void* y, int64_t* rank_load, uint64_t* dispatch_bytes, void* stream) {
+int director_layer_submit_host(director_ctx* ctx, int32_t T, const float* logits, const void* x, const void* w_gate,
+                               const void* w_up, const void* w_down, const void* ws_gate, const void* ws_up,
+                               const void* ws_down, void* y, int64_t* rank_load, uint64_t* dispatch_bytes, void* stream,
+                               int64_t* ticket) {
     REQUIRE_CTX(ctx);
     REQUIRE_T(ctx, T);
     REQUIRE_PLACEMENT(ctx);
-    if (!logits || !x || !y) return DIRECTOR_ERR_INVALID_ARG;
+    if (!logits || !x || !y || !ticket) return DIRECTOR_ERR_INVALID_ARG;
     REQUIRE_PTR(w_gate);
     REQUIRE_PTR(w_up);
     REQUIRE_PTR(w_down);
@@ -268,33 +288,67 @@ int director_layer_forward_host(director_ctx* ctx, int32_t T, const float* logit
         REQUIRE_PTR(ws_down);
     }
     cudaStream_t st = as_stream(stream);
-    int64_t* c_w = ctx->e_cost;
+    const int slot = (int)(ctx->submitted & 1);
+    float* d_logits = ctx->e_logits2[slot];
+    void* d_x = ctx->e_x2[slot];
+    void* d_y = ctx->e_y2[slot];
+    int64_t* c_w = ctx->e_cost2[slot];
     int64_t* c_load = c_w + (size_t)s.R * s.E;
     int64_t* c_tok = c_load + s.R;
     uint64_t* c_bytes = reinterpret_cast<uint64_t*>(c_tok + (size_t)s.R * s.R);
 
-    if (cudaMemcpyAsync(ctx->e_logits, logits, sizeof(float) * (size_t)T * s.E, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(ctx->e_x, x, 2 * (size_t)T * s.H, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    // inputs: wait until the kernels of the batch that used this slot two submissions ago are done with it
+    if (cudaStreamWaitEvent(ctx->h2d_stream, ctx->ev_compute_done[slot], 0) != cudaSuccess ||
+        cudaMemcpyAsync(d_logits, logits, sizeof(float) * (size_t)T * s.E, cudaMemcpyHostToDevice, ctx->h2d_stream) != cudaSuccess ||
+        cudaMemcpyAsync(d_x, x, 2 * (size_t)T * s.H, cudaMemcpyHostToDevice, ctx->h2d_stream) != cudaSuccess ||
+        cudaEventRecord(ctx->ev_h2d_done[slot], ctx->h2d_stream) != cudaSuccess)
         return DIRECTOR_ERR_CUDA;
-    int rc = launch_route(ctx, T, ctx->e_logits, ctx->e_topk_idx, ctx->e_topk_w, st);
+    // kernels: need this batch's inputs, and the outputs of this slot must have left for the host
+    if (cudaStreamWaitEvent(st, ctx->ev_h2d_done[slot], 0) != cudaSuccess ||
+        cudaStreamWaitEvent(st, ctx->ev_d2h_done[slot], 0) != cudaSuccess)
+        return DIRECTOR_ERR_CUDA;
+    int rc = launch_route(ctx, T, d_logits, ctx->e_topk_idx, ctx->e_topk_w, st);
     if (rc == DIRECTOR_OK)
-        rc = launch_dispatch(ctx, T, ctx->e_x, ctx->e_topk_idx, ctx->e_xp, ctx->e_row_token, ctx->e_inv_row,
+        rc = launch_dispatch(ctx, T, d_x, ctx->e_topk_idx, ctx->e_xp, ctx->e_row_token, ctx->e_inv_row,
                              ctx->e_dest_rank, ctx->d_seg_offsets, st);
     if (rc == DIRECTOR_OK)
         rc = launch_expert_ffn(ctx, T, ctx->e_xp, ctx->d_seg_offsets, w_gate, w_up, w_down, ctx->e_yp,
-                               shared ? ctx->e_x : nullptr, ws_gate, ws_up, ws_down, ctx->e_y_shared, st);
+                               shared ? d_x : nullptr, ws_gate, ws_up, ws_down, ctx->e_y_shared, st);
     if (rc == DIRECTOR_OK)
-        rc = launch_combine(ctx, T, ctx->e_yp, ctx->e_inv_row, ctx->e_topk_w, shared ? ctx->e_y_shared : nullptr,
-                            ctx->e_y, st);
+        rc = launch_combine(ctx, T, ctx->e_yp, ctx->e_inv_row, ctx->e_topk_w, shared ? ctx->e_y_shared : nullptr, d_y, st);
     if (rc == DIRECTOR_OK) rc = launch_cost(ctx, T, ctx->e_topk_idx, nullptr, c_w, c_load, c_tok, c_bytes, st);
     if (rc != DIRECTOR_OK) return rc;
-    if (cudaMemcpyAsync(y, ctx->e_y, 2 * (size_t)T * s.H, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DIRECTOR_ERR_CUDA;
-    if (rank_load && cudaMemcpyAsync(rank_load, c_load, sizeof(int64_t) * s.R, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    if (cudaEventRecord(ctx->ev_compute_done[slot], st) != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    // outputs
+    if (cudaStreamWaitEvent(ctx->d2h_stream, ctx->ev_compute_done[slot], 0) != cudaSuccess ||
+        cudaMemcpyAsync(y, d_y, 2 * (size_t)T * s.H, cudaMemcpyDeviceToHost, ctx->d2h_stream) != cudaSuccess)
         return DIRECTOR_ERR_CUDA;
-    if (dispatch_bytes &&
-        cudaMemcpyAsync(dispatch_bytes, c_bytes, sizeof(uint64_t) * s.R * s.R, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    if (rank_load &&
+        cudaMemcpyAsync(rank_load, c_load, sizeof(int64_t) * s.R, cudaMemcpyDeviceToHost, ctx->d2h_stream) != cudaSuccess)
         return DIRECTOR_ERR_CUDA;
-    return cuda_status(cudaStreamSynchronize(st));
+    if (dispatch_bytes && cudaMemcpyAsync(dispatch_bytes, c_bytes, sizeof(uint64_t) * s.R * s.R, cudaMemcpyDeviceToHost,
+                                          ctx->d2h_stream) != cudaSuccess)
+        return DIRECTOR_ERR_CUDA;
+    if (cudaEventRecord(ctx->ev_d2h_done[slot], ctx->d2h_stream) != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    *ticket = ctx->submitted++;
+    return DIRECTOR_OK;
+}
+
+int director_layer_wait_host(director_ctx* ctx, int64_t ticket) {
+    REQUIRE_CTX(ctx);
+    if (ticket < 0 || ticket >= ctx->submitted) return DIRECTOR_ERR_INVALID_ARG;
+    if (ticket + 2 < ctx->submitted) return DIRECTOR_OK;   // its slot was reused, which waited for it
+    return cuda_status(cudaEventSynchronize(ctx->ev_d2h_done[ticket & 1]));
+}
+
+int director_layer_forward_host(director_ctx* ctx, int32_t T, const float* logits, const void* x, const void* w_gate,
+                                const void* w_up, const void* w_down, const void* ws_gate, const void* ws_up,
+                                const void* ws_down, void* y, int64_t* rank_load, uint64_t* dispatch_bytes, void* stream) {
+    int64_t ticket = -1;
+    const int rc = director_layer_submit_host(ctx, T, logits, x, w_gate, w_up, w_down, ws_gate, ws_up, ws_down, y,
+                                              rank_load, dispatch_bytes, stream, &ticket);
+    if (rc != DIRECTOR_OK) return rc;
+    return director_layer_wait_host(ctx, ticket);
 }
 
 int director_last_status(director_ctx* ctx, void* stream) {

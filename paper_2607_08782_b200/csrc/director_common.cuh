@@ -52,19 +52,24 @@ struct director_ctx {
     int32_t* d_one_seg = nullptr;      // [2] segment table {0, T} used for the shared experts
     int32_t* d_zero_expert = nullptr;  // [1] = {0}
 
-    // buffers of director_layer_forward_host
-    float* e_logits = nullptr;
-    void* e_x = nullptr;
+    // buffers of the host-buffer entry points; inputs, y and the histograms exist twice so that the
+    // copies of one batch overlap the kernels of its neighbours
+    float* e_logits2[2] = {nullptr, nullptr};
+    void* e_x2[2] = {nullptr, nullptr};
+    void* e_y2[2] = {nullptr, nullptr};
+    int64_t* e_cost2[2] = {nullptr, nullptr};   // workload [R,E] | rank_load [R] | dispatch_tokens [R,R] | bytes [R,R]
+    cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+    cudaEvent_t ev_h2d_done[2] = {nullptr, nullptr}, ev_compute_done[2] = {nullptr, nullptr},
+                ev_d2h_done[2] = {nullptr, nullptr};
+    int64_t submitted = 0;
     int32_t* e_topk_idx = nullptr;
     float* e_topk_w = nullptr;
     void* e_xp = nullptr;
     void* e_yp = nullptr;
-    void* e_y = nullptr;
     void* e_y_shared = nullptr;
     int32_t* e_row_token = nullptr;
     int32_t* e_inv_row = nullptr;
     int32_t* e_dest_rank = nullptr;
-    int64_t* e_cost = nullptr;          // workload [R,E] | rank_load [R] | dispatch_tokens [R,R] | bytes [R,R]
 
     void* encode_tiled = nullptr;       // cuTensorMapEncodeTiled, resolved through the runtime
 

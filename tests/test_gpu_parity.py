@@ -228,3 +228,52 @@ def test_c4_qwen15_shaped():
 @pytest.mark.parametrize("T", synth.C5_SWEEP)
 def test_c5_qwen3_shaped_sweep(T):
     _full_size("c5_qwen3", T, [("round-robin", _primary), ("load-balanced", _balanced)])
+
+
+def test_host_buffer_entry_points_match_the_device_path():
+    """director_layer_forward_host and the pipelined submit/wait pair give the same bits as the
+    device-pointer stages, also with three different batches in flight back to back."""
+    import torch
+    shape, logits, x, weights = _custom(61, 900, 256, 12, 3, 256, 1, 4, 4, 1.2)
+    X = _random_placement(61, 12, 4, 4, 3)
+    case = GpuCase(shape, logits, x, weights)
+    L, d = case.layer, case.layer.d
+    batches = []
+    for i, T in enumerate((900, 333, 640)):
+        lg = np.ascontiguousarray(np.roll(logits, i * 3, axis=1)[:T])
+        xb = np.ascontiguousarray(x[i:i + T] if i + T <= 900 else x[:T])
+        L.set_placement(X)
+        L.route(T, torch.from_numpy(lg).cuda())
+        from paper_2607_08782_b200.layer import bf16_bits_to_tensor, tensor_to_bf16_bits
+        xd = bf16_bits_to_tensor(xb)
+        L.dispatch(T, xd)
+        L.expert_ffn(T, xd)
+        L.combine(T)
+        L.placement_cost(T)
+        torch.cuda.synchronize()
+        batches.append(dict(T=T, lg=torch.from_numpy(lg).pin_memory(), x=torch.from_numpy(xb.view(np.int16)).pin_memory(),
+                            y_ref=tensor_to_bf16_bits(L.y[:T]).copy(), load_ref=L.rank_load.cpu().numpy().copy(),
+                            bytes_ref=L.dispatch_bytes.cpu().numpy().copy(),
+                            y=torch.zeros((T, shape.H), dtype=torch.int16).pin_memory(),
+                            load=torch.zeros((shape.R,), dtype=torch.int64).pin_memory(),
+                            byt=torch.zeros((shape.R, shape.R), dtype=torch.int64).pin_memory()))
+    # blocking form
+    b = batches[0]
+    d.layer_forward_host(b["T"], b["lg"], b["x"], *L.w, *L.ws, b["y"], b["load"], b["byt"])
+    assert np.array_equal(b["y"].numpy().view(np.uint16), b["y_ref"])
+    assert np.array_equal(b["load"].numpy(), b["load_ref"]) and np.array_equal(b["byt"].numpy(), b["bytes_ref"])
+    # pipelined form, two in flight
+    for b in batches:
+        b["y"].zero_()
+    tickets = []
+    for i, b in enumerate(batches * 2):
+        if i >= 2:
+            d.layer_wait_host(tickets[i - 2])
+        tickets.append(d.layer_submit_host(b["T"], b["lg"], b["x"], *L.w, *L.ws, b["y"], b["load"], b["byt"]))
+    for t in tickets[-2:]:
+        d.layer_wait_host(t)
+    for b in batches:
+        assert np.array_equal(b["y"].numpy().view(np.uint16), b["y_ref"])
+        assert np.array_equal(b["load"].numpy(), b["load_ref"])
+    assert d.last_status() == 0
+    assert case.layer.d.lib.director_layer_wait_host(d._ctx, 10 ** 6) == 1      # unknown ticket
