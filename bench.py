@@ -184,6 +184,8 @@ def build_layer(args, device):
     else:
         X, pname = placement.greedy_balanced(N, s.R, s.C_max, synth.primary_ranks(s)), "primaries + greedy replicas"
     layer.set_placement(X)
+    if args.ffn_variant is not None:
+        layer.d.set_ffn_variant(args.ffn_variant)
     return wl, layer, logits, x, X, pname
 
 
@@ -302,6 +304,8 @@ def main():
     ap.add_argument("--config", default="c2_mixtral", choices=sorted(WORKLOAD_TEXT))
     ap.add_argument("--tokens", type=int, default=None, help="batch size override (c5_qwen3 sweep: 1, 64, 1024, 32768)")
     ap.add_argument("--placement", default="auto", choices=["auto", "primary"])
+    ap.add_argument("--ffn-variant", type=int, default=None, choices=[0, 1, 2],
+                    help="expert-FFN tile scheme: 0 = one CTA per 128x256 tile, 1 = CTA pairs (256x256); default: library's")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-clocks", nargs=2, metavar=("UUID", "PATH"), help=argparse.SUPPRESS)
     args = ap.parse_args()

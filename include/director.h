@@ -192,6 +192,15 @@ int director_layer_wait_host(director_ctx* ctx, int64_t ticket);
  * clears it. */
 int director_last_status(director_ctx* ctx, void* stream);
 
+/* Tile scheme of the expert-FFN GEMMs (results are bit-identical across schemes):
+ *   2 (default) weight-stationary CTA pairs: 256 weight rows x up to 256 tokens per tile, the token count
+ *               of a tile is a runtime operand in steps of 32, so ragged segment tails cost almost nothing;
+ *   1           token-stationary CTA pairs: 256 tokens x 256 weight rows per tile;
+ *   0           token-stationary single CTAs: 128 tokens x 256 weight rows per tile.
+ * Scheme 2 falls back to scheme 0 when w_gate and w_up cannot be described by one strided tensor map
+ * (their addresses differ by 2^40 bytes or more). */
+int director_set_ffn_variant(director_ctx* ctx, int32_t variant);
+
 /* Number of kernels this context has launched since it was created. */
 int64_t director_launch_count(const director_ctx* ctx);
 

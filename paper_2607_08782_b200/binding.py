@@ -23,7 +23,7 @@ EXPORTED = (
     "director_expert_ffn", "director_combine", "director_placement_cost", "director_layer_forward_host",
     "director_last_status", "director_launch_count", "director_set_profiling", "director_kernel_time",
     "director_status_string", "director_dispatch_index_static", "director_layer_submit_host",
-    "director_layer_wait_host",
+    "director_layer_wait_host", "director_set_ffn_variant",
 )
 
 
@@ -65,6 +65,7 @@ def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.director_launch_count.argtypes = [vp]
     lib.director_launch_count.restype = c_int64
     lib.director_set_profiling.argtypes = [vp, c_int32]
+    lib.director_set_ffn_variant.argtypes = [vp, c_int32]
     lib.director_kernel_time.argtypes = [vp, c_char_p, POINTER(c_int64)]
     lib.director_kernel_time.restype = c_double
     lib.director_status_string.argtypes = [c_int]
@@ -177,6 +178,9 @@ class Director:
 
     def check_device_status(self):
         _check(self.last_status(), "device status")
+
+    def set_ffn_variant(self, variant: int):
+        _check(self.lib.director_set_ffn_variant(self._ctx, variant), "director_set_ffn_variant")
 
     def launch_count(self) -> int:
         return int(self.lib.director_launch_count(self._ctx))

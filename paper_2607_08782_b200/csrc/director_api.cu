@@ -361,6 +361,15 @@ int director_last_status(director_ctx* ctx, void* stream) {
     return h;
 }
 
+int director_set_ffn_variant(director_ctx* ctx, int32_t variant) {
+    REQUIRE_CTX(ctx);
+    if (variant < 0 || variant > 2) return DIRECTOR_ERR_INVALID_ARG;
+    ctx->ffn_variant = variant;
+    return DIRECTOR_OK;
+}
+
+int director_pair_clusters(const director_ctx* ctx) { return ctx ? ctx->pair_clusters : -1; }
+
 int64_t director_launch_count(const director_ctx* ctx) { return ctx ? ctx->launches : -1; }
 
 int director_set_profiling(director_ctx* ctx, int32_t enabled) {

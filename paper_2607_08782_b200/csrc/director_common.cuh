@@ -71,6 +71,8 @@ struct director_ctx {
     int32_t* e_inv_row = nullptr;
     int32_t* e_dest_rank = nullptr;
 
+    int pair_clusters = 0;              // CTA pairs the device can hold at once (pair variant's grid)
+    int ffn_variant = 2;                // tile scheme of the expert-FFN GEMMs, see director_set_ffn_variant
     void* encode_tiled = nullptr;       // cuTensorMapEncodeTiled, resolved through the runtime
 
     int64_t launches = 0;

@@ -21,129 +21,21 @@
 // the tile prefix from seg_offsets in its prologue.  Every mbarrier wait is bounded; on expiry the CTA
 // raises DIRECTOR_ERR_TIMEOUT, all roles drain and the CTA frees its TMEM and returns.
 #include "director_common.cuh"
+#include "director_umma.cuh"
 
 namespace director {
 
+int ffn_swap_init(director_ctx* ctx);   // director_ffn_swap.cu
+int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t rows, const int32_t* seg_offsets, const int32_t* slot_expert,
+                  int G, const void* w_gate, const void* w_up, const void* w_down, uint64_t n_experts, int Fw, void* hidden,
+                  void* out, cudaStream_t st);
+int ffn_pair_init(director_ctx* ctx);   // director_ffn_pair.cu
+int launch_gemm_pair(director_ctx* ctx, int mode, const char* name, const CUtensorMap& a, const CUtensorMap& b0,
+                     const CUtensorMap& b1, const umma::GroupedGemmParams& p, cudaStream_t st);
+
 namespace {
 
-constexpr int BLOCK_M = 128;
-constexpr int UMMA_N = 256;
-constexpr int BLOCK_K = 64;                 // bf16 per k-step: 128 bytes, one swizzle row
-constexpr int UMMA_K = 16;
-constexpr int STAGES = 4;
-constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2;       // 16 KB
-constexpr int B_HALF_BYTES = 128 * BLOCK_K * 2;      // 16 KB
-constexpr int STAGE_BYTES = A_BYTES + 2 * B_HALF_BYTES;
-constexpr int FFN_THREADS = 192;
-constexpr int TMEM_COLS = 512;
-constexpr int TABLE_INTS = 3 * (kMaxG + 1);
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + TABLE_INTS * 4;
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s
-
-// tcgen05 instruction descriptor, kind::f16: D=f32 (bits 4-5 = 1), A=B=bf16 (bits 7-9, 10-12 = 1),
-// both operands K-major (bits 15, 16 = 0), N>>3 at bit 17, M>>4 at bit 24.
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(UMMA_N >> 3) << 17) |
-                           ((uint32_t)(BLOCK_M >> 4) << 24);
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait.  Returns false if the wait expired or another role of this CTA already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    uint32_t n = 0;
-    while (!mbar_try(bar, parity)) {
-        if ((++n & 63u) == 0u) {
-            if (*abort_flag) return false;
-            if (global_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
-        }
-    }
-    return true;
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y) : "memory");
-}
-
-// Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows of 128 bytes, 8-row groups
-// 1024 bytes apart (SBO), descriptor version 1 (bit 46), layout type 2 = SWIZZLE_128B (bits 61-63).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-    return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
-           (2ull << 61);
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(IDESC), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr));
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-
-struct GroupedGemmParams {
-    const int32_t* seg_offsets;   // [G+1] first row of every segment
-    const int32_t* slot_expert;   // [G] expert of the segment (selects the B rows), < 0 = unused
-    int G;
-    int n_blocks;                 // output column blocks per expert
-    int k_steps;                  // K / 64
-    int b_rows_per_expert;        // rows of B per expert
-    int out_pitch;                // bf16 elements per output row
-    void* out;
-    int32_t* status;
-};
-
-struct Tile {
-    int row0, row_end, b_row, nb;
-};
+using namespace umma;
 
 // Walks the work list for one role; `g` is the role's private segment cursor.
 struct TileWalker {
@@ -374,6 +266,7 @@ bool make_map(director_ctx* ctx, CUtensorMap* map, const void* base, uint64_t ro
 template <int MODE>
 int launch_gemm(director_ctx* ctx, const char* name, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
                 const GroupedGemmParams& p, cudaStream_t st) {
+    if (ctx->ffn_variant >= 1) return launch_gemm_pair(ctx, MODE, name, a, b0, b1, p, st);
     LaunchScope scope(ctx, st, name);
     grouped_gemm_kernel<MODE><<<ctx->sm_count, FFN_THREADS, SMEM_BYTES, st>>>(a, b0, b1, p);
     return cuda_status(cudaGetLastError());
@@ -383,6 +276,11 @@ int launch_gemm(director_ctx* ctx, const char* name, const CUtensorMap& a, const
 int ffn_pass(director_ctx* ctx, const void* in, uint64_t rows, const int32_t* seg_offsets, const int32_t* slot_expert,
              int G, const void* w_gate, const void* w_up, const void* w_down, uint64_t n_experts, int Fw, void* hidden,
              void* out, cudaStream_t st) {
+    if (ctx->ffn_variant == 2) {
+        const int rc = ffn_pass_swap(ctx, in, rows, seg_offsets, slot_expert, G, w_gate, w_up, w_down, n_experts, Fw, hidden,
+                                     out, st);
+        if (rc != DIRECTOR_ERR_UNSUPPORTED) return rc;   // weight arrays not expressible as one map: tile scheme 0
+    }
     const int H = ctx->shape.H;
     CUtensorMap m_in, m_g, m_u, m_h, m_d;
     if (!make_map(ctx, &m_in, in, rows, H) || !make_map(ctx, &m_g, w_gate, n_experts * Fw, H) ||
@@ -403,7 +301,8 @@ __global__ void one_segment_kernel(int32_t* seg, int T) {
 
 }  // namespace
 
-int ffn_init(director_ctx*) {
+int ffn_init(director_ctx* ctx) {
+    if (ffn_pair_init(ctx) != DIRECTOR_OK || ffn_swap_init(ctx) != DIRECTOR_OK) return DIRECTOR_ERR_CUDA;
     if (cudaFuncSetAttribute(grouped_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
         cudaFuncSetAttribute(grouped_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
         return DIRECTOR_ERR_CUDA;

@@ -1,0 +1,381 @@
+// Weight-stationary ("swapped") CTA-pair variant of the grouped expert-FFN GEMMs (Section II-A expert
+// FFNs after dispatch).
+//
+// Segments are ragged: their lengths follow the routing skew, so tiling the TOKEN dimension in steps
+// of 128 or 256 rows (the M of the tensor-core instruction) pads every segment tail with rows that are
+// computed and thrown away (9-27 % extra work on the paper-shaped workloads).  Here the roles are
+// swapped: the weight rows are the M operand (always full: 128 rows per CTA, 256 per CTA pair) and the
+// tokens are the N operand, whose size is a runtime field of the instruction descriptor in steps of 32.
+// A segment tail then costs only its length rounded up to 32 tokens.
+//
+//   D[weight row, token] = sum_k W[weight row, k] * X[token, k]        (both operands K-major)
+//
+// CTA pair, tcgen05.mma cta_group::2, M = 256, N = tokens in the tile (32..256):
+//   CTA r supplies 128 weight rows (A) and half of the tile's tokens (B rows [r*N/2, (r+1)*N/2)).
+//   GEMM-1: CTA r's weight rows are 64 gate rows INTERLEAVED with the matching 64 up rows (a 3-D TMA box
+//           over {k, gate|up, f} builds the interleave on the fly from the two separate weight arrays), so
+//           TMEM lane 2j holds gate_f and lane 2j+1 holds up_f: SwiGLU is a lane-pair shuffle.
+//   GEMM-2: CTA r's weight rows are 128 consecutive rows of W_down.
+// The accumulator is [weight rows x tokens]; the epilogue writes it transposed (2-byte stores, one
+// token per instruction, 32-64 contiguous bytes per warp) into the row-major [tokens, features] outputs.
+// Barrier protocol, bounded waits and teardown are those of the plain CTA-pair kernel.
+#include "director_common.cuh"
+#include "director_umma.cuh"
+
+#include <cuda_bf16.h>
+
+namespace director {
+
+using namespace umma;
+
+namespace {
+
+constexpr int S_STAGES = 6;
+constexpr int S_STAGE_BYTES = A_BYTES + B_HALF_BYTES;          // 16 KB weights + 16 KB tokens per CTA per k-step
+constexpr int S_SMEM_BYTES = S_STAGES * S_STAGE_BYTES + 1024 + 256 + TABLE_INTS * 4;
+constexpr int TOKEN_TILE = 256;                                // tokens per full tile (N of the pair's MMA)
+constexpr int TOKEN_STEP = 32;                                 // granularity of N
+// Epilogue warps per TMEM lane quadrant.  The SwiGLU epilogue of GEMM-1 is long (shuffle, exp, reciprocal,
+// convert and a 2-byte store per element) and a lone warp per scheduler cannot hide its own latencies, so it
+// gets two warps per quadrant, each taking every other 32-token chunk.  GEMM-2's epilogue is a plain convert
+// and store; one warp per quadrant with a large register budget (all 32 stores of a chunk in flight) is faster.
+constexpr int EPI_GROUPS_GEMM1 = 2;
+constexpr int EPI_GROUPS_GEMM2 = 1;
+
+// kind::f16 descriptor for the pair without the N field: D=f32, A=B=bf16, K-major, M=256.
+constexpr uint32_t S_IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 4) << 24);
+
+__device__ __forceinline__ void umma_pair_n(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t cluster_bar, int x, int y,
+                                                 int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(cluster_bar), "r"(x), "r"(y), "r"(z) : "memory");
+}
+
+struct SwapParams {
+    const int32_t* seg_offsets;
+    const int32_t* slot_expert;
+    int G;
+    int w_blocks;              // weight-row blocks per expert (128 f per pair in GEMM-1, 256 h in GEMM-2)
+    int k_steps;
+    int w_rows_per_expert;     // F (GEMM-1, in units of f) or H (GEMM-2)
+    int out_pitch;             // bf16 elements per output row
+    int gate_first;            // GEMM-1: 1 if even lanes hold gate rows, 0 if they hold up rows
+    void* out;
+    int32_t* status;
+};
+
+struct SwapTile {
+    int row0;      // first token row of the tile
+    int valid;     // tokens of the tile that belong to the segment (1..256)
+    int n;         // valid rounded up to a multiple of 32: N of the MMA
+    int w_row;     // first weight row of the pair's block (f index for GEMM-1, W_down row for GEMM-2)
+    int wb;
+};
+
+struct SwapWalker {
+    const int32_t* seg_off;
+    const int32_t* tt_start;    // prefix of token tiles per segment
+    const int32_t* expert;
+    int w_blocks, w_rows_per_expert, rows_per_block, total, g = 0;
+    __device__ bool get(int w, SwapTile& t) {
+        if (w >= total) return false;
+        while (w >= tt_start[g + 1] * w_blocks) ++g;
+        const int nt = tt_start[g + 1] - tt_start[g];
+        const int local = w - tt_start[g] * w_blocks;
+        t.wb = local / nt;
+        const int tt = local - t.wb * nt;
+        t.row0 = seg_off[g] + tt * TOKEN_TILE;
+        t.valid = min(TOKEN_TILE, seg_off[g + 1] - t.row0);
+        t.n = (t.valid + TOKEN_STEP - 1) / TOKEN_STEP * TOKEN_STEP;
+        t.w_row = expert[g] * w_rows_per_expert + t.wb * rows_per_block;
+        return true;
+    }
+};
+
+// MODE 0: gate/up + SwiGLU (A from the 3-D interleaving map).  MODE 1: down projection (A from a 2-D map).
+template <int MODE, int EPI_GROUPS>
+__global__ void __launch_bounds__(64 + 128 * EPI_GROUPS, 1)
+grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
+                         const SwapParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;
+    uint8_t* gen = smem_raw + (tiles - raw) + S_STAGES * S_STAGE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(gen);             // full[6] empty[6] tfull[2] tempty[2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + 160);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + 164);
+    int32_t* warp_sum = reinterpret_cast<int32_t*>(gen + 176);     // [18]
+    int32_t* s_seg = reinterpret_cast<int32_t*>(gen + 256);
+    int32_t* s_tt = s_seg + (kMaxG + 1);
+    int32_t* s_exp = s_tt + (kMaxG + 1);
+
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (S_STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * S_STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * S_STAGES + 2 + a); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = p.G;
+    const uint32_t rank = cluster_ctarank();
+    const bool leader = rank == 0;
+    const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+
+    constexpr int n_threads = 64 + 128 * EPI_GROUPS;               // producer warp + MMA warp + epilogue warps
+    for (int g = threadIdx.x; g <= G; g += n_threads) s_seg[g] = __ldg(p.seg_offsets + g);
+    for (int g = threadIdx.x; g < G; g += n_threads) s_exp[g] = __ldg(p.slot_expert + g);
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < S_STAGES; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8 * EPI_GROUPS); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    {
+        auto tiles_of = [&](int g) {
+            const int len = s_seg[g + 1] - s_seg[g];
+            return (s_exp[g] >= 0 && len > 0) ? (len + TOKEN_TILE - 1) / TOKEN_TILE : 0;
+        };
+        const int per = (G + n_threads - 1) / n_threads;
+        const int lo = min((int)threadIdx.x * per, G), hi = min(lo + per, G);
+        int local = 0;
+        for (int g = lo; g < hi; ++g) local += tiles_of(g);
+        int incl = local;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) warp_sum[warp] = incl;
+        __syncthreads();
+        int base = incl - local;
+        for (int i = 0; i < warp; ++i) base += warp_sum[i];
+        for (int g = lo; g < hi; ++g) { s_tt[g] = base; base += tiles_of(g); }
+        if (threadIdx.x == n_threads - 1) s_tt[G] = base;
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    constexpr int ROWS_PER_BLOCK = (MODE == 0) ? 128 : 256;   // weight rows (f or h) per pair block
+    SwapWalker walker{s_seg, s_tt, s_exp, p.w_blocks, p.w_rows_per_expert, ROWS_PER_BLOCK, s_tt[G] * p.w_blocks};
+    SwapTile t;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int w = cluster_id; ok && walker.get(w, t); w += n_clusters) {
+                const int x_row = t.row0 + (int)rank * (t.n >> 1);          // this CTA's half of the tile's tokens
+                const int w_row = t.w_row + (int)rank * (ROWS_PER_BLOCK / 2);
+                for (int kb = 0; kb < p.k_steps; ++kb) {
+                    if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag))) break;
+                    const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
+                    const uint32_t a_dst = tiles + stage * S_STAGE_BYTES;
+                    mbar_expect_tx_cluster(leader_full, S_STAGE_BYTES);
+                    if (MODE == 0) tma_load_3d_pair(a_dst, &tm_w, leader_full, kb * BLOCK_K, 0, w_row);
+                    else tma_load_2d_pair(a_dst, &tm_w, leader_full, kb * BLOCK_K, w_row);
+                    tma_load_2d_pair(a_dst + A_BYTES, &tm_x, leader_full, kb * BLOCK_K, x_row);
+                    if (++stage == S_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && leader) {
+            int stage = 0, it = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int w = cluster_id; ok && walker.get(w, t); w += n_clusters, ++it) {
+                const int acc = it & 1;
+                if (!(ok = mbar_wait(tempty_bar(acc), (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag))) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TOKEN_TILE);
+                const uint32_t idesc = S_IDESC_BASE | ((uint32_t)(t.n >> 3) << 17);
+                for (int kb = 0; kb < p.k_steps; ++kb) {
+                    if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag))) break;
+                    tc_fence_after();
+                    const uint32_t a_src = tiles + stage * S_STAGE_BYTES;
+                    const uint64_t a_desc = smem_desc(a_src), b_desc = smem_desc(a_src + A_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                        umma_pair_n(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    umma_commit_both(empty_bar(stage));
+                    if (++stage == S_STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit_both(tfull_bar(acc));
+            }
+        }
+    } else {
+        const int quad = warp & 3;                                 // TMEM lane quadrant this warp may read
+        const int cgroup = EPI_GROUPS == 1 ? 0 : (warp - 2) >> 2;  // which of the 32-token chunks this warp takes
+        constexpr int CSTEP = 32 * EPI_GROUPS;
+        const int c_first = 32 * cgroup;
+        uint16_t* out = static_cast<uint16_t*>(p.out);
+        const int lane_row = quad * 32 + lane;                     // weight row of this thread inside the CTA's 128
+        int it = 0;
+        bool ok = true;
+        for (int w = cluster_id; ok && walker.get(w, t); w += n_clusters, ++it) {
+            const int acc = it & 1;
+            if (!(ok = mbar_wait(tfull_bar(acc), ((uint32_t)it >> 1) & 1u, abort_flag))) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * TOKEN_TILE);
+            if constexpr (MODE == 0) {
+                // even lane: one of (gate, up) for feature f, odd lane: the other; column = token.
+                // The two lanes of a pair split the tokens: the even lane finishes the even tokens, the odd lane
+                // the odd ones.  One shuffle per token pair hands each lane the partner value it needs, so all
+                // 32 lanes stay active and no branch separates the shuffles.
+                const int f = t.wb * 128 + (int)rank * 64 + (lane_row >> 1);
+                const bool odd = (lane & 1) != 0;
+                const bool i_am_gate = (!odd) == (p.gate_first != 0);
+                uint16_t* ocol = out + (size_t)(t.row0 + (odd ? 1 : 0)) * p.out_pitch + f;
+                const size_t two_rows = 2 * (size_t)p.out_pitch;
+#pragma unroll 1
+                for (int c = c_first; c < t.n; c += CSTEP) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + c, v);
+                    tmem_ld_wait();
+                    uint16_t* ptr = ocol + (size_t)c * p.out_pitch;     // my token of pair m is row c + 2m (+1 if odd)
+                    const int rem = t.valid - c - (odd ? 1 : 0);        // store pair m iff 2m < rem
+#pragma unroll
+                    for (int m = 0; m < 16; ++m) {
+                        const float mine = __uint_as_float(odd ? v[2 * m + 1] : v[2 * m]);   // my value at my token
+                        const float send = __uint_as_float(odd ? v[2 * m] : v[2 * m + 1]);   // my value at the partner's token
+                        const float other = __shfl_xor_sync(0xFFFFFFFFu, send, 1);           // partner's value at my token
+                        const float g = i_am_gate ? mine : other, u = i_am_gate ? other : mine;
+                        const float h = __fdividef(g * u, 1.0f + __expf(-g));
+                        if (2 * m < rem) *ptr = __bfloat16_as_ushort(__float2bfloat16_rn(h));
+                        ptr += two_rows;
+                    }
+                }
+            } else {
+                const int h_col = t.wb * 256 + (int)rank * 128 + lane_row;
+                uint16_t* ocol = out + (size_t)t.row0 * p.out_pitch + h_col;
+#pragma unroll 1
+                for (int c = c_first; c < t.n; c += CSTEP) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + c, v);
+                    tmem_ld_wait();
+                    uint16_t* ptr = ocol + (size_t)c * p.out_pitch;
+                    const int rem = t.valid - c;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        if (j < rem) *ptr = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[j])));
+                        ptr += p.out_pitch;
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (threadIdx.x == 0 && *abort_flag) director_set_status(p.status, DIRECTOR_ERR_TIMEOUT);
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// bf16 [rows, cols] row-major, box 64 x 128, 128-byte swizzle
+bool map_2d(director_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols) {
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {BLOCK_K, 128};
+    const cuuint32_t estr[2] = {1, 1};
+    return reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+               map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Two bf16 [rows, cols] matrices `first` and `first + delta` seen as one tensor {cols, 2, rows}; a box of
+// {64, 2, 64} lands in shared memory as 128 rows alternating between the two matrices.
+bool map_interleaved(director_ctx* ctx, CUtensorMap* map, const void* first, uint64_t delta_bytes, uint64_t rows,
+                     uint64_t cols) {
+    const cuuint64_t dims[3] = {cols, 2, rows};
+    const cuuint64_t strides[2] = {delta_bytes, cols * 2};
+    const cuuint32_t box[3] = {BLOCK_K, 2, 64};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+               map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(first), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int MODE, int EPI_GROUPS>
+int launch_swap(director_ctx* ctx, const char* name, const CUtensorMap& w, const CUtensorMap& x, const SwapParams& p,
+                cudaStream_t st) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * ctx->pair_clusters));
+    cfg.blockDim = dim3(64 + 128 * EPI_GROUPS);
+    cfg.dynamicSmemBytes = S_SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    LaunchScope scope(ctx, st, name);
+    return cuda_status(cudaLaunchKernelEx(&cfg, grouped_gemm_swap_kernel<MODE, EPI_GROUPS>, w, x, p));
+}
+
+}  // namespace
+
+int ffn_swap_init(director_ctx*) {
+    if (cudaFuncSetAttribute(grouped_gemm_swap_kernel<0, EPI_GROUPS_GEMM1>, cudaFuncAttributeMaxDynamicSharedMemorySize, S_SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(grouped_gemm_swap_kernel<1, EPI_GROUPS_GEMM2>, cudaFuncAttributeMaxDynamicSharedMemorySize, S_SMEM_BYTES) != cudaSuccess)
+        return DIRECTOR_ERR_CUDA;
+    return DIRECTOR_OK;
+}
+
+// in [rows, H] -> hidden [rows, Fw] -> out [rows, H] over a segment table, weight-stationary pair kernels.
+// Returns DIRECTOR_ERR_UNSUPPORTED if the two weight arrays cannot be described by one interleaving map.
+int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t rows, const int32_t* seg_offsets, const int32_t* slot_expert,
+                  int G, const void* w_gate, const void* w_up, const void* w_down, uint64_t n_experts, int Fw, void* hidden,
+                  void* out, cudaStream_t st) {
+    const int H = ctx->shape.H;
+    const uintptr_t pg = reinterpret_cast<uintptr_t>(w_gate), pu = reinterpret_cast<uintptr_t>(w_up);
+    if (pg == pu) return DIRECTOR_ERR_UNSUPPORTED;
+    const bool gate_first = pg < pu;
+    const uint64_t delta = gate_first ? pu - pg : pg - pu;
+    if (delta % 16 != 0 || delta >= (1ull << 40)) return DIRECTOR_ERR_UNSUPPORTED;
+    CUtensorMap m_in, m_gu, m_h, m_d;
+    if (!map_2d(ctx, &m_in, in, rows, H) || !map_2d(ctx, &m_h, hidden, rows, Fw) ||
+        !map_2d(ctx, &m_d, w_down, n_experts * H, Fw))
+        return DIRECTOR_ERR_CUDA;
+    if (!map_interleaved(ctx, &m_gu, gate_first ? w_gate : w_up, delta, n_experts * Fw, H)) return DIRECTOR_ERR_UNSUPPORTED;
+    SwapParams p1{seg_offsets, slot_expert, G, Fw / 128, H / BLOCK_K, Fw, Fw, gate_first ? 1 : 0, hidden, ctx->d_status};
+    int rc = launch_swap<0, EPI_GROUPS_GEMM1>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, p1, st);
+    if (rc != DIRECTOR_OK) return rc;
+    SwapParams p2{seg_offsets, slot_expert, G, H / 256, Fw / BLOCK_K, H, H, 1, out, ctx->d_status};
+    return launch_swap<1, EPI_GROUPS_GEMM2>(ctx, "grouped_gemm_down_kernel", m_d, m_h, p2, st);
+}
+
+}  // namespace director

@@ -277,3 +277,19 @@ def test_host_buffer_entry_points_match_the_device_path():
         assert np.array_equal(b["load"].numpy(), b["load_ref"])
     assert d.last_status() == 0
     assert case.layer.d.lib.director_layer_wait_host(d._ctx, 10 ** 6) == 1      # unknown ticket
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2])
+def test_every_ffn_tile_scheme_matches_the_oracle_and_the_others(variant):
+    """The three tile schemes of the expert-FFN GEMMs (single CTA, CTA pair, weight-stationary CTA pair)
+    accumulate every output in the same order, so they must agree bit for bit, and each must match the oracle."""
+    shape, logits, x, weights = _custom(71, 1500, 512, 16, 2, 384, 2, 4, 5, 1.0)
+    X = _random_placement(71, 16, 4, 5, 4)
+    case = GpuCase(shape, logits, x, weights)
+    case.layer.d.set_ffn_variant(variant)
+    g = case.run(X)
+    idx, w, w64, d, c = _oracle_front(shape, logits, x, X, 5)
+    _check_outputs(shape, g, x, weights, idx, w, w64, d, c, np.arange(0, 1500, 7), f"variant{variant}")
+    case.layer.d.set_ffn_variant(0)
+    g0 = case.run(X)
+    assert np.array_equal(g.yp, g0.yp) and np.array_equal(g.y, g0.y) and np.array_equal(g.y_shared, g0.y_shared)
