@@ -282,7 +282,7 @@ STAGE_KERNELS = {
     "dispatch": ["dispatch_count_scan_kernel", "dispatch_index_kernel", "dispatch_scatter_rows_kernel"],
     "expert_ffn": ["grouped_gemm_swiglu_kernel", "grouped_gemm_down_kernel", "one_segment_kernel"],
     "combine": ["combine_kernel"],
-    "placement_cost": ["cost_count_scan_kernel", "cost_kernel"],
+    "placement_cost": ["cost_workload_hist_kernel", "cost_from_workload_kernel", "cost_count_scan_kernel", "cost_kernel"],
 }
 
 

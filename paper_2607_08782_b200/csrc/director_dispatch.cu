@@ -73,10 +73,17 @@ count_scan_kernel(const int32_t* __restrict__ topk_idx, int T, int E, int K, int
     __syncthreads();
     for (int e = threadIdx.x; e < E; e += blockDim.x) {
         int run = 0;
-        for (int i = 0; i < n_tiles; ++i) {
-            const int c = __ldcg(tile_counts + (size_t)i * E + e);
-            tile_counts[(size_t)i * E + e] = run;
-            run += c;
+        // chunks of 16 tiles: all loads of a chunk are issued before the first store, so the loop runs at
+        // memory throughput instead of one L2 round trip per tile
+        for (int i0 = 0; i0 < n_tiles; i0 += 16) {
+            int c[16];
+#pragma unroll
+            for (int k = 0; k < 16; ++k) c[k] = (i0 + k < n_tiles) ? __ldcg(tile_counts + (size_t)(i0 + k) * E + e) : 0;
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                if (i0 + k < n_tiles) tile_counts[(size_t)(i0 + k) * E + e] = run;
+                run += c[k];
+            }
         }
         const int r0 = rep_start[e], r_e = rep_start[e + 1] - r0;
         for (int q = 0; q < r_e; ++q)               // replica q gets ceil((N_e - q) / r_e) rows
@@ -232,6 +239,93 @@ cost_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ sr
         if (h_load[i]) atomicAdd(rank_load + i, (unsigned long long)h_load[i]);
 }
 
+// ---- placement cost, fast path for the default block partition of tokens over source ranks ----
+//
+// With src(t) = floor(t*R/T) the tokens of a source rank are a contiguous range, and the n-th assignment of
+// an expert is numbered in ascending token order, so the assignments that rank j sends to expert e occupy a
+// contiguous range [a, b) of n.  Round-robin over r replicas gives replica q exactly
+//     f(b) - f(a),  f(x) = max(0, ceil((x - q) / r))
+// of them.  The whole cost therefore follows from the workload matrix W alone: one histogram kernel and one
+// warp-per-expert kernel, no per-assignment ranks.
+
+constexpr int kHistSmemInts = 4096;
+
+__global__ void __launch_bounds__(kTokenTile)
+workload_hist_kernel(const int32_t* __restrict__ topk_idx, int T, int E, int K, int R,
+                     unsigned long long* __restrict__ workload, unsigned long long* __restrict__ rank_load,
+                     unsigned long long* __restrict__ dispatch_tokens, unsigned long long* __restrict__ dispatch_bytes,
+                     int32_t* __restrict__ status) {
+    __shared__ uint32_t hist[kHistSmemInts];
+    if (blockIdx.x == 0) {      // the other outputs are accumulated by the next kernel: clear them here
+        for (int i = threadIdx.x; i < R * R; i += blockDim.x) { dispatch_tokens[i] = 0ull; dispatch_bytes[i] = 0ull; }
+        for (int i = threadIdx.x; i < R; i += blockDim.x) rank_load[i] = 0ull;
+    }
+    const int t0 = blockIdx.x * kTokenTile, t1 = min(t0 + kTokenTile, T) - 1;
+    const int src_lo = (int)(((long long)t0 * R) / T), src_hi = (int)(((long long)t1 * R) / T);
+    const int n_src = src_hi - src_lo + 1;
+    const bool use_smem = n_src * E <= kHistSmemInts;
+    if (use_smem) {
+        for (int i = threadIdx.x; i < n_src * E; i += blockDim.x) hist[i] = 0u;
+        __syncthreads();
+    }
+    const int t = t0 + threadIdx.x;
+    if (t < T) {
+        const int src = (int)(((long long)t * R) / T);
+        for (int s = 0; s < K; ++s) {
+            const int e = __ldg(topk_idx + (size_t)t * K + s);
+            if ((unsigned)e >= (unsigned)E) { director_set_status(status, DIRECTOR_ERR_BAD_INDEX); continue; }
+            if (use_smem) atomicAdd(&hist[(src - src_lo) * E + e], 1u);
+            else atomicAdd(workload + (size_t)src * E + e, 1ull);
+        }
+    }
+    if (use_smem) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < n_src * E; i += blockDim.x)
+            if (hist[i]) atomicAdd(workload + (size_t)src_lo * E + i, (unsigned long long)hist[i]);
+    }
+}
+
+// One warp per expert, lanes over the source ranks: prefix-scan the expert's column of W over the ranks
+// (the start a_j of rank j's range of n), split each range over the replicas, add into the outputs
+// (zeroed by workload_hist_kernel) with 64-bit global atomics.
+constexpr int kCostWarps = 8;
+
+__global__ void __launch_bounds__(kCostWarps * 32)
+cost_from_workload_kernel(const unsigned long long* __restrict__ workload, int E, int R, int C_max,
+                          const int32_t* __restrict__ rep_start, const int32_t* __restrict__ rep_slot,
+                          unsigned long long* __restrict__ rank_load, unsigned long long* __restrict__ dispatch_tokens,
+                          unsigned long long* __restrict__ dispatch_bytes, unsigned long long bytes_per_token) {
+    const int e = blockIdx.x * kCostWarps + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (e >= E) return;
+    const int r0 = __ldg(rep_start + e);
+    const uint32_t r = (uint32_t)(__ldg(rep_start + e + 1) - r0);
+    uint32_t carry = 0;                                        // assignments of e sent by ranks before this chunk
+    for (int j0 = 0; j0 < R; j0 += 32) {
+        const int j = j0 + lane;
+        const uint32_t w = j < R ? (uint32_t)workload[(size_t)j * E + e] : 0u;   // counts fit 32 bits: T*K < 2^31
+        uint32_t incl = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        const uint32_t b = carry + incl, a = b - w;            // rank j sends assignments n in [a, b)
+        if (w) {
+            for (uint32_t q = 0; q < r; ++q) {
+                const uint32_t fb = b > q ? (b - q + r - 1) / r : 0u, fa = a > q ? (a - q + r - 1) / r : 0u;
+                if (fb > fa) {
+                    const int dest = __ldg(rep_slot + r0 + q) / C_max;
+                    const unsigned long long n = fb - fa;
+                    atomicAdd(dispatch_tokens + (size_t)j * R + dest, n);
+                    atomicAdd(dispatch_bytes + (size_t)j * R + dest, n * bytes_per_token);
+                    atomicAdd(rank_load + dest, n);
+                }
+            }
+        }
+        carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    }
+}
+
 int launch_count_scan(director_ctx* ctx, const char* name, int T, const int32_t* topk_idx, int32_t* seg_a, int32_t* seg_b,
                       cudaStream_t st) {
     const director_shape& s = ctx->shape;
@@ -278,6 +372,26 @@ int launch_cost(director_ctx* ctx, int T, const int32_t* topk_idx, const int32_t
     const int n_tiles = (T + kTokenTile - 1) / kTokenTile;
     cudaError_t e;
     if ((e = cudaMemsetAsync(workload, 0, sizeof(int64_t) * s.R * s.E, st)) != cudaSuccess) return cuda_status(e);
+    if (src_rank == nullptr) {
+        {
+            LaunchScope scope(ctx, st, "cost_workload_hist_kernel");
+            workload_hist_kernel<<<n_tiles, kTokenTile, 0, st>>>(topk_idx, T, s.E, s.K, s.R,
+                                                                 reinterpret_cast<unsigned long long*>(workload),
+                                                                 reinterpret_cast<unsigned long long*>(rank_load),
+                                                                 reinterpret_cast<unsigned long long*>(dispatch_tokens),
+                                                                 reinterpret_cast<unsigned long long*>(dispatch_bytes),
+                                                                 ctx->d_status);
+            if (cudaGetLastError() != cudaSuccess) return DIRECTOR_ERR_CUDA;
+        }
+        LaunchScope scope(ctx, st, "cost_from_workload_kernel");
+        cost_from_workload_kernel<<<(s.E + kCostWarps - 1) / kCostWarps, kCostWarps * 32, 0, st>>>(reinterpret_cast<const unsigned long long*>(workload), s.E, s.R,
+                                                     s.C_max, ctx->d_rep_start, ctx->d_rep_slot,
+                                                     reinterpret_cast<unsigned long long*>(rank_load),
+                                                     reinterpret_cast<unsigned long long*>(dispatch_tokens),
+                                                     reinterpret_cast<unsigned long long*>(dispatch_bytes),
+                                                     (unsigned long long)s.H * 2ull);
+        return cuda_status(cudaGetLastError());
+    }
     if ((e = cudaMemsetAsync(rank_load, 0, sizeof(int64_t) * s.R, st)) != cudaSuccess) return cuda_status(e);
     if ((e = cudaMemsetAsync(dispatch_tokens, 0, sizeof(int64_t) * s.R * s.R, st)) != cudaSuccess) return cuda_status(e);
     if ((e = cudaMemsetAsync(dispatch_bytes, 0, sizeof(uint64_t) * s.R * s.R, st)) != cudaSuccess) return cuda_status(e);
