@@ -32,7 +32,7 @@ bool shape_supported(const director_shape& s) {
 
 void free_all(director_ctx* c) {
     void* ptrs[] = {c->d_rep_start, c->d_rep_slot, c->d_slot_expert, c->d_tile_counts, c->d_seg_offsets, c->d_ticket,
-                    c->d_status, c->d_hidden, c->d_hidden_shared, c->d_one_seg,
+                    c->d_status, c->d_hidden, c->d_hidden_shared, c->d_one_seg, c->d_sched,
                     c->d_zero_expert, c->e_logits2[0], c->e_logits2[1], c->e_x2[0], c->e_x2[1], c->e_topk_idx,
                     c->e_topk_w, c->e_xp, c->e_yp, c->e_y2[0], c->e_y2[1], c->e_y_shared, c->e_row_token, c->e_inv_row,
                     c->e_dest_rank, c->e_cost2[0], c->e_cost2[1]};
@@ -96,7 +96,7 @@ int director_create(const director_shape* shape, director_ctx** out) {
     bool ok = dev_alloc(&c->d_rep_start, s.E + 1) && dev_alloc(&c->d_rep_slot, (size_t)s.E * s.R) &&
               dev_alloc(&c->d_slot_expert, c->G) && dev_alloc(&c->d_tile_counts, (size_t)c->n_tiles_max * s.E) &&
               dev_alloc(&c->d_seg_offsets, c->G + 1) && dev_alloc(&c->d_ticket, 1) && dev_alloc(&c->d_status, 1) &&
-              dev_alloc(&c->d_one_seg, 2) &&
+              dev_alloc(&c->d_one_seg, 2) && dev_alloc(&c->d_sched, 4) &&
               dev_alloc(&c->d_zero_expert, 1) &&
               dev_alloc(reinterpret_cast<uint16_t**>(&c->d_hidden), A * s.F) &&
               dev_alloc(reinterpret_cast<uint16_t**>(&c->d_hidden_shared), T * s.S * s.F) &&

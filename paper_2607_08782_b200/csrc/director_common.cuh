@@ -49,6 +49,7 @@ struct director_ctx {
     // expert FFN workspace
     void* d_hidden = nullptr;          // bf16 [T_max*K, F]   SwiGLU activations of the routed experts
     void* d_hidden_shared = nullptr;   // bf16 [T_max, S*F]
+    unsigned int* d_sched = nullptr;   // [4] work-item counters of the GEMM launches of one expert_ffn call
     int32_t* d_one_seg = nullptr;      // [2] segment table {0, T} used for the shared experts
     int32_t* d_zero_expert = nullptr;  // [1] = {0}
 

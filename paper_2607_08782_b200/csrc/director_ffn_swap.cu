@@ -60,6 +60,37 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(cluster_bar), "r"(x), "r"(y), "r"(z) : "memory");
 }
 
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+// remote arrive that publishes this thread's earlier (remote) stores to the waiting CTA
+__device__ __forceinline__ void mbar_arrive_cluster_release(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_acquire_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_acquire_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_acquire_cluster(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    uint32_t n = 0;
+    while (!mbar_try_acquire_cluster(bar, parity)) {
+        if ((++n & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
+        }
+    }
+    return true;
+}
+
+constexpr int SCHED_SLOTS = 4;      // ring through which the leader's producer hands work items to the other roles
+
 struct SwapParams {
     const int32_t* seg_offsets;
     const int32_t* slot_expert;
@@ -71,6 +102,7 @@ struct SwapParams {
     int gate_first;            // GEMM-1: 1 if even lanes hold gate rows, 0 if they hold up rows
     void* out;
     int32_t* status;
+    unsigned int* counter;     // next unclaimed work item of this launch (zero when the kernel starts)
 };
 
 struct SwapTile {
@@ -111,9 +143,11 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     uint8_t* gen = smem_raw + (tiles - raw) + S_STAGES * S_STAGE_BYTES;
     uint64_t* bars = reinterpret_cast<uint64_t*>(gen);             // full[6] empty[6] tfull[2] tempty[2]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + 160);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + 164);
-    int32_t* warp_sum = reinterpret_cast<int32_t*>(gen + 176);     // [18]
+    // sched_full[4] at +128, sched_empty[4] at +160 (the leader's are the ones used)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + 192);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + 196);
+    volatile int* sched_item = reinterpret_cast<volatile int*>(gen + 200);   // [4]
+    int32_t* warp_sum = reinterpret_cast<int32_t*>(gen + 216);     // [10]
     int32_t* s_seg = reinterpret_cast<int32_t*>(gen + 256);
     int32_t* s_tt = s_seg + (kMaxG + 1);
     int32_t* s_exp = s_tt + (kMaxG + 1);
@@ -123,12 +157,13 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     auto empty_bar = [&](int s) { return bar0 + 8u * (S_STAGES + s); };
     auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * S_STAGES + a); };
     auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * S_STAGES + 2 + a); };
+    auto sched_full = [&](int q) { return bar0 + 128u + 8u * q; };
+    auto sched_empty = [&](int q) { return bar0 + 160u + 8u * q; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = p.G;
     const uint32_t rank = cluster_ctarank();
     const bool leader = rank == 0;
-    const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
 
     constexpr int n_threads = 64 + 128 * EPI_GROUPS;               // producer warp + MMA warp + epilogue warps
     for (int g = threadIdx.x; g <= G; g += n_threads) s_seg[g] = __ldg(p.seg_offsets + g);
@@ -137,6 +172,8 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
         *abort_flag = 0;
         for (int s = 0; s < S_STAGES; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8 * EPI_GROUPS); }
+        // a slot is free again once every consumer has read it: MMA thread, peer producer, all epilogue warps
+        for (int q = 0; q < SCHED_SLOTS; ++q) { mbar_init(sched_full(q), 1); mbar_init(sched_empty(q), 2 + 8 * EPI_GROUPS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -177,12 +214,68 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     SwapWalker walker{s_seg, s_tt, s_exp, p.w_blocks, p.w_rows_per_expert, ROWS_PER_BLOCK, s_tt[G] * p.w_blocks};
     SwapTile t;
 
+    // Work items (segment, weight block, token tile) are handed out dynamically, in their natural order, from a
+    // global counter: the leader's producer claims the next item whenever it is ready for one (it claims one
+    // ahead, so the atomic's latency hides behind the current item's loads) and publishes it through a small ring
+    // in both CTAs' shared memory.  Tail tiles are cheaper than full ones, so fixed assignments leave 6-15 % of
+    // imbalance between clusters; and since the items are still taken in order, clusters running at the same
+    // time keep working on neighbouring items and share their weight tiles in L2.
+    const int total_items = walker.total;
+    // consumer side of the ring: wait for item i, read it, hand the slot back
+    auto take_item = [&](int i, int& w) -> bool {
+        const int q = i & (SCHED_SLOTS - 1);
+        const uint32_t par = ((uint32_t)i / SCHED_SLOTS) & 1u;
+        const bool ok = leader ? mbar_wait(sched_full(q), par, abort_flag)
+                               : mbar_wait_acquire_cluster(sched_full(q), par, abort_flag);
+        if (ok) w = sched_item[q];
+        return ok;
+    };
+    auto release_item = [&](int i) {
+        const int q = i & (SCHED_SLOTS - 1);
+        if (leader) mbar_arrive(sched_empty(q));
+        else mbar_arrive_cluster(map_to_cta(sched_empty(q), 0));
+    };
+
     if (warp == 0) {
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int w = cluster_id; ok && walker.get(w, t); w += n_clusters) {
+            // leader: item i+1 is published (and item i+2 claimed) when item i starts, so neither the atomic's
+            // latency nor the trip to the peer's shared memory ever sits in front of a load
+            auto publish = [&](int i, int w) -> bool {
+                const int q = i & (SCHED_SLOTS - 1);
+                if (!mbar_wait(sched_empty(q), (((uint32_t)i / SCHED_SLOTS) & 1u) ^ 1u, abort_flag)) return false;
+                sched_item[q] = w;
+                st_cluster_u32(map_to_cta(smem_u32(const_cast<int*>(&sched_item[q])), 1), (uint32_t)w);
+                mbar_arrive(sched_full(q));
+                mbar_arrive_cluster_release(map_to_cta(sched_full(q), 1));
+                return true;
+            };
+            auto clamp_item = [&](unsigned int c) { return c < (unsigned)total_items ? (int)c : total_items; };
+            int w_cur = total_items;
+            unsigned int claim_ahead = 0u;
+            if (leader) {
+                w_cur = clamp_item(atomicAdd(p.counter, 1u));
+                claim_ahead = w_cur < total_items ? atomicAdd(p.counter, 1u) : (unsigned)total_items;
+                ok = publish(0, w_cur);
+            }
+            for (int i = 0; ok; ++i) {
+                int w;
+                if (leader) {
+                    w = w_cur;
+                    if (w < total_items) {
+                        const int w_next = clamp_item(claim_ahead);
+                        if (!(ok = publish(i + 1, w_next))) break;
+                        if (w_next < total_items) claim_ahead = atomicAdd(p.counter, 1u);
+                        w_cur = w_next;
+                    }
+                } else {
+                    if (!(ok = take_item(i, w))) break;
+                    release_item(i);
+                }
+                if (w >= total_items) break;
+                walker.get(w, t);
                 const int x_row = t.row0 + (int)rank * (t.n >> 1);          // this CTA's half of the tile's tokens
                 const int w_row = t.w_row + (int)rank * (ROWS_PER_BLOCK / 2);
                 for (int kb = 0; kb < p.k_steps; ++kb) {
@@ -199,10 +292,15 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
         }
     } else if (warp == 1) {
         if (lane == 0 && leader) {
-            int stage = 0, it = 0;
+            int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int w = cluster_id; ok && walker.get(w, t); w += n_clusters, ++it) {
+            for (int it = 0; ok; ++it) {
+                int w;
+                if (!(ok = take_item(it, w))) break;
+                release_item(it);
+                if (w >= total_items) break;
+                walker.get(w, t);
                 const int acc = it & 1;
                 if (!(ok = mbar_wait(tempty_bar(acc), (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag))) break;
                 tc_fence_after();
@@ -229,9 +327,14 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
         const int c_first = 32 * cgroup;
         uint16_t* out = static_cast<uint16_t*>(p.out);
         const int lane_row = quad * 32 + lane;                     // weight row of this thread inside the CTA's 128
-        int it = 0;
         bool ok = true;
-        for (int w = cluster_id; ok && walker.get(w, t); w += n_clusters, ++it) {
+        for (int it = 0; ok; ++it) {
+            int w;
+            if (!(ok = take_item(it, w))) break;
+            __syncwarp();
+            if (lane == 0) release_item(it);
+            if (w >= total_items) break;
+            walker.get(w, t);
             const int acc = it & 1;
             if (!(ok = mbar_wait(tfull_bar(acc), ((uint32_t)it >> 1) & 1u, abort_flag))) break;
             tc_fence_after();
@@ -359,7 +462,7 @@ int ffn_swap_init(director_ctx*) {
 // Returns DIRECTOR_ERR_UNSUPPORTED if the two weight arrays cannot be described by one interleaving map.
 int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t rows, const int32_t* seg_offsets, const int32_t* slot_expert,
                   int G, const void* w_gate, const void* w_up, const void* w_down, uint64_t n_experts, int Fw, void* hidden,
-                  void* out, cudaStream_t st) {
+                  void* out, unsigned int* counters /* 2 zeroed work-item counters */, cudaStream_t st) {
     const int H = ctx->shape.H;
     const uintptr_t pg = reinterpret_cast<uintptr_t>(w_gate), pu = reinterpret_cast<uintptr_t>(w_up);
     if (pg == pu) return DIRECTOR_ERR_UNSUPPORTED;
@@ -371,10 +474,10 @@ int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t rows, const int32_
         !map_2d(ctx, &m_d, w_down, n_experts * H, Fw))
         return DIRECTOR_ERR_CUDA;
     if (!map_interleaved(ctx, &m_gu, gate_first ? w_gate : w_up, delta, n_experts * Fw, H)) return DIRECTOR_ERR_UNSUPPORTED;
-    SwapParams p1{seg_offsets, slot_expert, G, Fw / 128, H / BLOCK_K, Fw, Fw, gate_first ? 1 : 0, hidden, ctx->d_status};
+    SwapParams p1{seg_offsets, slot_expert, G, Fw / 128, H / BLOCK_K, Fw, Fw, gate_first ? 1 : 0, hidden, ctx->d_status, counters};
     int rc = launch_swap<0, EPI_GROUPS_GEMM1>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, p1, st);
     if (rc != DIRECTOR_OK) return rc;
-    SwapParams p2{seg_offsets, slot_expert, G, H / 256, Fw / BLOCK_K, H, H, 1, out, ctx->d_status};
+    SwapParams p2{seg_offsets, slot_expert, G, H / 256, Fw / BLOCK_K, H, H, 1, out, ctx->d_status, counters + 1};
     return launch_swap<1, EPI_GROUPS_GEMM2>(ctx, "grouped_gemm_down_kernel", m_d, m_h, p2, st);
 }
 
