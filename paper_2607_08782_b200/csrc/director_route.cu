@@ -3,10 +3,11 @@
 //
 // LPT lanes per token (1, 2, 4 or 8, chosen from E), no branches that depend on the data.  A lane streams
 // every LPT-th group of eight logits of its token's row (two 16-byte loads; the lanes of a token read
-// adjacent groups, so a token's loads are contiguous), turns each logit into a 64-bit key
-//     (order-preserving image of the float) << 32 | (0xFFFFFFFF - expert id)
-// so that a plain unsigned comparison orders by (logit descending, expert id ascending), sorts the
-// eight keys with a 19-comparator network and merges them into the running top-8 (element-wise max
+// adjacent groups, so a token's loads are contiguous), turns each logit into the key
+//     (order-preserving 32-bit image of the float) << 8 | (255 - expert id)        (E <= 256)
+// which orders by (logit descending, expert id ascending) under a plain unsigned 64-bit comparison.
+// The lane sorts its eight keys with a 19-comparator network and merges them into the running top-8
+// (element-wise max
 // against the reversed list gives a bitonic sequence holding the 8 largest; 12 more comparators
 // sort it).  The lanes of a token then merge their lists pairwise through shuffles with the same step.
 // The weights are the softmax over the K winning logits, which equals the full softmax renormalised
@@ -28,14 +29,23 @@ __device__ __forceinline__ float bits_to_float(uint32_t k) {
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
 
+typedef unsigned long long rkey;
+
+__device__ __forceinline__ rkey make_key(uint32_t ordered, uint32_t expert) {
+    return ((unsigned long long)ordered << 8) | (255u - expert);
+}
+__device__ __forceinline__ unsigned long long key_bits(rkey k) { return k; }
+__device__ __forceinline__ rkey key_floor() { return 0ull; }   // below every real key
+
 // compare-exchange: afterwards a >= b
-__device__ __forceinline__ void cx(unsigned long long& a, unsigned long long& b) {
-    const unsigned long long hi = a > b ? a : b, lo = a > b ? b : a;
+__device__ __forceinline__ void cx(rkey& a, rkey& b) {
+    const bool swap = b > a;
+    const rkey hi = swap ? b : a, lo = swap ? a : b;
     a = hi;
     b = lo;
 }
 
-__device__ __forceinline__ void sort8_desc(unsigned long long (&k)[8]) {
+__device__ __forceinline__ void sort8_desc(rkey (&k)[8]) {
     cx(k[0], k[1]); cx(k[2], k[3]); cx(k[4], k[5]); cx(k[6], k[7]);
     cx(k[0], k[2]); cx(k[1], k[3]); cx(k[4], k[6]); cx(k[5], k[7]);
     cx(k[1], k[2]); cx(k[5], k[6]); cx(k[0], k[4]); cx(k[3], k[7]);
@@ -46,7 +56,7 @@ __device__ __forceinline__ void sort8_desc(unsigned long long (&k)[8]) {
 }
 
 // top[] and grp[] sorted descending -> top[] = the 8 largest of the 16, sorted descending
-__device__ __forceinline__ void merge_top8(unsigned long long (&top)[8], const unsigned long long (&grp)[8]) {
+__device__ __forceinline__ void merge_top8(rkey (&top)[8], const rkey (&grp)[8]) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) top[i] = top[i] > grp[7 - i] ? top[i] : grp[7 - i];
     cx(top[0], top[4]); cx(top[1], top[5]); cx(top[2], top[6]); cx(top[3], top[7]);
@@ -65,13 +75,13 @@ route_topk_kernel(const float* __restrict__ logits, int32_t* __restrict__ topk_i
     const int t = live ? t_raw : T - 1;                // surplus lanes redo the last token (keeps shuffles full)
     const float* row = logits + (size_t)t * E;
 
-    unsigned long long top[8];
+    rkey top[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) top[i] = 0ull;      // below every real key
+    for (int i = 0; i < 8; ++i) top[i] = key_floor();
     uint32_t max_abs = 0u;                           // largest |logit| bit pattern: >= 0x7F800000 iff Inf/NaN present
 
-    for (int e0 = 8 * sub; e0 < E; e0 += 8 * LPT) {
-        float v[8];
+    // software pipeline: the loads of the lane's next group are in flight while the current one is sorted
+    auto load_group = [&](int e0, float (&v)[8]) {
         if (VEC && e0 + 8 <= E) {
             const float4 a = __ldg(reinterpret_cast<const float4*>(row + e0));
             const float4 b = __ldg(reinterpret_cast<const float4*>(row + e0 + 4));
@@ -80,22 +90,30 @@ route_topk_kernel(const float* __restrict__ logits, int32_t* __restrict__ topk_i
 #pragma unroll
             for (int i = 0; i < 8; ++i) v[i] = (e0 + i < E) ? __ldg(row + e0 + i) : 0.0f;
         }
-        unsigned long long grp[8];
+    };
+    float v[8], v_next[8];
+    if (8 * sub < E) load_group(8 * sub, v);
+    for (int e0 = 8 * sub; e0 < E; e0 += 8 * LPT) {
+        const int e_next = e0 + 8 * LPT;
+        if (e_next < E) load_group(e_next, v_next);
+        rkey grp[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const uint32_t raw = __float_as_uint(v[i]) & 0x7FFFFFFFu;
             const bool real = e0 + i < E;
             max_abs = real ? max(max_abs, raw) : max_abs;
             const uint32_t hi = raw > 0x7F800000u ? 1u : ordered_bits(v[i]);     // NaN orders below every number
-            grp[i] = real ? ((unsigned long long)hi << 32) | (uint32_t)(0xFFFFFFFFu - (uint32_t)(e0 + i)) : 0ull;
+            grp[i] = real ? make_key(hi, (uint32_t)(e0 + i)) : key_floor();
         }
         sort8_desc(grp);
         merge_top8(top, grp);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = v_next[i];
     }
     // merge the lists of the token's lanes (butterfly: afterwards every lane holds the token's top 8)
 #pragma unroll
     for (int step = 1; step < LPT; step <<= 1) {
-        unsigned long long other[8];
+        rkey other[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) other[i] = __shfl_xor_sync(0xFFFFFFFFu, top[i], step);
         max_abs = max(max_abs, __shfl_xor_sync(0xFFFFFFFFu, max_abs, step));
@@ -105,32 +123,34 @@ route_topk_kernel(const float* __restrict__ logits, int32_t* __restrict__ topk_i
     if (max_abs >= 0x7F800000u) director_set_status(status, DIRECTOR_ERR_NONFINITE);
 
     // softmax over the K winners relative to the largest
-    const float l0 = bits_to_float((uint32_t)(top[0] >> 32));
+    uint32_t win_bits[8];
+    int win_idx[8];
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+        const unsigned long long kb = key_bits(top[s]);
+        win_bits[s] = (uint32_t)(kb >> 8);
+        win_idx[s] = 255 - (int)(kb & 0xFFull);
+    }
+    const float l0 = bits_to_float(win_bits[0]);
     float p[8], sum = 0.0f;
 #pragma unroll
     for (int s = 0; s < 8; ++s) {
-        p[s] = s < K ? expf(bits_to_float((uint32_t)(top[s] >> 32)) - l0) : 0.0f;
+        p[s] = s < K ? expf(bits_to_float(win_bits[s]) - l0) : 0.0f;
         sum += p[s];
     }
     const float inv = 1.0f / sum;
     int32_t* oi = topk_idx + (size_t)t * K;
     float* ow = topk_w + (size_t)t * K;
     if (K == 8) {
-        int4 i0, i1;
-        float4 w0, w1;
-        i0.x = (int)(0xFFFFFFFFu - (uint32_t)top[0]); i0.y = (int)(0xFFFFFFFFu - (uint32_t)top[1]);
-        i0.z = (int)(0xFFFFFFFFu - (uint32_t)top[2]); i0.w = (int)(0xFFFFFFFFu - (uint32_t)top[3]);
-        i1.x = (int)(0xFFFFFFFFu - (uint32_t)top[4]); i1.y = (int)(0xFFFFFFFFu - (uint32_t)top[5]);
-        i1.z = (int)(0xFFFFFFFFu - (uint32_t)top[6]); i1.w = (int)(0xFFFFFFFFu - (uint32_t)top[7]);
-        w0 = make_float4(p[0] * inv, p[1] * inv, p[2] * inv, p[3] * inv);
-        w1 = make_float4(p[4] * inv, p[5] * inv, p[6] * inv, p[7] * inv);
-        reinterpret_cast<int4*>(oi)[0] = i0; reinterpret_cast<int4*>(oi)[1] = i1;
-        reinterpret_cast<float4*>(ow)[0] = w0; reinterpret_cast<float4*>(ow)[1] = w1;
+        reinterpret_cast<int4*>(oi)[0] = make_int4(win_idx[0], win_idx[1], win_idx[2], win_idx[3]);
+        reinterpret_cast<int4*>(oi)[1] = make_int4(win_idx[4], win_idx[5], win_idx[6], win_idx[7]);
+        reinterpret_cast<float4*>(ow)[0] = make_float4(p[0] * inv, p[1] * inv, p[2] * inv, p[3] * inv);
+        reinterpret_cast<float4*>(ow)[1] = make_float4(p[4] * inv, p[5] * inv, p[6] * inv, p[7] * inv);
     } else {
 #pragma unroll
         for (int s = 0; s < 8; ++s)
             if (s < K) {
-                oi[s] = (int)(0xFFFFFFFFu - (uint32_t)top[s]);
+                oi[s] = win_idx[s];
                 ow[s] = p[s] * inv;
             }
     }
@@ -140,9 +160,11 @@ route_topk_kernel(const float* __restrict__ logits, int32_t* __restrict__ topk_i
 
 int launch_route(director_ctx* ctx, int T, const float* logits, int32_t* topk_idx, float* topk_w, cudaStream_t st) {
     const int E = ctx->shape.E, K = ctx->shape.K;
-    // lanes per token: one per group of eight experts, at most 8 (more lanes = more parallelism for the same work)
+    // lanes per token: splitting a token over more lanes adds merge work, so use the fewest lanes (at most one per
+    // group of eight experts, at most 8) that give the GPU about 128 K threads and each lane at most four groups
     const int groups = (E + 7) / 8;
-    const int lpt = groups >= 8 ? 8 : groups >= 4 ? 4 : groups >= 2 ? 2 : 1;
+    int lpt = 1;
+    while (lpt < 8 && 2 * lpt <= groups && ((long long)T * lpt < 131072 || groups > 4 * lpt)) lpt *= 2;
     const long long threads = (long long)T * lpt;
     const dim3 grid((unsigned)((threads + kRouteThreads - 1) / kRouteThreads)), block(kRouteThreads);
     LaunchScope scope(ctx, st, "route_topk_kernel");
