@@ -37,8 +37,8 @@ UNIT = "tokens/s"
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
 # from the ncu captures summarised under profiles/ (None until a capture for that workload exists).
 NCU_TRAFFIC_BYTES = {
-    # profiles/grouped_gemm_dram_c2_mixtral.md: gate||up GEMM, full-size workload, 2 435 702 016 B read + 227 459 584 B written
-    "c2_mixtral": 2663161600,
+    # profiles/grouped_gemm_dram_c2_mixtral.md: gate||up GEMM, full-size workload, 2 424 978 176 B read + 230 159 360 B written
+    "c2_mixtral": 2655137536,
 }
 
 
