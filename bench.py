@@ -318,21 +318,16 @@ def main():
 
     import numpy as np
     import torch
-    import torch.distributed as dist
+    from paper_2607_08782_b200.multirank import Ranks
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the layer has no CPU implementation")
     torch.cuda.set_device(local_rank)
     device = f"cuda:{local_rank}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(device))
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
+    ranks = Ranks("nccl", device)
+    rank, world = ranks.rank, ranks.world
+    barrier = ranks.barrier
 
     wl, layer, logits, x, X, pname = build_layer(args, device)
     s = wl.shape
@@ -379,10 +374,7 @@ def main():
                 kernel_ms[k] = (ms / n, n // args.steps)
     layer.d.set_profiling(False)
     layer.d.check_device_status()
-    if world > 1:
-        t = torch.tensor([ms_total], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = ranks.max_over_ranks(ms_total)
     ms_per_step = ms_total / args.steps
     value = world * T * args.steps / (ms_total * 1e-3)
 
@@ -418,10 +410,7 @@ def main():
     t0 = time.perf_counter()
     layer.d.layer_forward_host(T, h_logits, h_x, *layer.w, *layer.ws, h_y[0], h_load[0], h_bytes[0])
     single_ms = (time.perf_counter() - t0) * 1e3
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = ranks.max_over_ranks(e2e_ms)
     layer.d.check_device_status()
     # the host-path result must be the same bits as the device-path result
     same = bool(torch.equal(h_y[0].cuda().view(torch.bfloat16), layer.y[:T])) and \
@@ -435,8 +424,7 @@ def main():
                   "histograms out, two batches in flight; wall clock around the loop, synchronised on both sides"}
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        ranks.close()
         return
 
     # ---- roofline of the dominant kernel and per-stage figures ----
@@ -495,8 +483,7 @@ def main():
         "ffn_tflops": round(work["ffn_flop"] / (stage_ms("expert_ffn") * 1e-3) / 1e12, 1) if stage_ms("expert_ffn") else None,
     }
     print(json.dumps(out))
-    if world > 1:
-        dist.destroy_process_group()
+    ranks.close()
 
 
 if __name__ == "__main__":
