@@ -295,6 +295,64 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def run_placement_search(args, device):
+    """Extra measurement (not the headline): candidates per second of director_placement_cost_batch, the scoring
+    loop of the placement search (Section VI-C), and one full search on the workload."""
+    import numpy as np
+    import torch
+    from paper_2607_08782_b200 import optimizer as opt
+    from paper_2607_08782_b200 import synth
+    from paper_2607_08782_b200.binding import Director
+    shape = synth.shape_for(args.config, args.tokens)
+    s = shape
+    logits = torch.from_numpy(synth.make_logits(s)).to(device)
+    d = Director(s.T, s.H, s.F, s.E, s.K, s.S, s.R, s.C_max)
+    X0 = synth.placement_from_ranks(synth.primary_ranks(s), s.R)
+    d.set_placement(X0)
+    idx = torch.empty((s.T, s.K), dtype=torch.int32, device=device)
+    w = torch.empty((s.T, s.K), dtype=torch.float32, device=device)
+    W = torch.empty((s.R, s.E), dtype=torch.int64, device=device)
+    load = torch.empty((s.R,), dtype=torch.int64, device=device)
+    dt = torch.empty((s.R, s.R), dtype=torch.int64, device=device)
+    db = torch.empty((s.R, s.R), dtype=torch.int64, device=device)
+    d.route(s.T, logits, idx, w)
+    d.placement_cost(s.T, idx, None, W, load, dt, db)
+    torch.cuda.synchronize()
+    n = 4096
+    rng = np.random.default_rng(0)
+    Xb = np.zeros((n, s.E, s.R), dtype=np.uint8)
+    for c in range(n):
+        ranks_c = np.repeat(np.arange(s.R), s.C_max)[rng.permutation(s.R * s.C_max)[:s.E]]
+        Xb[c, np.arange(s.E), ranks_c] = 1
+    Xd = torch.from_numpy(Xb).to(device)
+    o_load = torch.empty((n, s.R), dtype=torch.int64, device=device)
+    o_disp = torch.empty((n, s.R, s.R), dtype=torch.int64, device=device)
+    o_sum = torch.empty((n, 4), dtype=torch.int64, device=device)
+    for _ in range(3):
+        d.placement_cost_batch(W, n, Xd, o_load, o_disp, o_sum)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        d.placement_cost_batch(W, n, Xd, o_load, o_disp, o_sum)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    model = opt.LatencyModel(1.0, 0.0, 0.2 / (2 * s.H), 2 * s.H)
+    ev = opt.GpuPlacementEvaluator(d, W)
+    base = ev(X0[None])[0]
+    t0 = time.perf_counter()
+    res = opt.optimize_placement(W.cpu().numpy(), s.C_max, model, ev, allow_replicas=True)
+    search_s = time.perf_counter() - t0
+    print(json.dumps({
+        "metric": "placement_candidates_per_s", "value": n / (ms * 1e-3), "unit": "candidates/s", "n_gpus": 1,
+        "steps": args.steps, "ms_per_step": ms, "higher_is_better": True, "data": "synthetic",
+        "config": {"workload": WORKLOAD_TEXT[args.config], "candidates_per_call": n, "E": s.E, "R": s.R},
+        "search": {"seconds": search_s, "candidates_scored": ev.evaluated, "rounds": res["rounds"],
+                   "latency_before": float(model.latency(base[0], base[1])), "latency_after": res["latency"],
+                   "lp_bound": res["lp_bound"]}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -307,6 +365,8 @@ def main():
     ap.add_argument("--ffn-variant", type=int, default=None, choices=[0, 1, 2],
                     help="expert-FFN tile scheme: 0 = one CTA per 128x256 tile, 1 = CTA pairs (256x256); default: library's")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stage", default="layer", choices=["layer", "placement_search"],
+                    help="layer (default): the MoE layer step; placement_search: batched scoring of candidate placements")
     ap.add_argument("--sample-clocks", nargs=2, metavar=("UUID", "PATH"), help=argparse.SUPPRESS)
     args = ap.parse_args()
     if args.sample_clocks:
@@ -329,6 +389,10 @@ def main():
     rank, world = ranks.rank, ranks.world
     barrier = ranks.barrier
 
+    if args.stage == "placement_search":
+        run_placement_search(args, device)
+        ranks.close()
+        return
     wl, layer, logits, x, X, pname = build_layer(args, device)
     s = wl.shape
     T = s.T

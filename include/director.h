@@ -131,6 +131,20 @@ int director_placement_cost(director_ctx* ctx, int32_t T, const int32_t* topk_id
                             const int32_t* token_src_rank, int64_t* workload, int64_t* rank_load,
                             int64_t* dispatch_tokens, uint64_t* dispatch_bytes, void* stream);
 
+/* Batched placement cost (Section VI-C: the placement search scores many candidate placements against the
+ * same workload; Eq. 1 and Eq. 3 per candidate).  Needs no placement set on the context.
+ * workload: dev int64 [R,E], the matrix W as written by director_placement_cost for the block partition of
+ * tokens over source ranks (the closed form used here relies on each rank's tokens being contiguous).
+ * X: dev uint8 [n,E,R], n candidate placement matrices (entries 0/1; replicas allowed, round-robin split as in
+ * director_dispatch).  rank_load: dev int64 [n,R].  dispatch_tokens: dev int64 [n,R,R] (multiply by 2*H for
+ * bytes).  summary: dev int64 [n,4] = {max_j rank_load[j]  (Eq. 2's straggler),  max_j sum_{k!=j} dispatch_tokens[j][k]
+ * (Eq. 4's straggler, in tokens),  total cross-rank tokens,  1 if the candidate satisfies Eq. 6's assignment and
+ * capacity constraints else 0}.  1 <= n <= 65535.  Results equal director_placement_cost's for every valid
+ * candidate. */
+int director_placement_cost_batch(director_ctx* ctx, const int64_t* workload, int32_t n_candidates,
+                                  const uint8_t* X, int64_t* rank_load, int64_t* dispatch_tokens,
+                                  int64_t* summary, void* stream);
+
 /* Dispatch indices without a context and without any allocation.  (The paper has no counterpart:
  * this entry point exists for the library's users, not for the method.)
  *

@@ -23,7 +23,7 @@ EXPORTED = (
     "director_expert_ffn", "director_combine", "director_placement_cost", "director_layer_forward_host",
     "director_last_status", "director_launch_count", "director_set_profiling", "director_kernel_time",
     "director_status_string", "director_dispatch_index_static", "director_layer_submit_host",
-    "director_layer_wait_host", "director_set_ffn_variant",
+    "director_layer_wait_host", "director_set_ffn_variant", "director_placement_cost_batch",
 )
 
 
@@ -58,6 +58,7 @@ def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.director_combine.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp]
     lib.director_placement_cost.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp, vp]
     lib.director_layer_forward_host.argtypes = [vp, c_int32] + [vp] * 12
+    lib.director_placement_cost_batch.argtypes = [vp, vp, c_int32, vp, vp, vp, vp, vp]
     lib.director_layer_submit_host.argtypes = [vp, c_int32] + [vp] * 13
     lib.director_layer_wait_host.argtypes = [vp, c_int64]
     lib.director_dispatch_index_static.argtypes = [c_int32] * 5 + [vp] * 9
@@ -149,6 +150,12 @@ class Director:
         _check(self.lib.director_placement_cost(self._ctx, T, _ptr(topk_idx), _ptr(token_src_rank), _ptr(workload),
                                                 _ptr(rank_load), _ptr(dispatch_tokens), _ptr(dispatch_bytes),
                                                 _stream()), "director_placement_cost")
+
+    def placement_cost_batch(self, workload, n, X, rank_load, dispatch_tokens, summary):
+        """n candidate placements X (CUDA uint8 [n,E,R]) against one workload matrix (CUDA int64 [R,E])."""
+        _check(self.lib.director_placement_cost_batch(self._ctx, _ptr(workload), n, _ptr(X), _ptr(rank_load),
+                                                      _ptr(dispatch_tokens), _ptr(summary), _stream()),
+               "director_placement_cost_batch")
 
     def layer_forward_host(self, T, logits, x, w_gate, w_up, w_down, ws_gate, ws_up, ws_down, y,
                            rank_load=None, dispatch_bytes=None):

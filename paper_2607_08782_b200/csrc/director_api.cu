@@ -269,6 +269,17 @@ int director_placement_cost(director_ctx* ctx, int32_t T, const int32_t* topk_id
                        as_stream(stream));
 }
 
+int director_placement_cost_batch(director_ctx* ctx, const int64_t* workload, int32_t n_candidates, const uint8_t* X,
+                                  int64_t* rank_load, int64_t* dispatch_tokens, int64_t* summary, void* stream) {
+    REQUIRE_CTX(ctx);
+    if (n_candidates < 1 || n_candidates > 65535) return DIRECTOR_ERR_INVALID_ARG;
+    if (!workload || !X || !rank_load || !dispatch_tokens || !summary) return DIRECTOR_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(workload) | reinterpret_cast<uintptr_t>(rank_load) |
+         reinterpret_cast<uintptr_t>(dispatch_tokens) | reinterpret_cast<uintptr_t>(summary)) & 7u)
+        return DIRECTOR_ERR_INVALID_ARG;
+    return launch_cost_batch(ctx, workload, n_candidates, X, rank_load, dispatch_tokens, summary, as_stream(stream));
+}
+
 int director_layer_submit_host(director_ctx* ctx, int32_t T, const float* logits, const void* x, const void* w_gate,
                                const void* w_up, const void* w_down, const void* ws_gate, const void* ws_up,
                                const void* ws_down, void* y, int64_t* rank_load, uint64_t* dispatch_bytes, void* stream,

@@ -123,6 +123,8 @@ int launch_dispatch(director_ctx*, int T, const void* x, const int32_t* topk_idx
                     int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, cudaStream_t);
 int launch_cost(director_ctx*, int T, const int32_t* topk_idx, const int32_t* src_rank, int64_t* workload,
                 int64_t* rank_load, int64_t* dispatch_tokens, uint64_t* dispatch_bytes, cudaStream_t);
+int launch_cost_batch(director_ctx*, const int64_t* workload, int n, const uint8_t* X, int64_t* rank_load,
+                      int64_t* dispatch_tokens, int64_t* summary, cudaStream_t);
 int launch_expert_ffn(director_ctx*, int T, const void* xp, const int32_t* seg_offsets, const void* w_gate,
                       const void* w_up, const void* w_down, void* yp, const void* x, const void* ws_gate,
                       const void* ws_up, const void* ws_down, void* y_shared, cudaStream_t);

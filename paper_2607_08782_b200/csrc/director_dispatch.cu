@@ -326,6 +326,97 @@ cost_from_workload_kernel(const unsigned long long* __restrict__ workload, int E
     }
 }
 
+// ---- batched placement cost: many candidate placements against one workload matrix ----
+//
+// Section VI-C: the placement search evaluates candidate after candidate against the same predicted workload.
+// With W fixed, a candidate's per-rank load (Eq. 1) and dispatch volume (Eq. 3) follow from its placement matrix
+// alone by the closed form above, so a whole batch of candidates is one launch: one warp per (candidate, expert).
+// A candidate is given as its raw matrix X[E][R]; the replicas of an expert are its set ranks in ascending order.
+
+__global__ void __launch_bounds__(kCostWarps * 32)
+cost_batch_kernel(const unsigned long long* __restrict__ workload, int E, int R, const uint8_t* __restrict__ X,
+                  unsigned long long* __restrict__ rank_load, unsigned long long* __restrict__ dispatch_tokens) {
+    const int e = blockIdx.x * kCostWarps + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    const int c = blockIdx.y;
+    if (e >= E) return;
+    const uint8_t* xrow = X + ((size_t)c * E + e) * R;
+    // replica set of e under candidate c as two 32-bit rank masks
+    const uint32_t m0 = __ballot_sync(0xFFFFFFFFu, lane < R && xrow[lane] != 0);
+    const uint32_t m1 = __ballot_sync(0xFFFFFFFFu, lane + 32 < R && xrow[lane + 32] != 0);
+    const uint32_t r = (uint32_t)(__popc(m0) + __popc(m1));
+    if (r == 0) return;                                         // unhosted expert: candidate is flagged invalid elsewhere
+    unsigned long long* load_c = rank_load + (size_t)c * R;
+    unsigned long long* disp_c = dispatch_tokens + (size_t)c * R * R;
+    uint32_t carry = 0;
+    for (int j0 = 0; j0 < R; j0 += 32) {
+        const int j = j0 + lane;
+        const uint32_t w = j < R ? (uint32_t)workload[(size_t)j * E + e] : 0u;
+        uint32_t incl = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        const uint32_t b = carry + incl, a = b - w;
+        if (w) {
+            uint32_t rem0 = m0, rem1 = m1;
+            for (uint32_t q = 0; q < r; ++q) {                  // q-th replica = q-th set rank
+                int dest;
+                if (rem0) { dest = __ffs(rem0) - 1; rem0 &= rem0 - 1; }
+                else { dest = 32 + __ffs(rem1) - 1; rem1 &= rem1 - 1; }
+                const uint32_t fb = b > q ? (b - q + r - 1) / r : 0u, fa = a > q ? (a - q + r - 1) / r : 0u;
+                if (fb > fa) {
+                    atomicAdd(disp_c + (size_t)j * R + dest, (unsigned long long)(fb - fa));
+                    atomicAdd(load_c + dest, (unsigned long long)(fb - fa));
+                }
+            }
+        }
+        carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    }
+}
+
+// One CTA per candidate: validity (every expert hosted, at most C_max experts per rank) and the reductions the
+// objective is built from: max_j lambda_j (Eq. 2), max_j sum_{k != j} D[j][k] (Eq. 4), total cross-rank tokens.
+__global__ void __launch_bounds__(64)
+cost_batch_summary_kernel(int E, int R, int C_max, const uint8_t* __restrict__ X,
+                          const unsigned long long* __restrict__ rank_load,
+                          const unsigned long long* __restrict__ dispatch_tokens, long long* __restrict__ summary) {
+    __shared__ long long s_load[kMaxR], s_send[kMaxR];
+    __shared__ int s_bad;
+    const int c = blockIdx.x, j = threadIdx.x;
+    if (j == 0) s_bad = 0;
+    __syncthreads();
+    const uint8_t* Xc = X + (size_t)c * E * R;
+    if (j < R) {
+        int hosted = 0;
+        for (int e = 0; e < E; ++e) hosted += Xc[(size_t)e * R + j] != 0;
+        if (hosted > C_max) atomicOr(&s_bad, 1);
+        long long send = 0;
+        for (int k = 0; k < R; ++k)
+            if (k != j) send += (long long)dispatch_tokens[((size_t)c * R + j) * R + k];
+        s_send[j] = send;
+        s_load[j] = (long long)rank_load[(size_t)c * R + j];
+    }
+    for (int e = j; e < E; e += blockDim.x) {
+        int any = 0;
+        for (int k = 0; k < R; ++k) any |= Xc[(size_t)e * R + k];
+        if (!any) atomicOr(&s_bad, 1);
+    }
+    __syncthreads();
+    if (j == 0) {
+        long long max_load = 0, max_send = 0, cross = 0;
+        for (int k = 0; k < R; ++k) {
+            max_load = max(max_load, s_load[k]);
+            max_send = max(max_send, s_send[k]);
+            cross += s_send[k];
+        }
+        summary[4 * c + 0] = max_load;
+        summary[4 * c + 1] = max_send;
+        summary[4 * c + 2] = cross;
+        summary[4 * c + 3] = s_bad ? 0 : 1;
+    }
+}
+
 int launch_count_scan(director_ctx* ctx, const char* name, int T, const int32_t* topk_idx, int32_t* seg_a, int32_t* seg_b,
                       cudaStream_t st) {
     const director_shape& s = ctx->shape;
@@ -364,6 +455,26 @@ int launch_dispatch(director_ctx* ctx, int T, const void* x, const int32_t* topk
         rc = cuda_status(cudaGetLastError());
     }
     return rc;
+}
+
+int launch_cost_batch(director_ctx* ctx, const int64_t* workload, int n, const uint8_t* X, int64_t* rank_load,
+                      int64_t* dispatch_tokens, int64_t* summary, cudaStream_t st) {
+    const director_shape& s = ctx->shape;
+    if (cudaMemsetAsync(rank_load, 0, sizeof(int64_t) * (size_t)n * s.R, st) != cudaSuccess ||
+        cudaMemsetAsync(dispatch_tokens, 0, sizeof(int64_t) * (size_t)n * s.R * s.R, st) != cudaSuccess)
+        return DIRECTOR_ERR_CUDA;
+    {
+        LaunchScope scope(ctx, st, "cost_batch_kernel");
+        cost_batch_kernel<<<dim3((s.E + kCostWarps - 1) / kCostWarps, n), kCostWarps * 32, 0, st>>>(
+            reinterpret_cast<const unsigned long long*>(workload), s.E, s.R, X,
+            reinterpret_cast<unsigned long long*>(rank_load), reinterpret_cast<unsigned long long*>(dispatch_tokens));
+        if (cudaGetLastError() != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    }
+    LaunchScope scope(ctx, st, "cost_batch_summary_kernel");
+    cost_batch_summary_kernel<<<n, 64, 0, st>>>(s.E, s.R, s.C_max, X, reinterpret_cast<const unsigned long long*>(rank_load),
+                                                reinterpret_cast<const unsigned long long*>(dispatch_tokens),
+                                                reinterpret_cast<long long*>(summary));
+    return cuda_status(cudaGetLastError());
 }
 
 int launch_cost(director_ctx* ctx, int T, const int32_t* topk_idx, const int32_t* src_rank, int64_t* workload,
