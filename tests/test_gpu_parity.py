@@ -293,3 +293,33 @@ def test_every_ffn_tile_scheme_matches_the_oracle_and_the_others(variant):
     case.layer.d.set_ffn_variant(0)
     g0 = case.run(X)
     assert np.array_equal(g.yp, g0.yp) and np.array_equal(g.y, g0.y) and np.array_equal(g.y_shared, g0.y_shared)
+
+
+def test_single_expert_reduces_to_a_dense_swiglu_mlp():
+    """E = K = R = 1: routing and permutation are the identity and the layer is a dense SwiGLU MLP, which is three
+    library matrix products (written out here with NumPy, not through the oracle)."""
+    shape, logits, x, weights = _custom(91, 333, 512, 1, 1, 384, 0, 1, 1, 1.0)
+    X = np.ones((1, 1), dtype=np.uint8)
+    case = GpuCase(shape, logits, x, weights)
+    g = case.run(X)
+    assert g.status == 0
+    assert np.array_equal(g.topk_idx, np.zeros((333, 1), dtype=np.int32)) and np.allclose(g.topk_w, 1.0)
+    assert np.array_equal(g.inv_row.ravel(), np.arange(333)) and g.seg_offsets.tolist() == [0, 333]
+    assert np.array_equal(g.xp, x)
+    f = lambda b: (b.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    xv, wg, wu, wd = f(x), f(weights.w_gate[0]), f(weights.w_up[0]), f(weights.w_down[0])
+    gv = xv @ wg.T
+    want = ((gv / (1.0 + np.exp(-gv))) * (xv @ wu.T)) @ wd.T
+    got = f(g.y)
+    assert rel_l2(got, want) <= REL_L2_TOL and max_abs(got, want) <= MAX_ABS_TOL
+    assert g.rank_load.tolist() == [333] and g.dispatch_tokens.tolist() == [[333]]
+
+
+def test_k1_and_minimum_hidden_size_with_t_below_t_max():
+    """K = 1, H = 256 (the smallest supported), a context created for a larger T_max than the batch."""
+    shape, logits, x, weights = _custom(92, 100, 256, 9, 1, 128, 0, 3, 3, 1.5)
+    X = _random_placement(92, 9, 3, 3, 0)
+    case = GpuCase(shape, logits, x, weights, T_max=4096)
+    g = case.run(X, T=100)
+    idx, w, w64, d, c = _oracle_front(shape, logits, x, X, 3)
+    _check_outputs(shape, g, x, weights, idx, w, w64, d, c, np.arange(100), "k1")
