@@ -364,6 +364,8 @@ def main():
     ap.add_argument("--placement", default="auto", choices=["auto", "primary"])
     ap.add_argument("--ffn-variant", type=int, default=None, choices=[0, 1, 2],
                     help="expert-FFN tile scheme: 0 = one CTA per 128x256 tile, 1 = CTA pairs (256x256); default: library's")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay the device-resident step from a CUDA graph (decode-sized batches); no per-kernel timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--stage", default="layer", choices=["layer", "placement_search"],
                     help="layer (default): the MoE layer step; placement_search: batched scoring of candidate placements")
@@ -416,18 +418,29 @@ def main():
         layer.forward(T, logits, x)
     barrier()
     torch.cuda.synchronize()
-    layer.d.set_profiling(True)
+    graph, launches_per_pass = None, 0
+    if args.graph:
+        n_c = layer.d.launch_count()
+        graph = layer.capture(T, logits, x)
+        launches_per_pass = (layer.d.launch_count() - n_c) // 2      # capture() runs the pass twice (warm-up + record)
+    else:
+        layer.d.set_profiling(True)
     n0 = layer.d.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     wall0 = time.time()
     ev0.record()
     for _ in range(args.steps):
-        layer.forward(T, logits, x)
+        if graph is None:
+            layer.forward(T, logits, x)
+        else:
+            graph.replay()
     ev1.record()
     torch.cuda.synchronize()
     wall1 = time.time()
     barrier()
     launches = layer.d.launch_count() - n0
+    if graph is not None:                                  # replays launch the kernels recorded in the graph
+        launches = args.steps * launches_per_pass
     ms_total = ev0.elapsed_time(ev1)
     clocks = sampler.stop(wall0, wall1) if sampler else {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
     kernel_ms = {}
@@ -542,7 +555,7 @@ def main():
                    "l2": "inputs larger than L2: every step streams the expert weights "
                          f"({3 * s.E * s.F * s.H * 2 / 1e9:.2f} GB) and activations through HBM",
                    "parallelism": "single GPU, logical ranks" if world == 1 else f"{world} independent replicas"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "cuda_graph": bool(args.graph), "roofline": roofline,
         "cpu_baseline": cpu_baseline, "stages": stages, "kernels": kernels,
         "ffn_tflops": round(work["ffn_flop"] / (stage_ms("expert_ffn") * 1e-3) / 1e12, 1) if stage_ms("expert_ffn") else None,
     }

@@ -77,3 +77,17 @@ class MoELayer:
         if with_cost:
             self.placement_cost(T)
         return self.y[:T]
+
+    def capture(self, T, logits, x, with_cost=True):
+        """Records one pass of the layer (fixed T, fixed input and output buffers) into a CUDA graph and returns it;
+        `graph.replay()` re-runs the pass with a single launch, which matters for decode-sized batches where the
+        nine kernel launches cost more than the kernels.  Per-kernel profiling must be off while capturing."""
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):                      # first pass outside the capture: lazy module loading
+            self.forward(T, logits, x, with_cost)
+        torch.cuda.current_stream().wait_stream(side)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.forward(T, logits, x, with_cost)
+        return graph

@@ -323,3 +323,32 @@ def test_k1_and_minimum_hidden_size_with_t_below_t_max():
     g = case.run(X, T=100)
     idx, w, w64, d, c = _oracle_front(shape, logits, x, X, 3)
     _check_outputs(shape, g, x, weights, idx, w, w64, d, c, np.arange(100), "k1")
+
+
+def test_cuda_graph_replay_reproduces_the_direct_pass():
+    """Every entry point is capturable: a graph of the whole layer replays to the same bits, also after the
+    inputs in the captured buffers have changed."""
+    import torch
+    from paper_2607_08782_b200.layer import tensor_to_bf16_bits
+    shape, logits, x, weights = _custom(95, 200, 256, 16, 4, 256, 1, 4, 5, 1.2)
+    X = _random_placement(95, 16, 4, 5, 3)
+    case = GpuCase(shape, logits, x, weights)
+    L, T = case.layer, shape.T
+    L.set_placement(X)
+    L.forward(T, case.logits, case.x)
+    torch.cuda.synchronize()
+    y_direct, load_direct = tensor_to_bf16_bits(L.y[:T]).copy(), L.rank_load.cpu().numpy().copy()
+    graph = L.capture(T, case.logits, case.x)
+    L.y.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert np.array_equal(tensor_to_bf16_bits(L.y[:T]), y_direct) and np.array_equal(L.rank_load.cpu().numpy(), load_direct)
+    # new inputs written into the captured buffers
+    case.logits.copy_(torch.roll(case.logits, 5, dims=1))
+    graph.replay()
+    torch.cuda.synchronize()
+    y_graph = tensor_to_bf16_bits(L.y[:T]).copy()
+    L.forward(T, case.logits, case.x)
+    torch.cuda.synchronize()
+    assert np.array_equal(tensor_to_bf16_bits(L.y[:T]), y_graph)
+    assert L.d.last_status() == 0
