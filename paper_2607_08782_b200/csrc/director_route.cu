@@ -1,17 +1,22 @@
 // (a1) Top-k softmax gating: Section II-A "the gating network computes relevance scores and
 // selects a small subset of experts ... weighted summation based on the scores".
 //
-// LPT lanes per token (1, 2, 4 or 8, chosen from E), no branches that depend on the data.  A lane streams
-// every LPT-th group of eight logits of its token's row (two 16-byte loads; the lanes of a token read
-// adjacent groups, so a token's loads are contiguous), turns each logit into the key
-//     (order-preserving 32-bit image of the float) << 8 | (255 - expert id)        (E <= 256)
-// which orders by (logit descending, expert id ascending) under a plain unsigned 64-bit comparison.
-// The lane sorts its eight keys with a 19-comparator network and merges them into the running top-8
-// (element-wise max
-// against the reversed list gives a bitonic sequence holding the 8 largest; 12 more comparators
-// sort it).  The lanes of a token then merge their lists pairwise through shuffles with the same step.
-// The weights are the softmax over the K winning logits, which equals the full softmax renormalised
-// over the winners.  HBM traffic is 4E bytes in and 8K bytes out per token.
+// LPT lanes per token (1, 2, 4 or 8, chosen from E and T), no data-dependent branches on the common path.
+// A lane streams every LPT-th group of eight logits of its token's row (two 16-byte loads, the next group
+// prefetched; the lanes of a token read adjacent groups, so a token's loads are contiguous).
+//
+// Fast path, 32-bit keys: key = (top 24 bits of the order-preserving image of the float) << 8 | (255 - expert).
+// A compare-exchange on such keys is one integer max and one integer min.  The lane sorts its eight keys with a
+// 19-comparator network and merges them into its running top-8 (element-wise max against the reversed list
+// gives a bitonic sequence holding the 8 largest; 12 more comparators sort it); the largest key ever rejected
+// is tracked too.  The token's lanes then merge their lists pairwise through shuffles.  Dropping the float's low
+// 8 bits cannot change the answer if the K winners and the best rejected element all differ in the 24 bits
+// kept - then their order is the order of the exact values and everything else is strictly smaller.  That is
+// checked, and the rare token that fails the check (two candidates within 2^-15 of each other, or real ties)
+// is redone by one lane with exact 64-bit keys (logit image << 8 | 255 - expert), which order by (logit
+// descending, expert id ascending).  Winners' exact logits are re-read by index for the weights.
+// The weights are the softmax over the K winning logits, which equals the full softmax renormalised over the
+// winners.  HBM traffic is 4E bytes in and 8K bytes out per token.
 #include "director_common.cuh"
 
 namespace director {
@@ -64,6 +69,53 @@ __device__ __forceinline__ void merge_top8(rkey (&top)[8], const rkey (&grp)[8])
     cx(top[0], top[1]); cx(top[2], top[3]); cx(top[4], top[5]); cx(top[6], top[7]);
 }
 
+// ---- 32-bit fast path ----
+__device__ __forceinline__ void cx32(uint32_t& a, uint32_t& b) {
+    const uint32_t hi = max(a, b), lo = min(a, b);
+    a = hi;
+    b = lo;
+}
+__device__ __forceinline__ void sort8_desc32(uint32_t (&k)[8]) {
+    cx32(k[0], k[1]); cx32(k[2], k[3]); cx32(k[4], k[5]); cx32(k[6], k[7]);
+    cx32(k[0], k[2]); cx32(k[1], k[3]); cx32(k[4], k[6]); cx32(k[5], k[7]);
+    cx32(k[1], k[2]); cx32(k[5], k[6]); cx32(k[0], k[4]); cx32(k[3], k[7]);
+    cx32(k[1], k[5]); cx32(k[2], k[6]);
+    cx32(k[1], k[4]); cx32(k[3], k[6]);
+    cx32(k[2], k[4]); cx32(k[3], k[5]);
+    cx32(k[3], k[4]);
+}
+// as merge_top8, also folding the rejected keys into `rej` (the largest key not in top[])
+__device__ __forceinline__ void merge_top8_32(uint32_t (&top)[8], const uint32_t (&grp)[8], uint32_t& rej) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint32_t hi = max(top[i], grp[7 - i]), lo = min(top[i], grp[7 - i]);
+        top[i] = hi;
+        rej = max(rej, lo);
+    }
+    cx32(top[0], top[4]); cx32(top[1], top[5]); cx32(top[2], top[6]); cx32(top[3], top[7]);
+    cx32(top[0], top[2]); cx32(top[1], top[3]); cx32(top[4], top[6]); cx32(top[5], top[7]);
+    cx32(top[0], top[1]); cx32(top[2], top[3]); cx32(top[4], top[5]); cx32(top[6], top[7]);
+}
+
+// Exact top-8 of a whole row by one thread with 64-bit keys (the fallback of the fast path).
+__device__ __noinline__ void exact_top8(const float* __restrict__ row, int E, rkey (&top)[8]) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) top[i] = key_floor();
+    for (int e0 = 0; e0 < E; e0 += 8) {
+        rkey grp[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const bool real = e0 + i < E;
+            const float v = real ? __ldg(row + e0 + i) : 0.0f;
+            const uint32_t raw = __float_as_uint(v) & 0x7FFFFFFFu;
+            const uint32_t hi = raw > 0x7F800000u ? 1u : ordered_bits(v);     // NaN orders below every number
+            grp[i] = real ? make_key(hi, (uint32_t)(e0 + i)) : key_floor();
+        }
+        sort8_desc(grp);
+        merge_top8(top, grp);
+    }
+}
+
 // VEC: the row can be read with 16-byte loads (E % 4 == 0; rows are then 16-byte aligned).
 template <bool VEC, int LPT>
 __global__ void __launch_bounds__(kRouteThreads)
@@ -75,9 +127,10 @@ route_topk_kernel(const float* __restrict__ logits, int32_t* __restrict__ topk_i
     const int t = live ? t_raw : T - 1;                // surplus lanes redo the last token (keeps shuffles full)
     const float* row = logits + (size_t)t * E;
 
-    rkey top[8];
+    uint32_t top[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) top[i] = key_floor();
+    for (int i = 0; i < 8; ++i) top[i] = 0u;        // below every real key
+    uint32_t rej = 0u;                               // largest key seen that is not in top[]
     uint32_t max_abs = 0u;                           // largest |logit| bit pattern: >= 0x7F800000 iff Inf/NaN present
 
     // software pipeline: the loads of the lane's next group are in flight while the current one is sorted
@@ -96,41 +149,59 @@ route_topk_kernel(const float* __restrict__ logits, int32_t* __restrict__ topk_i
     for (int e0 = 8 * sub; e0 < E; e0 += 8 * LPT) {
         const int e_next = e0 + 8 * LPT;
         if (e_next < E) load_group(e_next, v_next);
-        rkey grp[8];
+        uint32_t grp[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const uint32_t raw = __float_as_uint(v[i]) & 0x7FFFFFFFu;
             const bool real = e0 + i < E;
             max_abs = real ? max(max_abs, raw) : max_abs;
             const uint32_t hi = raw > 0x7F800000u ? 1u : ordered_bits(v[i]);     // NaN orders below every number
-            grp[i] = real ? make_key(hi, (uint32_t)(e0 + i)) : key_floor();
+            grp[i] = real ? (hi & 0xFFFFFF00u) | (255u - (uint32_t)(e0 + i)) : 0u;
         }
-        sort8_desc(grp);
-        merge_top8(top, grp);
+        sort8_desc32(grp);
+        merge_top8_32(top, grp, rej);
 #pragma unroll
         for (int i = 0; i < 8; ++i) v[i] = v_next[i];
     }
     // merge the lists of the token's lanes (butterfly: afterwards every lane holds the token's top 8)
 #pragma unroll
     for (int step = 1; step < LPT; step <<= 1) {
-        rkey other[8];
+        uint32_t other[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) other[i] = __shfl_xor_sync(0xFFFFFFFFu, top[i], step);
+        rej = max(rej, __shfl_xor_sync(0xFFFFFFFFu, rej, step));
         max_abs = max(max_abs, __shfl_xor_sync(0xFFFFFFFFu, max_abs, step));
-        merge_top8(top, other);
+        merge_top8_32(top, other, rej);
     }
     if (!live || sub != 0) return;
     if (max_abs >= 0x7F800000u) director_set_status(status, DIRECTOR_ERR_NONFINITE);
 
-    // softmax over the K winners relative to the largest
-    uint32_t win_bits[8];
-    int win_idx[8];
+    // the truncated keys decide exactly iff the K winners and the runner-up differ pairwise in the bits kept
+    bool exact = true;
 #pragma unroll
     for (int s = 0; s < 8; ++s) {
-        const unsigned long long kb = key_bits(top[s]);
-        win_bits[s] = (uint32_t)(kb >> 8);
-        win_idx[s] = 255 - (int)(kb & 0xFFull);
+        const uint32_t next = s < 7 ? top[s + 1] : rej;
+        if (s < K) exact = exact && ((top[s] >> 8) != (next >> 8));
     }
+    uint32_t win_bits[8];
+    int win_idx[8];
+    if (exact) {
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+            win_idx[s] = 255 - (int)(top[s] & 0xFFu);
+            win_bits[s] = s < K ? ordered_bits(__ldg(row + win_idx[s])) : 0u;
+        }
+    } else {
+        rkey top64[8];
+        exact_top8(row, E, top64);
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+            const unsigned long long kb = key_bits(top64[s]);
+            win_bits[s] = (uint32_t)(kb >> 8);
+            win_idx[s] = 255 - (int)(kb & 0xFFull);
+        }
+    }
+    // softmax over the K winners relative to the largest
     const float l0 = bits_to_float(win_bits[0]);
     float p[8], sum = 0.0f;
 #pragma unroll
