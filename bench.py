@@ -185,7 +185,7 @@ def build_layer(args, device):
         X, pname = placement.greedy_balanced(N, s.R, s.C_max, synth.primary_ranks(s)), "primaries + greedy replicas"
     layer.set_placement(X)
     if args.ffn_variant is not None:
-        layer.d.set_ffn_variant(args.ffn_variant)
+        layer.set_ffn_variant(args.ffn_variant)
     return wl, layer, logits, x, X, pname
 
 
@@ -364,6 +364,9 @@ def main():
     ap.add_argument("--placement", default="auto", choices=["auto", "primary"])
     ap.add_argument("--ffn-variant", type=int, default=None, choices=[0, 1, 2],
                     help="expert-FFN tile scheme: 0 = one CTA per 128x256 tile, 1 = CTA pairs (256x256); default: library's")
+    ap.add_argument("--fused", action="store_true",
+                    help="index-only dispatch + director_expert_ffn_gather (the GEMM gathers rows from x) instead of the "
+                         "materialised permutation")
     ap.add_argument("--graph", action="store_true",
                     help="replay the device-resident step from a CUDA graph (decode-sized batches); no per-kernel timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -402,7 +405,7 @@ def main():
 
     # ---- device-resident throughput ----
     for _ in range(max(args.warmup, 3)):
-        layer.forward(T, logits, x)
+        layer.forward(T, logits, x, fused=args.fused)
     torch.cuda.synchronize()
     layer.d.check_device_status()
 
@@ -415,13 +418,13 @@ def main():
             sampler = None
     # keep the GPU busy while the sampler starts so that the first samples see load clocks
     for _ in range(3):
-        layer.forward(T, logits, x)
+        layer.forward(T, logits, x, fused=args.fused)
     barrier()
     torch.cuda.synchronize()
     graph, launches_per_pass = None, 0
     if args.graph:
         n_c = layer.d.launch_count()
-        graph = layer.capture(T, logits, x)
+        graph = layer.capture(T, logits, x, fused=args.fused)
         launches_per_pass = (layer.d.launch_count() - n_c) // 2      # capture() runs the pass twice (warm-up + record)
     else:
         layer.d.set_profiling(True)
@@ -431,7 +434,7 @@ def main():
     ev0.record()
     for _ in range(args.steps):
         if graph is None:
-            layer.forward(T, logits, x)
+            layer.forward(T, logits, x, fused=args.fused)
         else:
             graph.replay()
     ev1.record()

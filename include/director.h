@@ -91,7 +91,8 @@ int director_route(director_ctx* ctx, int32_t T, const float* logits,
  * x: dev bf16 [T,H].  topk_idx: dev int32 [T,K].
  * xp: dev bf16 [T*K,H] permuted copies of the rows of x.   row_token: dev int32 [T*K], token of
  * each row.  inv_row: dev int32 [T,K], row of each assignment.  dest_rank: dev int32 [T,K].
- * seg_offsets: dev int32 [R*C_max+1], first row of each slot's segment, last entry T*K. */
+ * seg_offsets: dev int32 [R*C_max+1], first row of each slot's segment, last entry T*K.
+ * xp may be NULL: only the indices are produced (x is then not read), for use with director_expert_ffn_gather. */
 int director_dispatch(director_ctx* ctx, int32_t T, const void* x, const int32_t* topk_idx,
                       void* xp, int32_t* row_token, int32_t* inv_row, int32_t* dest_rank,
                       int32_t* seg_offsets, void* stream);
@@ -110,6 +111,21 @@ int director_expert_ffn(director_ctx* ctx, int32_t T, const void* xp, const int3
                         const void* w_gate, const void* w_up, const void* w_down, void* yp,
                         const void* x, const void* ws_gate, const void* ws_up, const void* ws_down,
                         void* y_shared, void* stream);
+
+/* (a3) fused with the row movement of (a2): the routed experts read row i of the permuted order directly as
+ * x[row_token[i]], so no permuted copy xp exists (the single-GPU analogue of hiding the dispatch cost the paper
+ * attributes to the first all-to-all, Section I).  x: dev bf16 [T,H].  row_token, seg_offsets: as written by
+ * director_dispatch (which may be called with xp = NULL).  Other arguments as for director_expert_ffn; the
+ * shared experts run iff the context has S > 0 and y_shared != NULL.  Results are bit-identical to
+ * director_dispatch + director_expert_ffn.  Needs the default tile scheme (director_set_ffn_variant 2), otherwise
+ * DIRECTOR_ERR_UNSUPPORTED.
+ * Cost: the weight-stationary GEMM reads each token tile once per 256-row weight block, so the gather is repeated
+ * 2F/256 times per token row and runs as one-row TMA boxes; it saves memory (no xp), not time - the layer's
+ * default path materialises xp once. */
+int director_expert_ffn_gather(director_ctx* ctx, int32_t T, const void* x, const int32_t* row_token,
+                               const int32_t* seg_offsets, const void* w_gate, const void* w_up,
+                               const void* w_down, void* yp, const void* ws_gate, const void* ws_up,
+                               const void* ws_down, void* y_shared, void* stream);
 
 /* (a4) Combine (Section II-A weighted summation; Section II-B second all-to-all):
  *   y[t,:] = bf16( sum_s topk_w[t,s] * yp[inv_row[t,s],:]  (+ y_shared[t,:]) ), fp32 accumulation

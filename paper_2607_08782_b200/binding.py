@@ -24,6 +24,7 @@ EXPORTED = (
     "director_last_status", "director_launch_count", "director_set_profiling", "director_kernel_time",
     "director_status_string", "director_dispatch_index_static", "director_layer_submit_host",
     "director_layer_wait_host", "director_set_ffn_variant", "director_placement_cost_batch",
+    "director_expert_ffn_gather",
 )
 
 
@@ -55,6 +56,7 @@ def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.director_route.argtypes = [vp, c_int32, vp, vp, vp, vp]
     lib.director_dispatch.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.director_expert_ffn.argtypes = [vp, c_int32] + [vp] * 12
+    lib.director_expert_ffn_gather.argtypes = [vp, c_int32] + [vp] * 12
     lib.director_combine.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp]
     lib.director_placement_cost.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp, vp]
     lib.director_layer_forward_host.argtypes = [vp, c_int32] + [vp] * 12
@@ -141,6 +143,13 @@ class Director:
         _check(self.lib.director_expert_ffn(self._ctx, T, _ptr(xp), _ptr(seg_offsets), _ptr(w_gate), _ptr(w_up),
                                             _ptr(w_down), _ptr(yp), _ptr(x), _ptr(ws_gate), _ptr(ws_up),
                                             _ptr(ws_down), _ptr(y_shared), _stream()), "director_expert_ffn")
+
+    def expert_ffn_gather(self, T, x, row_token, seg_offsets, w_gate, w_up, w_down, yp, ws_gate=None, ws_up=None,
+                          ws_down=None, y_shared=None):
+        _check(self.lib.director_expert_ffn_gather(self._ctx, T, _ptr(x), _ptr(row_token), _ptr(seg_offsets),
+                                                   _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(yp), _ptr(ws_gate),
+                                                   _ptr(ws_up), _ptr(ws_down), _ptr(y_shared), _stream()),
+               "director_expert_ffn_gather")
 
     def combine(self, T, yp, inv_row, topk_w, y_shared, y):
         _check(self.lib.director_combine(self._ctx, T, _ptr(yp), _ptr(inv_row), _ptr(topk_w), _ptr(y_shared),

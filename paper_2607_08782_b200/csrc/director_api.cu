@@ -208,9 +208,11 @@ int director_dispatch(director_ctx* ctx, int32_t T, const void* x, const int32_t
     REQUIRE_CTX(ctx);
     REQUIRE_T(ctx, T);
     REQUIRE_PLACEMENT(ctx);
-    REQUIRE_PTR(x);
     REQUIRE_PTR(topk_idx);
-    REQUIRE_PTR(xp);
+    if (xp != nullptr) {      // xp == NULL: indices only
+        REQUIRE_PTR(x);
+        REQUIRE_PTR(xp);
+    }
     REQUIRE_PTR(row_token);
     REQUIRE_PTR(inv_row);
     REQUIRE_PTR(dest_rank);
@@ -237,8 +239,34 @@ int director_expert_ffn(director_ctx* ctx, int32_t T, const void* xp, const int3
         REQUIRE_PTR(ws_down);
         REQUIRE_PTR(y_shared);
     }
-    return launch_expert_ffn(ctx, T, xp, seg_offsets, w_gate, w_up, w_down, yp, x, ws_gate, ws_up, ws_down, y_shared,
-                             as_stream(stream));
+    return launch_expert_ffn(ctx, T, xp, nullptr, seg_offsets, w_gate, w_up, w_down, yp, x, ws_gate, ws_up, ws_down,
+                             y_shared, as_stream(stream));
+}
+
+int director_expert_ffn_gather(director_ctx* ctx, int32_t T, const void* x, const int32_t* row_token,
+                               const int32_t* seg_offsets, const void* w_gate, const void* w_up, const void* w_down,
+                               void* yp, const void* ws_gate, const void* ws_up, const void* ws_down, void* y_shared,
+                               void* stream) {
+    REQUIRE_CTX(ctx);
+    REQUIRE_T(ctx, T);
+    REQUIRE_PLACEMENT(ctx);
+    REQUIRE_PTR(x);
+    REQUIRE_PTR(row_token);
+    REQUIRE_PTR(seg_offsets);
+    REQUIRE_PTR(w_gate);
+    REQUIRE_PTR(w_up);
+    REQUIRE_PTR(w_down);
+    REQUIRE_PTR(yp);
+    const bool shared = ctx->shape.S > 0 && y_shared != nullptr;
+    if (shared) {
+        REQUIRE_PTR(ws_gate);
+        REQUIRE_PTR(ws_up);
+        REQUIRE_PTR(ws_down);
+        REQUIRE_PTR(y_shared);
+    }
+    if (ctx->ffn_variant != 2) return DIRECTOR_ERR_UNSUPPORTED;
+    return launch_expert_ffn(ctx, T, nullptr, row_token, seg_offsets, w_gate, w_up, w_down, yp, x, ws_gate, ws_up, ws_down,
+                             shared ? y_shared : nullptr, as_stream(stream));
 }
 
 int director_combine(director_ctx* ctx, int32_t T, const void* yp, const int32_t* inv_row, const float* topk_w,
@@ -318,13 +346,17 @@ int director_layer_submit_host(director_ctx* ctx, int32_t T, const float* logits
     if (cudaStreamWaitEvent(st, ctx->ev_h2d_done[slot], 0) != cudaSuccess ||
         cudaStreamWaitEvent(st, ctx->ev_d2h_done[slot], 0) != cudaSuccess)
         return DIRECTOR_ERR_CUDA;
+    // the permuted rows are materialised once: the weight-stationary GEMM reads every token tile once per weight
+    // block, so gathering inside it (director_expert_ffn_gather) repeats the gather 2F/256 times and measured slower
+    const bool fused = false;
     int rc = launch_route(ctx, T, d_logits, ctx->e_topk_idx, ctx->e_topk_w, st);
     if (rc == DIRECTOR_OK)
-        rc = launch_dispatch(ctx, T, d_x, ctx->e_topk_idx, ctx->e_xp, ctx->e_row_token, ctx->e_inv_row,
+        rc = launch_dispatch(ctx, T, d_x, ctx->e_topk_idx, fused ? nullptr : ctx->e_xp, ctx->e_row_token, ctx->e_inv_row,
                              ctx->e_dest_rank, ctx->d_seg_offsets, st);
     if (rc == DIRECTOR_OK)
-        rc = launch_expert_ffn(ctx, T, ctx->e_xp, ctx->d_seg_offsets, w_gate, w_up, w_down, ctx->e_yp,
-                               shared ? d_x : nullptr, ws_gate, ws_up, ws_down, ctx->e_y_shared, st);
+        rc = launch_expert_ffn(ctx, T, ctx->e_xp, fused ? ctx->e_row_token : nullptr, ctx->d_seg_offsets, w_gate, w_up,
+                               w_down, ctx->e_yp, (shared || fused) ? d_x : nullptr, ws_gate, ws_up, ws_down,
+                               shared ? ctx->e_y_shared : nullptr, st);
     if (rc == DIRECTOR_OK)
         rc = launch_combine(ctx, T, ctx->e_yp, ctx->e_inv_row, ctx->e_topk_w, shared ? ctx->e_y_shared : nullptr, d_y, st);
     if (rc == DIRECTOR_OK) rc = launch_cost(ctx, T, ctx->e_topk_idx, nullptr, c_w, c_load, c_tok, c_bytes, st);

@@ -125,9 +125,9 @@ int launch_cost(director_ctx*, int T, const int32_t* topk_idx, const int32_t* sr
                 int64_t* rank_load, int64_t* dispatch_tokens, uint64_t* dispatch_bytes, cudaStream_t);
 int launch_cost_batch(director_ctx*, const int64_t* workload, int n, const uint8_t* X, int64_t* rank_load,
                       int64_t* dispatch_tokens, int64_t* summary, cudaStream_t);
-int launch_expert_ffn(director_ctx*, int T, const void* xp, const int32_t* seg_offsets, const void* w_gate,
-                      const void* w_up, const void* w_down, void* yp, const void* x, const void* ws_gate,
-                      const void* ws_up, const void* ws_down, void* y_shared, cudaStream_t);
+int launch_expert_ffn(director_ctx*, int T, const void* xp, const int32_t* row_token, const int32_t* seg_offsets,
+                      const void* w_gate, const void* w_up, const void* w_down, void* yp, const void* x,
+                      const void* ws_gate, const void* ws_up, const void* ws_down, void* y_shared, cudaStream_t);
 int launch_combine(director_ctx*, int T, const void* yp, const int32_t* inv_row, const float* topk_w,
                    const void* y_shared, void* y, cudaStream_t);
 

@@ -444,7 +444,7 @@ int launch_dispatch(director_ctx* ctx, int T, const void* x, const int32_t* topk
         rc = cuda_status(cudaGetLastError());
         if (rc != DIRECTOR_OK) return rc;
     }
-    {
+    if (xp != nullptr) {      // xp == nullptr: indices only (the expert FFN then gathers its rows from x itself)
         const int row_vec = s.H * 2 / 16;
         const int slices = (s.H * 2 + kSliceBytes - 1) / kSliceBytes;
         const long long items = (long long)T * slices;

@@ -26,9 +26,10 @@
 namespace director {
 
 int ffn_swap_init(director_ctx* ctx);   // director_ffn_swap.cu
-int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t rows, const int32_t* seg_offsets, const int32_t* slot_expert,
-                  int G, const void* w_gate, const void* w_up, const void* w_down, uint64_t n_experts, int Fw, void* hidden,
-                  void* out, unsigned int* counters, cudaStream_t st);
+int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int32_t* gather_rows, uint64_t rows,
+                  const int32_t* seg_offsets, const int32_t* slot_expert, int G, const void* w_gate, const void* w_up,
+                  const void* w_down, uint64_t n_experts, int Fw, void* hidden, void* out, unsigned int* counters,
+                  cudaStream_t st);
 int ffn_pair_init(director_ctx* ctx);   // director_ffn_pair.cu
 int launch_gemm_pair(director_ctx* ctx, int mode, const char* name, const CUtensorMap& a, const CUtensorMap& b0,
                      const CUtensorMap& b1, const umma::GroupedGemmParams& p, cudaStream_t st);
@@ -273,14 +274,16 @@ int launch_gemm(director_ctx* ctx, const char* name, const CUtensorMap& a, const
 }
 
 // One SwiGLU FFN pass over a segment table: in [rows, H] -> hidden [rows, Fw] -> out [rows, H].
-int ffn_pass(director_ctx* ctx, const void* in, uint64_t rows, const int32_t* seg_offsets, const int32_t* slot_expert,
-             int G, const void* w_gate, const void* w_up, const void* w_down, uint64_t n_experts, int Fw, void* hidden,
-             void* out, unsigned int* counters, cudaStream_t st) {
+int ffn_pass(director_ctx* ctx, const void* in, uint64_t in_rows, const int32_t* gather_rows, uint64_t rows,
+             const int32_t* seg_offsets, const int32_t* slot_expert, int G, const void* w_gate, const void* w_up,
+             const void* w_down, uint64_t n_experts, int Fw, void* hidden, void* out, unsigned int* counters,
+             cudaStream_t st) {
     if (ctx->ffn_variant == 2) {
-        const int rc = ffn_pass_swap(ctx, in, rows, seg_offsets, slot_expert, G, w_gate, w_up, w_down, n_experts, Fw, hidden,
-                                     out, counters, st);
+        const int rc = ffn_pass_swap(ctx, in, in_rows, gather_rows, rows, seg_offsets, slot_expert, G, w_gate, w_up, w_down,
+                                     n_experts, Fw, hidden, out, counters, st);
         if (rc != DIRECTOR_ERR_UNSUPPORTED) return rc;   // weight arrays not expressible as one map: tile scheme 0
     }
+    if (gather_rows != nullptr) return DIRECTOR_ERR_UNSUPPORTED;   // only the weight-stationary scheme gathers
     const int H = ctx->shape.H;
     CUtensorMap m_in, m_g, m_u, m_h, m_d;
     if (!make_map(ctx, &m_in, in, rows, H) || !make_map(ctx, &m_g, w_gate, n_experts * Fw, H) ||
@@ -309,23 +312,28 @@ int ffn_init(director_ctx* ctx) {
     return DIRECTOR_OK;
 }
 
-int launch_expert_ffn(director_ctx* ctx, int T, const void* xp, const int32_t* seg_offsets, const void* w_gate,
-                      const void* w_up, const void* w_down, void* yp, const void* x, const void* ws_gate,
-                      const void* ws_up, const void* ws_down, void* y_shared, cudaStream_t st) {
+// row_token == nullptr: the routed experts read the permuted rows xp.  Otherwise they gather row i as
+// x[row_token[i]] and xp is not used.
+int launch_expert_ffn(director_ctx* ctx, int T, const void* xp, const int32_t* row_token, const int32_t* seg_offsets,
+                      const void* w_gate, const void* w_up, const void* w_down, void* yp, const void* x,
+                      const void* ws_gate, const void* ws_up, const void* ws_down, void* y_shared, cudaStream_t st) {
     const director_shape& s = ctx->shape;
     // work-item counters of the (up to four) GEMM launches below
     if (cudaMemsetAsync(ctx->d_sched, 0, 4 * sizeof(unsigned int), st) != cudaSuccess) return DIRECTOR_ERR_CUDA;
-    int rc = ffn_pass(ctx, xp, (uint64_t)T * s.K, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up, w_down, s.E,
-                      s.F, ctx->d_hidden, yp, ctx->d_sched, st);
-    if (rc != DIRECTOR_OK || s.S == 0 || x == nullptr) return rc;
+    const uint64_t A = (uint64_t)T * s.K;
+    int rc = row_token ? ffn_pass(ctx, x, (uint64_t)T, row_token, A, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up,
+                                  w_down, s.E, s.F, ctx->d_hidden, yp, ctx->d_sched, st)
+                       : ffn_pass(ctx, xp, A, nullptr, A, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up, w_down,
+                                  s.E, s.F, ctx->d_hidden, yp, ctx->d_sched, st);
+    if (rc != DIRECTOR_OK || s.S == 0 || x == nullptr || y_shared == nullptr) return rc;
     {
         LaunchScope scope(ctx, st, "one_segment_kernel");
         one_segment_kernel<<<1, 1, 0, st>>>(ctx->d_one_seg, T);
         if ((rc = cuda_status(cudaGetLastError())) != DIRECTOR_OK) return rc;
     }
     // The S shared experts as one FFN of width S*F over all T rows of x (a single segment, "expert" 0).
-    return ffn_pass(ctx, x, (uint64_t)T, ctx->d_one_seg, ctx->d_zero_expert, 1, ws_gate, ws_up, ws_down, 1, s.S * s.F,
-                    ctx->d_hidden_shared, y_shared, ctx->d_sched + 2, st);
+    return ffn_pass(ctx, x, (uint64_t)T, nullptr, (uint64_t)T, ctx->d_one_seg, ctx->d_zero_expert, 1, ws_gate, ws_up,
+                    ws_down, 1, s.S * s.F, ctx->d_hidden_shared, y_shared, ctx->d_sched + 2, st);
 }
 
 }  // namespace director

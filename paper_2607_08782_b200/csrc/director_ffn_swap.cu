@@ -103,6 +103,7 @@ struct SwapParams {
     void* out;
     int32_t* status;
     unsigned int* counter;     // next unclaimed work item of this launch (zero when the kernel starts)
+    const int32_t* row_token;  // GATHER only: token of every permuted row (the tokens operand is gathered from x)
 };
 
 struct SwapTile {
@@ -134,7 +135,10 @@ struct SwapWalker {
 };
 
 // MODE 0: gate/up + SwiGLU (A from the 3-D interleaving map).  MODE 1: down projection (A from a 2-D map).
-template <int MODE, int EPI_GROUPS>
+// GATHER (GEMM-1 only): the token rows are not read from a permuted copy but gathered straight from the layer
+// input x through row_token - tm_x then describes x with a one-row box and the whole producer warp issues the
+// loads, four rows per lane - so the dispatch step needs no row copies at all.
+template <int MODE, int EPI_GROUPS, bool GATHER>
 __global__ void __launch_bounds__(64 + 128 * EPI_GROUPS, 1)
 grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
                          const SwapParams p) {
@@ -236,7 +240,79 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
         else mbar_arrive_cluster(map_to_cta(sched_empty(q), 0));
     };
 
-    if (warp == 0) {
+    if (warp == 0 && GATHER) {
+        // whole warp: lane 0 schedules and loads the weight tile, every lane gathers four token rows per k-step
+        int stage = 0;
+        uint32_t phase = 0;
+        int ok = 1;
+        auto publish = [&](int i, int w) -> bool {
+            const int q = i & (SCHED_SLOTS - 1);
+            if (!mbar_wait(sched_empty(q), (((uint32_t)i / SCHED_SLOTS) & 1u) ^ 1u, abort_flag)) return false;
+            sched_item[q] = w;
+            st_cluster_u32(map_to_cta(smem_u32(const_cast<int*>(&sched_item[q])), 1), (uint32_t)w);
+            mbar_arrive(sched_full(q));
+            mbar_arrive_cluster_release(map_to_cta(sched_full(q), 1));
+            return true;
+        };
+        auto clamp_item = [&](unsigned int c) { return c < (unsigned)total_items ? (int)c : total_items; };
+        int w_cur = total_items;
+        unsigned int claim_ahead = 0u;
+        if (lane == 0 && leader) {
+            w_cur = clamp_item(atomicAdd(p.counter, 1u));
+            claim_ahead = w_cur < total_items ? atomicAdd(p.counter, 1u) : (unsigned)total_items;
+            ok = publish(0, w_cur) ? 1 : 0;
+        }
+        ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+        for (int i = 0; ok; ++i) {
+            int w = 0;
+            if (lane == 0) {
+                if (leader) {
+                    w = w_cur;
+                    if (w < total_items) {
+                        const int w_next = clamp_item(claim_ahead);
+                        ok = publish(i + 1, w_next) ? 1 : 0;
+                        if (ok && w_next < total_items) claim_ahead = atomicAdd(p.counter, 1u);
+                        w_cur = w_next;
+                    }
+                } else {
+                    ok = take_item(i, w) ? 1 : 0;
+                    if (ok) release_item(i);
+                }
+            }
+            ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+            w = __shfl_sync(0xFFFFFFFFu, w, 0);
+            if (!ok || w >= total_items) break;
+            walker.get(w, t);
+            const int half = t.n >> 1;                                  // token rows this CTA supplies (multiple of 16)
+            const int x_row = t.row0 + (int)rank * half;
+            const int w_row = t.w_row + (int)rank * (ROWS_PER_BLOCK / 2);
+            const bool active = 4 * lane < half;
+            int tok[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {                               // rows past the tile's last token repeat it
+                const int row = min(x_row + 4 * lane + r, t.row0 + t.valid - 1);
+                tok[r] = active ? __ldg(p.row_token + row) : 0;
+            }
+            const uint32_t tx = (uint32_t)(A_BYTES + half * 128);
+            for (int kb = 0; kb < p.k_steps; ++kb) {
+                if (lane == 0) ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag) ? 1 : 0;
+                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                if (!ok) break;
+                const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
+                const uint32_t a_dst = tiles + stage * S_STAGE_BYTES;
+                if (lane == 0) {
+                    mbar_expect_tx_cluster(leader_full, tx);
+                    tma_load_3d_pair(a_dst, &tm_w, leader_full, kb * BLOCK_K, 0, w_row);
+                }
+                if (active) {
+#pragma unroll
+                    for (int r = 0; r < 4; ++r)
+                        tma_load_2d_pair(a_dst + A_BYTES + (4 * lane + r) * 128, &tm_x, leader_full, kb * BLOCK_K, tok[r]);
+                }
+                if (++stage == S_STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 0) {
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
@@ -404,11 +480,11 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// bf16 [rows, cols] row-major, box 64 x 128, 128-byte swizzle
-bool map_2d(director_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols) {
+// bf16 [rows, cols] row-major, box 64 x box_rows, 128-byte swizzle
+bool map_2d(director_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows = 128) {
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {cols * 2};
-    const cuuint32_t box[2] = {BLOCK_K, 128};
+    const cuuint32_t box[2] = {BLOCK_K, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
                map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
@@ -430,7 +506,7 @@ bool map_interleaved(director_ctx* ctx, CUtensorMap* map, const void* first, uin
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int MODE, int EPI_GROUPS>
+template <int MODE, int EPI_GROUPS, bool GATHER>
 int launch_swap(director_ctx* ctx, const char* name, const CUtensorMap& w, const CUtensorMap& x, const SwapParams& p,
                 cudaStream_t st) {
     cudaLaunchConfig_t cfg = {};
@@ -446,23 +522,27 @@ int launch_swap(director_ctx* ctx, const char* name, const CUtensorMap& w, const
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     LaunchScope scope(ctx, st, name);
-    return cuda_status(cudaLaunchKernelEx(&cfg, grouped_gemm_swap_kernel<MODE, EPI_GROUPS>, w, x, p));
+    return cuda_status(cudaLaunchKernelEx(&cfg, grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER>, w, x, p));
 }
 
 }  // namespace
 
 int ffn_swap_init(director_ctx*) {
-    if (cudaFuncSetAttribute(grouped_gemm_swap_kernel<0, EPI_GROUPS_GEMM1>, cudaFuncAttributeMaxDynamicSharedMemorySize, S_SMEM_BYTES) != cudaSuccess ||
-        cudaFuncSetAttribute(grouped_gemm_swap_kernel<1, EPI_GROUPS_GEMM2>, cudaFuncAttributeMaxDynamicSharedMemorySize, S_SMEM_BYTES) != cudaSuccess)
+    if (cudaFuncSetAttribute(grouped_gemm_swap_kernel<0, EPI_GROUPS_GEMM1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, S_SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(grouped_gemm_swap_kernel<0, EPI_GROUPS_GEMM1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, S_SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(grouped_gemm_swap_kernel<1, EPI_GROUPS_GEMM2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, S_SMEM_BYTES) != cudaSuccess)
         return DIRECTOR_ERR_CUDA;
     return DIRECTOR_OK;
 }
 
 // in [rows, H] -> hidden [rows, Fw] -> out [rows, H] over a segment table, weight-stationary pair kernels.
+// With gather_rows != nullptr, `in` is the un-permuted layer input [in_rows, H] and row i of the segment table
+// is in[gather_rows[i]].
 // Returns DIRECTOR_ERR_UNSUPPORTED if the two weight arrays cannot be described by one interleaving map.
-int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t rows, const int32_t* seg_offsets, const int32_t* slot_expert,
-                  int G, const void* w_gate, const void* w_up, const void* w_down, uint64_t n_experts, int Fw, void* hidden,
-                  void* out, unsigned int* counters /* 2 zeroed work-item counters */, cudaStream_t st) {
+int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int32_t* gather_rows, uint64_t rows,
+                  const int32_t* seg_offsets, const int32_t* slot_expert, int G, const void* w_gate, const void* w_up,
+                  const void* w_down, uint64_t n_experts, int Fw, void* hidden, void* out,
+                  unsigned int* counters /* 2 zeroed work-item counters */, cudaStream_t st) {
     const int H = ctx->shape.H;
     const uintptr_t pg = reinterpret_cast<uintptr_t>(w_gate), pu = reinterpret_cast<uintptr_t>(w_up);
     if (pg == pu) return DIRECTOR_ERR_UNSUPPORTED;
@@ -470,15 +550,17 @@ int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t rows, const int32_
     const uint64_t delta = gate_first ? pu - pg : pg - pu;
     if (delta % 16 != 0 || delta >= (1ull << 40)) return DIRECTOR_ERR_UNSUPPORTED;
     CUtensorMap m_in, m_gu, m_h, m_d;
-    if (!map_2d(ctx, &m_in, in, rows, H) || !map_2d(ctx, &m_h, hidden, rows, Fw) ||
+    if (!map_2d(ctx, &m_in, in, in_rows, H, gather_rows ? 1 : 128) || !map_2d(ctx, &m_h, hidden, rows, Fw) ||
         !map_2d(ctx, &m_d, w_down, n_experts * H, Fw))
         return DIRECTOR_ERR_CUDA;
     if (!map_interleaved(ctx, &m_gu, gate_first ? w_gate : w_up, delta, n_experts * Fw, H)) return DIRECTOR_ERR_UNSUPPORTED;
-    SwapParams p1{seg_offsets, slot_expert, G, Fw / 128, H / BLOCK_K, Fw, Fw, gate_first ? 1 : 0, hidden, ctx->d_status, counters};
-    int rc = launch_swap<0, EPI_GROUPS_GEMM1>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, p1, st);
+    SwapParams p1{seg_offsets, slot_expert, G, Fw / 128, H / BLOCK_K, Fw, Fw, gate_first ? 1 : 0, hidden, ctx->d_status,
+                  counters, gather_rows};
+    int rc = gather_rows ? launch_swap<0, EPI_GROUPS_GEMM1, true>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, p1, st)
+                         : launch_swap<0, EPI_GROUPS_GEMM1, false>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, p1, st);
     if (rc != DIRECTOR_OK) return rc;
-    SwapParams p2{seg_offsets, slot_expert, G, H / 256, Fw / BLOCK_K, H, H, 1, out, ctx->d_status, counters + 1};
-    return launch_swap<1, EPI_GROUPS_GEMM2>(ctx, "grouped_gemm_down_kernel", m_d, m_h, p2, st);
+    SwapParams p2{seg_offsets, slot_expert, G, H / 256, Fw / BLOCK_K, H, H, 1, out, ctx->d_status, counters + 1, nullptr};
+    return launch_swap<1, EPI_GROUPS_GEMM2, false>(ctx, "grouped_gemm_down_kernel", m_d, m_h, p2, st);
 }
 
 }  // namespace director

@@ -26,6 +26,7 @@ class MoELayer:
                  ws_down=None, device="cuda"):
         self.dims = dict(T_max=T_max, H=H, F=F, E=E, K=K, S=S, R=R, C_max=C_max)
         self.d = Director(T_max, H, F, E, K, S, R, C_max)
+        self.ffn_variant = 2
         self.w = (w_gate, w_up, w_down)
         self.ws = (ws_gate, ws_up, ws_down)
         A, G = T_max * K, R * C_max
@@ -49,11 +50,23 @@ class MoELayer:
     def set_placement(self, X: np.ndarray):
         self.d.set_placement(X)
 
+    def set_ffn_variant(self, variant: int):
+        """Tile scheme of the expert GEMMs (see director_set_ffn_variant); only scheme 2 can gather from x."""
+        self.d.set_ffn_variant(variant)
+        self.ffn_variant = variant
+
     def route(self, T, logits):
         self.d.route(T, logits, self.topk_idx, self.topk_w)
 
-    def dispatch(self, T, x):
-        self.d.dispatch(T, x, self.topk_idx, self.xp, self.row_token, self.inv_row, self.dest_rank, self.seg_offsets)
+    def dispatch(self, T, x, indices_only=False):
+        self.d.dispatch(T, x, self.topk_idx, None if indices_only else self.xp, self.row_token, self.inv_row,
+                        self.dest_rank, self.seg_offsets)
+
+    def expert_ffn_gather(self, T, x):
+        """The routed experts read their rows from x through row_token (no permuted copy)."""
+        S = self.dims["S"]
+        self.d.expert_ffn_gather(T, x, self.row_token, self.seg_offsets, *self.w, self.yp,
+                                 *(self.ws if S > 0 else (None, None, None)), self.y_shared if S > 0 else None)
 
     def expert_ffn(self, T, x=None):
         S = self.dims["S"]
@@ -68,26 +81,33 @@ class MoELayer:
         self.d.placement_cost(T, self.topk_idx, token_src_rank, self.workload, self.rank_load,
                               self.dispatch_tokens, self.dispatch_bytes)
 
-    def forward(self, T, logits, x, with_cost=True):
-        """One pass of the whole layer on device tensors; returns y[:T] (a view of the owned buffer)."""
+    def forward(self, T, logits, x, with_cost=True, fused=False):
+        """One pass of the whole layer on device tensors; returns y[:T] (a view of the owned buffer).
+        fused: dispatch produces indices only and the expert GEMM gathers its rows from x.  Off by default: the
+        weight-stationary GEMM re-reads a token tile once per weight block, so the gather is repeated 2F/256 times
+        and costs more than the single row copy it saves."""
         self.route(T, logits)
-        self.dispatch(T, x)
-        self.expert_ffn(T, x)
+        if fused and self.ffn_variant == 2:
+            self.dispatch(T, x, indices_only=True)
+            self.expert_ffn_gather(T, x)
+        else:
+            self.dispatch(T, x)
+            self.expert_ffn(T, x)
         self.combine(T)
         if with_cost:
             self.placement_cost(T)
         return self.y[:T]
 
-    def capture(self, T, logits, x, with_cost=True):
+    def capture(self, T, logits, x, with_cost=True, fused=False):
         """Records one pass of the layer (fixed T, fixed input and output buffers) into a CUDA graph and returns it;
         `graph.replay()` re-runs the pass with a single launch, which matters for decode-sized batches where the
         nine kernel launches cost more than the kernels.  Per-kernel profiling must be off while capturing."""
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):                      # first pass outside the capture: lazy module loading
-            self.forward(T, logits, x, with_cost)
+            self.forward(T, logits, x, with_cost, fused)
         torch.cuda.current_stream().wait_stream(side)
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
-            self.forward(T, logits, x, with_cost)
+            self.forward(T, logits, x, with_cost, fused)
         return graph

@@ -352,3 +352,28 @@ def test_cuda_graph_replay_reproduces_the_direct_pass():
     torch.cuda.synchronize()
     assert np.array_equal(tensor_to_bf16_bits(L.y[:T]), y_graph)
     assert L.d.last_status() == 0
+
+
+@pytest.mark.parametrize("seed,T,H,E,K,F,S,R,C,extra", [
+    (101, 900, 256, 12, 3, 256, 1, 4, 4, 3),
+    (102, 37, 512, 6, 2, 128, 0, 3, 3, 2),           # every tile is a short tail
+    (103, 2100, 256, 40, 4, 384, 0, 8, 6, 6),
+])
+def test_gathering_gemm_matches_the_materialised_permutation_bit_for_bit(seed, T, H, E, K, F, S, R, C, extra):
+    """director_dispatch(xp=NULL) + director_expert_ffn_gather == director_dispatch + director_expert_ffn."""
+    import torch
+    from paper_2607_08782_b200.layer import tensor_to_bf16_bits
+    shape, logits, x, weights = _custom(seed, T, H, E, K, F, S, R, C)
+    X = _random_placement(seed, E, R, C, extra)
+    case = GpuCase(shape, logits, x, weights)
+    g = case.run(X)                                           # materialised path (also checked against the oracle elsewhere)
+    L = case.layer
+    L.yp.zero_()
+    L.xp.fill_(float("nan"))                                  # the gathering path must not touch or read xp
+    L.forward(T, case.logits, case.x, fused=True)
+    torch.cuda.synchronize()
+    assert L.d.last_status() == 0
+    assert np.array_equal(tensor_to_bf16_bits(L.yp[:T * K]), g.yp)
+    assert np.array_equal(tensor_to_bf16_bits(L.y[:T]), g.y)
+    assert np.array_equal(L.inv_row[:T].cpu().numpy(), g.inv_row)
+    assert bool(torch.isnan(L.xp[:T * K]).all())
