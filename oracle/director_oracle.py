@@ -122,8 +122,12 @@ def _slot_of(hosted, C_max: int, rank: int, e: int) -> int:
 # (a2) dispatch: Section II-B "tokens are packaged and sent to the GPUs hosting their experts"
 # ----------------------------------------------------------------------------------------------
 
-def dispatch(topk_idx: np.ndarray, X: np.ndarray, C_max: int, x_bits: np.ndarray | None = None):
+def dispatch(topk_idx: np.ndarray, X: np.ndarray, C_max: int, x_bits: np.ndarray | None = None,
+             policy: str = "round_robin", src: np.ndarray | None = None):
     """Placement-aware permutation of the T*K (token, choice) assignments.
+
+    policy "local_first" is handled by dispatch_local_first (below); the text here is the default
+    round-robin rule.
 
     For expert e take its assignments in ascending token id, n = 0,1,... being the position in
     that list.  With r_e replicas on ranks reps[e][0] < reps[e][1] < ..., assignment n goes to
@@ -134,6 +138,10 @@ def dispatch(topk_idx: np.ndarray, X: np.ndarray, C_max: int, x_bits: np.ndarray
     Returns dict: row_token int32 [A], inv_row int32 [T,K], dest_rank int32 [T,K],
     seg_offsets int32 [R*C_max+1], slot_expert int32 [R*C_max], xp (uint16 [A,H] or None).
     """
+    if policy == "local_first":
+        return dispatch_local_first(topk_idx, X, C_max, x_bits, src)
+    if policy != "round_robin":
+        raise ValueError(policy)
     idx = np.asarray(topk_idx)
     T, K = idx.shape
     E, R = np.asarray(X).shape
@@ -173,6 +181,76 @@ def dispatch(topk_idx: np.ndarray, X: np.ndarray, C_max: int, x_bits: np.ndarray
         xp = np.asarray(x_bits)[row_token]       # exact row copies
     return dict(row_token=row_token, inv_row=inv_row, dest_rank=dest_rank,
                 seg_offsets=seg_offsets.astype(np.int32), slot_expert=slot_expert, xp=xp)
+
+
+def dispatch_local_first(topk_idx: np.ndarray, X: np.ndarray, C_max: int, x_bits: np.ndarray | None = None,
+                         src: np.ndarray | None = None):
+    """Locality-first replica choice (a reading of this build: the paper replicates experts to cut
+    the dispatch volume of Eq. 3 but does not say which replica a token uses).
+
+    Token t lives on rank src(t) (default: source_ranks).  Its assignment to expert e
+      * stays on rank src(t) when that rank hosts a replica of e (x_{e,src(t)} = 1);
+      * otherwise it is the m-th such "travelling" assignment of e in ascending token id
+        (m = 0,1,...) and goes to replica reps[e][m mod r_e].
+    A segment (rank, expert) holds the assignments that chose it in ascending token id; segments
+    are laid out in slot order exactly as in the round-robin rule.  Same outputs as dispatch().
+    """
+    idx = np.asarray(topk_idx)
+    T, K = idx.shape
+    Xa = np.asarray(X)
+    E, R = Xa.shape
+    A = T * K
+    reps, hosted, slot_expert = placement_tables(Xa, C_max)
+    G = R * C_max
+    src = source_ranks(T, R) if src is None else np.asarray(src)
+
+    dest_rank = np.full((T, K), -1, dtype=np.int32)
+    travelling = np.zeros(E, dtype=np.int64)            # m counter per expert
+    for t in range(T):                                  # ascending token id
+        for s in range(K):
+            e = int(idx[t, s])
+            j = int(src[t])
+            if Xa[e, j]:
+                dest_rank[t, s] = j
+            else:
+                dest_rank[t, s] = reps[e][travelling[e] % len(reps[e])]
+                travelling[e] += 1
+
+    slot = np.empty((T, K), dtype=np.int64)
+    for t in range(T):
+        for s in range(K):
+            slot[t, s] = _slot_of(hosted, C_max, int(dest_rank[t, s]), int(idx[t, s]))
+    seg_len = np.bincount(slot.reshape(-1), minlength=G)
+    seg_offsets = np.zeros(G + 1, dtype=np.int64)
+    seg_offsets[1:] = np.cumsum(seg_len)
+    assert seg_offsets[G] == A
+
+    inv_row = np.full((T, K), -1, dtype=np.int32)
+    row_token = np.full(A, -1, dtype=np.int32)
+    fill = seg_offsets[:-1].copy()
+    for t in range(T):                                  # ascending token id inside every segment
+        for s in range(K):
+            g = slot[t, s]
+            inv_row[t, s] = fill[g]
+            row_token[fill[g]] = t
+            fill[g] += 1
+    xp = None
+    if x_bits is not None:
+        xp = np.asarray(x_bits)[row_token]
+    return dict(row_token=row_token, inv_row=inv_row, dest_rank=dest_rank,
+                seg_offsets=seg_offsets.astype(np.int32), slot_expert=slot_expert, xp=xp)
+
+
+def dedup_dispatch_tokens(dest_rank: np.ndarray, src: np.ndarray, R: int) -> np.ndarray:
+    """Dispatch volume in tokens when a token whose several experts sit on one rank is sent there once:
+    U[j,k] = number of distinct tokens on rank j with at least one assignment executed on rank k.
+    (Eq. 3 counts every assignment; this is the volume a de-duplicating all-to-all would move.)"""
+    dest = np.asarray(dest_rank)
+    U = np.zeros((R, R), dtype=np.int64)
+    for t in range(dest.shape[0]):
+        for k in set(int(v) for v in dest[t] if v >= 0):
+            U[int(src[t]), k] += 1
+    return U
 
 
 # ----------------------------------------------------------------------------------------------
@@ -241,7 +319,8 @@ def combine(yp: np.ndarray, inv_row: np.ndarray, topk_w: np.ndarray, y_shared: n
 # (a5) placement cost: Section VI-A workload matrix W, Eq. 1 (load), Eq. 3 (dispatch volume)
 # ----------------------------------------------------------------------------------------------
 
-def placement_cost(topk_idx: np.ndarray, X: np.ndarray, C_max: int, H: int, src: np.ndarray | None = None):
+def placement_cost(topk_idx: np.ndarray, X: np.ndarray, C_max: int, H: int, src: np.ndarray | None = None,
+                   policy: str = "round_robin"):
     """Per executed assignment (token t on rank src(t), expert e, destination replica rank k):
     W[src, e] += 1;  rank_load[k] += 1 (Eq. 1 counted per executed assignment);
     dispatch_tokens[src, k] += 1;  dispatch_bytes = dispatch_tokens * d with d = 2*H bytes
@@ -252,7 +331,7 @@ def placement_cost(topk_idx: np.ndarray, X: np.ndarray, C_max: int, H: int, src:
     E, R = np.asarray(X).shape
     if src is None:
         src = source_ranks(T, R)
-    dest = dispatch(idx, X, C_max)["dest_rank"]
+    dest = dispatch(idx, X, C_max, policy=policy, src=src)["dest_rank"]
     W = np.zeros((R, E), dtype=np.int64)
     lam = np.zeros(R, dtype=np.int64)
     D = np.zeros((R, R), dtype=np.int64)

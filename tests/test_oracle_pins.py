@@ -447,3 +447,156 @@ def test_replicate_hottest():
     assert Y.sum() == 6 and Y[1].sum() == 2 and Y[3].sum() == 2
     assert Y[1, 0] == 1          # hottest expert -> least loaded rank (0, load 5)
     assert Y[3, 2] == 1          # second hottest -> next least loaded rank (2, load 7)
+
+
+# ------------------------------------------------------- locality-first replica choice, de-duplicated volume
+
+def _sorted_local_first(idx, X, C_max, src):
+    """Definition by lists and sorting (no running counters): per expert, the travelling assignments are those
+    whose home rank does not host it, numbered by sorting them on token id; then one global sort."""
+    T, K = idx.shape
+    E, R = X.shape
+    reps = [[j for j in range(R) if X[e, j]] for e in range(E)]
+    dest = {}
+    for e in range(E):
+        mine = sorted((t, s) for t in range(T) for s in range(K) if idx[t, s] == e)
+        away = [ts for ts in mine if not X[e, src[ts[0]]]]
+        for ts in mine:
+            dest[ts] = int(src[ts[0]]) if X[e, src[ts[0]]] else reps[e][away.index(ts) % len(reps[e])]
+    order = sorted((dest[(t, s)], int(idx[t, s]), t, s) for t in range(T) for s in range(K))
+    inv_row = np.zeros((T, K), dtype=np.int32)
+    dr = np.zeros((T, K), dtype=np.int32)
+    row_token = np.zeros(T * K, dtype=np.int32)
+    for row, (j, e, t, s) in enumerate(order):
+        inv_row[t, s], dr[t, s], row_token[row] = row, j, t
+    seg = [0]
+    for j in range(R):
+        hosted = [e for e in range(E) if X[e, j]]
+        for p in range(C_max):
+            seg.append(seg[-1] + (sum(1 for o in order if o[0] == j and o[1] == hosted[p]) if p < len(hosted) else 0))
+    return inv_row, dr, row_token, np.array(seg, dtype=np.int32)
+
+
+@pytest.mark.parametrize("seed,E,K,R,C,extra,custom_src", [(0, 8, 2, 4, 3, 4, False), (1, 8, 2, 4, 3, 4, True),
+                                                            (2, 6, 3, 3, 4, 5, True), (3, 5, 5, 2, 5, 3, False),
+                                                            (4, 4, 1, 4, 1, 0, True), (5, 8, 2, 4, 2, 0, False)])
+def test_local_first_dispatch_equals_sort_based_definition(seed, E, K, R, C, extra, custom_src):
+    rng = _rng(100 + seed)
+    T = 43
+    idx, _, _ = orc.route(rng.normal(size=(T, E)).astype(np.float32) - 0.5 * np.arange(E, dtype=np.float32), K)
+    X = _random_placement(rng, E, R, C, extra)
+    src = rng.integers(0, R, size=T).astype(np.int32) if custom_src else orc.source_ranks(T, R)
+    d = orc.dispatch(idx, X, C, policy="local_first", src=src if custom_src else None)
+    inv_row, dest, row_token, seg = _sorted_local_first(idx, X, C, src)
+    assert np.array_equal(d["inv_row"], inv_row)
+    assert np.array_equal(d["dest_rank"], dest)
+    assert np.array_equal(d["row_token"], row_token)
+    assert np.array_equal(d["seg_offsets"], seg)
+
+
+def test_local_first_without_replicas_is_the_round_robin_dispatch():
+    rng = _rng(120)
+    T, E, K, R, C = 61, 8, 2, 4, 2
+    idx, _, _ = orc.route(rng.normal(size=(T, E)).astype(np.float32), K)
+    X = _random_placement(rng, E, R, C, 0)
+    src = rng.integers(0, R, size=T).astype(np.int32)
+    a, b = orc.dispatch(idx, X, C), orc.dispatch(idx, X, C, policy="local_first", src=src)
+    for k in ("row_token", "inv_row", "dest_rank", "seg_offsets", "slot_expert"):
+        assert np.array_equal(a[k], b[k]), k
+
+
+def test_local_first_with_every_expert_everywhere_moves_nothing():
+    rng = _rng(121)
+    T, E, K, R, H = 50, 4, 2, 3, 64
+    idx, _, _ = orc.route(rng.normal(size=(T, E)).astype(np.float32), K)
+    X = np.ones((E, R), dtype=np.uint8)
+    src = orc.source_ranks(T, R)
+    d = orc.dispatch(idx, X, E, policy="local_first")
+    assert np.array_equal(d["dest_rank"], np.repeat(src[:, None], K, axis=1))
+    c = orc.placement_cost(idx, X, E, H, policy="local_first")
+    D = c["dispatch_tokens"]
+    assert np.array_equal(D, np.diag(np.bincount(src, minlength=R) * K))
+    assert orc.cost_summary(c)["cross_rank_bytes"] == 0
+    assert c["rank_load"].tolist() == (np.bincount(src, minlength=R) * K).tolist()
+
+
+def test_local_first_invariants_and_never_more_cross_traffic_than_round_robin():
+    for seed in range(6):
+        rng = _rng(130 + seed)
+        T, E, K, R, C, H = 97, 12, 3, 4, 5, 128
+        idx, _, _ = orc.route(rng.normal(size=(T, E)).astype(np.float32) - 0.3 * np.arange(E, dtype=np.float32), K)
+        X = _random_placement(rng, E, R, C, 6)
+        src = rng.integers(0, R, size=T).astype(np.int32)
+        d = orc.dispatch(idx, X, C, policy="local_first", src=src)
+        dest, inv_row, row_token, seg = d["dest_rank"], d["inv_row"], d["row_token"], d["seg_offsets"]
+        # a hosted expert is used at home; a travelling assignment lands on some replica
+        for t in range(T):
+            for s in range(K):
+                e = idx[t, s]
+                assert X[e, dest[t, s]] == 1
+                if X[e, src[t]]:
+                    assert dest[t, s] == src[t]
+        # travelling assignments of an expert are dealt round-robin: replica counts differ by at most one,
+        # earlier replicas hold the extras
+        for e in range(E):
+            tt, ss = np.nonzero(idx == e)
+            away = [dest[t, s] for t, s in zip(tt, ss) if not X[e, src[t]]]
+            reps = np.flatnonzero(X[e])
+            counts = [away.count(j) for j in reps]
+            assert max(counts) - min(counts) <= 1 and counts == sorted(counts, reverse=True)
+        # permutation structure
+        assert sorted(inv_row.reshape(-1).tolist()) == list(range(T * K))
+        assert np.array_equal(row_token[inv_row], np.repeat(np.arange(T)[:, None], K, axis=1))
+        for g in range(R * C):
+            rows = row_token[seg[g]:seg[g + 1]]
+            assert np.all(np.diff(rows) > 0)                       # ascending token id, no token twice
+            if len(rows):
+                e = d["slot_expert"][g]
+                assert e >= 0 and all(e in idx[t] for t in rows)
+        # Eq. 3 volume off the diagonal can only shrink
+        lf = orc.cost_summary(orc.placement_cost(idx, X, C, H, src, policy="local_first"))
+        rr = orc.cost_summary(orc.placement_cost(idx, X, C, H, src))
+        assert lf["cross_rank_bytes"] <= rr["cross_rank_bytes"]
+        cl = orc.placement_cost(idx, X, C, H, src, policy="local_first")
+        assert cl["rank_load"].sum() == T * K and np.array_equal(cl["workload"], orc.placement_cost(idx, X, C, H, src)["workload"])
+
+
+def test_layer_output_does_not_depend_on_the_replica_policy():
+    wl = synth.make_workload("c1_tiny")
+    s, w = wl.shape, wl.weights
+    idx, _, ww = orc.route(wl.logits, s.K)
+    X = _random_placement(_rng(150), s.E, s.R, 4, 6)
+    ys = []
+    for policy in ("round_robin", "local_first"):
+        d = orc.dispatch(idx, X, 4, wl.x, policy=policy)
+        yp = orc.expert_ffn(d["xp"], d["seg_offsets"], d["slot_expert"], w.w_gate, w.w_up, w.w_down)
+        ys.append(orc.combine(yp, d["inv_row"], ww))
+    assert np.allclose(ys[0], ys[1], rtol=1e-12, atol=1e-15)      # same rows, other segment shapes: fp64 rounding order only
+
+
+def test_dedup_volume_properties():
+    rng = _rng(140)
+    T, E, R, C = 83, 10, 4, 4
+    X = _random_placement(rng, E, R, C, 5)
+    src = rng.integers(0, R, size=T).astype(np.int32)
+    for K in (1, 3):
+        idx, _, _ = orc.route(rng.normal(size=(T, E)).astype(np.float32), K)
+        for policy in ("round_robin", "local_first"):
+            dest = orc.dispatch(idx, X, C, policy=policy, src=src)["dest_rank"]
+            U = orc.dedup_dispatch_tokens(dest, src, R)
+            D = orc.placement_cost(idx, X, C, 64, src, policy=policy)["dispatch_tokens"]
+            assert np.all(U <= D)
+            if K == 1:
+                assert np.array_equal(U, D)
+            # distinct (token, destination) pairs, counted with a library routine
+            pairs = np.unique(np.stack([np.repeat(np.arange(T), K), dest.reshape(-1)], axis=1), axis=0)
+            want = np.zeros((R, R), dtype=np.int64)
+            np.add.at(want, (src[pairs[:, 0]], pairs[:, 1]), 1)
+            assert np.array_equal(U, want)
+            assert np.all(U.sum(axis=1) >= np.bincount(src, minlength=R))      # every token goes somewhere
+    # all experts on one rank: every token is sent there exactly once whatever K
+    X1 = np.zeros((E, R), dtype=np.uint8)
+    X1[:, 2] = 1
+    idx, _, _ = orc.route(rng.normal(size=(T, E)).astype(np.float32), 3)
+    U = orc.dedup_dispatch_tokens(orc.dispatch(idx, X1, E)["dest_rank"], src, R)
+    assert np.array_equal(U[:, 2], np.bincount(src, minlength=R)) and U.sum() == T
