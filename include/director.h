@@ -85,7 +85,8 @@ int director_route(director_ctx* ctx, int32_t T, const float* logits,
 
 /* (a2) Dispatch (Section II-B: tokens are packaged and sent to the ranks hosting their experts;
  * here an on-device permutation, the bytes that would cross ranks are counted by
- * director_placement_cost).  The n-th assignment of expert e in ascending token order goes to
+ * director_placement_cost).  Under the default replica policy (see director_set_replica_policy) the n-th
+ * assignment of expert e in ascending token order goes to
  * replica n mod r_e of e (replicas ordered by rank) and becomes row n div r_e of that replica's
  * segment; segments lie in slot order.
  * x: dev bf16 [T,H].  topk_idx: dev int32 [T,K].
@@ -96,6 +97,32 @@ int director_route(director_ctx* ctx, int32_t T, const float* logits,
 int director_dispatch(director_ctx* ctx, int32_t T, const void* x, const int32_t* topk_idx,
                       void* xp, int32_t* row_token, int32_t* inv_row, int32_t* dest_rank,
                       int32_t* seg_offsets, void* stream);
+
+/* Which replica of a replicated expert an assignment uses.  The paper replicates hot experts to shrink the
+ * dispatch volume of Eq. 3 (Section III) without fixing this choice; both rules below are this library's.
+ *   ROUND_ROBIN (default)  the n-th assignment of expert e (ascending token id) uses replica n mod r_e.
+ *   LOCAL_FIRST            an assignment whose token lives on a rank hosting e stays there; the others are
+ *                          numbered m = 0,1,... in ascending token id and use replica m mod r_e.
+ * In both, a segment holds its assignments in ascending token id.  The policy applies to director_dispatch,
+ * director_dispatch_src, director_placement_cost, director_placement_cost_batch and the host entry points. */
+enum { DIRECTOR_REPLICA_ROUND_ROBIN = 0, DIRECTOR_REPLICA_LOCAL_FIRST = 1 };
+int director_set_replica_policy(director_ctx* ctx, int32_t policy);
+
+/* director_dispatch with an explicit home rank per token.  token_src_rank: dev int32 [T] with values in [0,R),
+ * or NULL for the block partition src(t) = floor(t*R/T) that director_dispatch uses.  Only LOCAL_FIRST looks at
+ * it; a value out of range sets DIRECTOR_ERR_BAD_INDEX in the device status and the token is treated as having
+ * no home (all its assignments travel). */
+int director_dispatch_src(director_ctx* ctx, int32_t T, const void* x, const int32_t* topk_idx,
+                          const int32_t* token_src_rank, void* xp, int32_t* row_token, int32_t* inv_row,
+                          int32_t* dest_rank, int32_t* seg_offsets, void* stream);
+
+/* De-duplicated dispatch volume (a variant of Eq. 3's count): dedup_tokens[j*R+k] = number of tokens on rank j with
+ * at least one assignment executed on rank k, i.e. what the first all-to-all of Section II-B moves when a token
+ * whose several experts share a rank is sent there once.  dest_rank: dev int32 [T,K] as written by
+ * director_dispatch (entries < 0 are skipped).  token_src_rank: dev int32 [T] or NULL (block partition).
+ * dedup_tokens: dev int64 [R,R], overwritten. */
+int director_dedup_dispatch_tokens(director_ctx* ctx, int32_t T, const int32_t* dest_rank,
+                                   const int32_t* token_src_rank, int64_t* dedup_tokens, void* stream);
 
 /* (a3) Expert FFNs (Section II-A: each expert is an FFN sub-network), SwiGLU, bf16 operands,
  * fp32 accumulation on the tensor cores:  for every row i of the segment of slot g (expert e)

@@ -24,8 +24,11 @@ EXPORTED = (
     "director_last_status", "director_launch_count", "director_set_profiling", "director_kernel_time",
     "director_status_string", "director_dispatch_index_static", "director_layer_submit_host",
     "director_layer_wait_host", "director_set_ffn_variant", "director_placement_cost_batch",
-    "director_expert_ffn_gather",
+    "director_expert_ffn_gather", "director_set_replica_policy", "director_dispatch_src",
+    "director_dedup_dispatch_tokens",
 )
+
+REPLICA_ROUND_ROBIN, REPLICA_LOCAL_FIRST = 0, 1
 
 
 class DirectorShape(ctypes.Structure):
@@ -69,6 +72,9 @@ def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.director_launch_count.restype = c_int64
     lib.director_set_profiling.argtypes = [vp, c_int32]
     lib.director_set_ffn_variant.argtypes = [vp, c_int32]
+    lib.director_set_replica_policy.argtypes = [vp, c_int32]
+    lib.director_dispatch_src.argtypes = [vp, c_int32] + [vp] * 9
+    lib.director_dedup_dispatch_tokens.argtypes = [vp, c_int32, vp, vp, vp, vp]
     lib.director_kernel_time.argtypes = [vp, c_char_p, POINTER(c_int64)]
     lib.director_kernel_time.restype = c_double
     lib.director_status_string.argtypes = [c_int]
@@ -137,6 +143,19 @@ class Director:
         _check(self.lib.director_dispatch(self._ctx, T, _ptr(x), _ptr(topk_idx), _ptr(xp), _ptr(row_token),
                                           _ptr(inv_row), _ptr(dest_rank), _ptr(seg_offsets), _stream()),
                "director_dispatch")
+
+    def dispatch_src(self, T, x, topk_idx, token_src_rank, xp, row_token, inv_row, dest_rank, seg_offsets):
+        _check(self.lib.director_dispatch_src(self._ctx, T, _ptr(x), _ptr(topk_idx), _ptr(token_src_rank), _ptr(xp),
+                                              _ptr(row_token), _ptr(inv_row), _ptr(dest_rank), _ptr(seg_offsets),
+                                              _stream()), "director_dispatch_src")
+
+    def set_replica_policy(self, policy: int):
+        _check(self.lib.director_set_replica_policy(self._ctx, policy), "director_set_replica_policy")
+
+    def dedup_dispatch_tokens(self, T, dest_rank, token_src_rank, dedup_tokens):
+        _check(self.lib.director_dedup_dispatch_tokens(self._ctx, T, _ptr(dest_rank), _ptr(token_src_rank),
+                                                       _ptr(dedup_tokens), _stream()),
+               "director_dedup_dispatch_tokens")
 
     def expert_ffn(self, T, xp, seg_offsets, w_gate, w_up, w_down, yp, x=None, ws_gate=None, ws_up=None,
                    ws_down=None, y_shared=None):

@@ -32,6 +32,7 @@ bool shape_supported(const director_shape& s) {
 
 void free_all(director_ctx* c) {
     void* ptrs[] = {c->d_rep_start, c->d_rep_slot, c->d_slot_expert, c->d_tile_counts, c->d_seg_offsets, c->d_ticket,
+                    c->d_host_mask, c->d_tile_rep,
                     c->d_status, c->d_hidden, c->d_hidden_shared, c->d_one_seg, c->d_sched,
                     c->d_zero_expert, c->e_logits2[0], c->e_logits2[1], c->e_x2[0], c->e_x2[1], c->e_topk_idx,
                     c->e_topk_w, c->e_xp, c->e_yp, c->e_y2[0], c->e_y2[1], c->e_y_shared, c->e_row_token, c->e_inv_row,
@@ -96,6 +97,7 @@ int director_create(const director_shape* shape, director_ctx** out) {
     bool ok = dev_alloc(&c->d_rep_start, s.E + 1) && dev_alloc(&c->d_rep_slot, (size_t)s.E * s.R) &&
               dev_alloc(&c->d_slot_expert, c->G) && dev_alloc(&c->d_tile_counts, (size_t)c->n_tiles_max * s.E) &&
               dev_alloc(&c->d_seg_offsets, c->G + 1) && dev_alloc(&c->d_ticket, 1) && dev_alloc(&c->d_status, 1) &&
+              dev_alloc(&c->d_host_mask, s.E) && dev_alloc(&c->d_tile_rep, (size_t)c->n_tiles_max * c->G) &&
               dev_alloc(&c->d_one_seg, 2) && dev_alloc(&c->d_sched, 4) &&
               dev_alloc(&c->d_zero_expert, 1) &&
               dev_alloc(reinterpret_cast<uint16_t**>(&c->d_hidden), A * s.F) &&
@@ -127,7 +129,7 @@ int director_create(const director_shape* shape, director_ctx** out) {
                                               &qres) == cudaSuccess &&
              qres == cudaDriverEntryPointSuccess && c->encode_tiled != nullptr;
     }
-    if (ok) ok = ffn_init(c) == DIRECTOR_OK;
+    if (ok) ok = ffn_init(c) == DIRECTOR_OK && dispatch_local_init(c) == DIRECTOR_OK;
     if (ok) {
         ok = cudaStreamCreateWithFlags(&c->h2d_stream, cudaStreamNonBlocking) == cudaSuccess &&
              cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking) == cudaSuccess;
@@ -183,12 +185,18 @@ int director_set_placement(director_ctx* ctx, const uint8_t* X, void* stream) {
         if ((int32_t)rep_slot.size() == rep_start[e]) return DIRECTOR_ERR_PLACEMENT;
     }
     rep_start[E] = (int32_t)rep_slot.size();
+    std::vector<unsigned long long> host_mask(E, 0ull);
+    for (int e = 0; e < E; ++e)
+        for (int j = 0; j < R; ++j)
+            if (slot_of[(size_t)e * R + j] >= 0) host_mask[e] |= 1ull << j;
     cudaStream_t st = as_stream(stream);
     // pageable sources: the runtime stages them before returning, so the vectors may die here
     if (cudaMemcpyAsync(ctx->d_rep_start, rep_start.data(), rep_start.size() * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
         cudaMemcpyAsync(ctx->d_rep_slot, rep_slot.data(), rep_slot.size() * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(ctx->d_slot_expert, slot_expert.data(), slot_expert.size() * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        cudaMemcpyAsync(ctx->d_slot_expert, slot_expert.data(), slot_expert.size() * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(ctx->d_host_mask, host_mask.data(), host_mask.size() * 8, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return DIRECTOR_ERR_CUDA;
+    ctx->n_replicas = rep_start[E];
     ctx->h_slot_expert = slot_expert;
     ctx->placement_set = true;
     return DIRECTOR_OK;
@@ -217,7 +225,44 @@ int director_dispatch(director_ctx* ctx, int32_t T, const void* x, const int32_t
     REQUIRE_PTR(inv_row);
     REQUIRE_PTR(dest_rank);
     REQUIRE_PTR(seg_offsets);
-    return launch_dispatch(ctx, T, x, topk_idx, xp, row_token, inv_row, dest_rank, seg_offsets, as_stream(stream));
+    return launch_dispatch(ctx, T, x, topk_idx, nullptr, xp, row_token, inv_row, dest_rank, seg_offsets, as_stream(stream));
+}
+
+int director_dispatch_src(director_ctx* ctx, int32_t T, const void* x, const int32_t* topk_idx,
+                          const int32_t* token_src_rank, void* xp, int32_t* row_token, int32_t* inv_row,
+                          int32_t* dest_rank, int32_t* seg_offsets, void* stream) {
+    REQUIRE_CTX(ctx);
+    REQUIRE_T(ctx, T);
+    REQUIRE_PLACEMENT(ctx);
+    REQUIRE_PTR(topk_idx);
+    if (token_src_rank != nullptr && (reinterpret_cast<uintptr_t>(token_src_rank) & 3u)) return DIRECTOR_ERR_INVALID_ARG;
+    if (xp != nullptr) {
+        REQUIRE_PTR(x);
+        REQUIRE_PTR(xp);
+    }
+    REQUIRE_PTR(row_token);
+    REQUIRE_PTR(inv_row);
+    REQUIRE_PTR(dest_rank);
+    REQUIRE_PTR(seg_offsets);
+    return launch_dispatch(ctx, T, x, topk_idx, token_src_rank, xp, row_token, inv_row, dest_rank, seg_offsets,
+                           as_stream(stream));
+}
+
+int director_set_replica_policy(director_ctx* ctx, int32_t policy) {
+    REQUIRE_CTX(ctx);
+    if (policy != DIRECTOR_REPLICA_ROUND_ROBIN && policy != DIRECTOR_REPLICA_LOCAL_FIRST) return DIRECTOR_ERR_INVALID_ARG;
+    ctx->replica_policy = policy;
+    return DIRECTOR_OK;
+}
+
+int director_dedup_dispatch_tokens(director_ctx* ctx, int32_t T, const int32_t* dest_rank,
+                                   const int32_t* token_src_rank, int64_t* dedup_tokens, void* stream) {
+    REQUIRE_CTX(ctx);
+    REQUIRE_T(ctx, T);
+    if (dest_rank == nullptr || (reinterpret_cast<uintptr_t>(dest_rank) & 3u)) return DIRECTOR_ERR_INVALID_ARG;
+    if (token_src_rank != nullptr && (reinterpret_cast<uintptr_t>(token_src_rank) & 3u)) return DIRECTOR_ERR_INVALID_ARG;
+    if (dedup_tokens == nullptr || (reinterpret_cast<uintptr_t>(dedup_tokens) & 7u)) return DIRECTOR_ERR_INVALID_ARG;
+    return launch_dedup_volume(ctx, T, dest_rank, token_src_rank, dedup_tokens, as_stream(stream));
 }
 
 int director_expert_ffn(director_ctx* ctx, int32_t T, const void* xp, const int32_t* seg_offsets, const void* w_gate,
@@ -351,7 +396,7 @@ int director_layer_submit_host(director_ctx* ctx, int32_t T, const float* logits
     const bool fused = false;
     int rc = launch_route(ctx, T, d_logits, ctx->e_topk_idx, ctx->e_topk_w, st);
     if (rc == DIRECTOR_OK)
-        rc = launch_dispatch(ctx, T, d_x, ctx->e_topk_idx, fused ? nullptr : ctx->e_xp, ctx->e_row_token, ctx->e_inv_row,
+        rc = launch_dispatch(ctx, T, d_x, ctx->e_topk_idx, nullptr, fused ? nullptr : ctx->e_xp, ctx->e_row_token, ctx->e_inv_row,
                              ctx->e_dest_rank, ctx->d_seg_offsets, st);
     if (rc == DIRECTOR_OK)
         rc = launch_expert_ffn(ctx, T, ctx->e_xp, fused ? ctx->e_row_token : nullptr, ctx->d_seg_offsets, w_gate, w_up,

@@ -39,9 +39,13 @@ struct director_ctx {
     int32_t* d_rep_slot = nullptr;     // [E*R] slot id of each replica, replicas by ascending rank
     int32_t* d_slot_expert = nullptr;  // [G] expert of each slot or -1
     std::vector<int32_t> h_slot_expert;
+    unsigned long long* d_host_mask = nullptr;   // [E] bit j set iff rank j hosts the expert
+    int n_replicas = 0;                // rep_start[E]: hosted (expert, rank) pairs of the current placement
+    int replica_policy = 0;            // DIRECTOR_REPLICA_*: which replica an assignment uses
 
     // dispatch / cost workspace
     int32_t* d_tile_counts = nullptr;   // [n_tiles_max, E] per-tile expert counts -> exclusive prefix
+    int32_t* d_tile_rep = nullptr;      // [n_tiles_max, G] per-tile replica counts (locality-first dispatch)
     int32_t* d_seg_offsets = nullptr;   // [G+1] internal copy (placement-cost path, host forward)
     unsigned int* d_ticket = nullptr;   // last-CTA-done counter, self-resetting
     int32_t* d_status = nullptr;        // sticky device status word
@@ -119,8 +123,17 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // Stage launchers implemented in the individual translation units.  All validate nothing:
 // the extern "C" wrappers in director_api.cu check arguments first.
 int launch_route(director_ctx*, int T, const float* logits, int32_t* topk_idx, float* topk_w, cudaStream_t);
-int launch_dispatch(director_ctx*, int T, const void* x, const int32_t* topk_idx, void* xp, int32_t* row_token,
-                    int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, cudaStream_t);
+int launch_dispatch(director_ctx*, int T, const void* x, const int32_t* topk_idx, const int32_t* src_rank, void* xp,
+                    int32_t* row_token, int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, cudaStream_t);
+int launch_scatter_rows(director_ctx*, int T, const void* x, const int32_t* inv_row, void* xp, cudaStream_t);
+int dispatch_local_init(director_ctx*);
+int launch_dispatch_local_first(director_ctx*, int T, const void* x, const int32_t* topk_idx, const int32_t* src_rank,
+                                void* xp, int32_t* row_token, int32_t* inv_row, int32_t* dest_rank,
+                                int32_t* seg_offsets, cudaStream_t);
+int launch_cost_local_first(director_ctx*, int T, const int32_t* topk_idx, const int32_t* src_rank, int64_t* workload,
+                            int64_t* rank_load, int64_t* dispatch_tokens, uint64_t* dispatch_bytes, cudaStream_t);
+int launch_dedup_volume(director_ctx*, int T, const int32_t* dest_rank, const int32_t* src_rank, int64_t* dedup_tokens,
+                        cudaStream_t);
 int launch_cost(director_ctx*, int T, const int32_t* topk_idx, const int32_t* src_rank, int64_t* workload,
                 int64_t* rank_load, int64_t* dispatch_tokens, uint64_t* dispatch_bytes, cudaStream_t);
 int launch_cost_batch(director_ctx*, const int64_t* workload, int n, const uint8_t* X, int64_t* rank_load,

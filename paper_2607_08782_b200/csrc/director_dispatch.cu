@@ -246,7 +246,8 @@ cost_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ sr
 // contiguous range [a, b) of n.  Round-robin over r replicas gives replica q exactly
 //     f(b) - f(a),  f(x) = max(0, ceil((x - q) / r))
 // of them.  The whole cost therefore follows from the workload matrix W alone: one histogram kernel and one
-// warp-per-expert kernel, no per-assignment ranks.
+// warp-per-expert kernel, no per-assignment ranks.  Under the locality-first rule the ranks that host e keep their
+// own W[j][e] assignments and the same closed form runs over the remaining (travelling) ranks' counts.
 
 constexpr int kHistSmemInts = 4096;
 
@@ -293,16 +294,27 @@ constexpr int kCostWarps = 8;
 __global__ void __launch_bounds__(kCostWarps * 32)
 cost_from_workload_kernel(const unsigned long long* __restrict__ workload, int E, int R, int C_max,
                           const int32_t* __restrict__ rep_start, const int32_t* __restrict__ rep_slot,
+                          const unsigned long long* __restrict__ host_mask /* non-null: locality-first rule */,
                           unsigned long long* __restrict__ rank_load, unsigned long long* __restrict__ dispatch_tokens,
                           unsigned long long* __restrict__ dispatch_bytes, unsigned long long bytes_per_token) {
     const int e = blockIdx.x * kCostWarps + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (e >= E) return;
     const int r0 = __ldg(rep_start + e);
     const uint32_t r = (uint32_t)(__ldg(rep_start + e + 1) - r0);
+    const unsigned long long hm = host_mask ? __ldg(host_mask + e) : 0ull;
     uint32_t carry = 0;                                        // assignments of e sent by ranks before this chunk
     for (int j0 = 0; j0 < R; j0 += 32) {
         const int j = j0 + lane;
-        const uint32_t w = j < R ? (uint32_t)workload[(size_t)j * E + e] : 0u;   // counts fit 32 bits: T*K < 2^31
+        uint32_t w = j < R ? (uint32_t)workload[(size_t)j * E + e] : 0u;   // counts fit 32 bits: T*K < 2^31
+        if (j < R && ((hm >> j) & 1ull)) {
+            // locality first: a rank that hosts e serves its own tokens; only the others' assignments are numbered
+            if (w) {
+                atomicAdd(dispatch_tokens + (size_t)j * R + j, (unsigned long long)w);
+                atomicAdd(dispatch_bytes + (size_t)j * R + j, (unsigned long long)w * bytes_per_token);
+                atomicAdd(rank_load + j, (unsigned long long)w);
+            }
+            w = 0u;
+        }
         uint32_t incl = w;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -335,7 +347,8 @@ cost_from_workload_kernel(const unsigned long long* __restrict__ workload, int E
 
 __global__ void __launch_bounds__(kCostWarps * 32)
 cost_batch_kernel(const unsigned long long* __restrict__ workload, int E, int R, const uint8_t* __restrict__ X,
-                  unsigned long long* __restrict__ rank_load, unsigned long long* __restrict__ dispatch_tokens) {
+                  int local_first, unsigned long long* __restrict__ rank_load,
+                  unsigned long long* __restrict__ dispatch_tokens) {
     const int e = blockIdx.x * kCostWarps + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     const int c = blockIdx.y;
     if (e >= E) return;
@@ -350,7 +363,14 @@ cost_batch_kernel(const unsigned long long* __restrict__ workload, int E, int R,
     uint32_t carry = 0;
     for (int j0 = 0; j0 < R; j0 += 32) {
         const int j = j0 + lane;
-        const uint32_t w = j < R ? (uint32_t)workload[(size_t)j * E + e] : 0u;
+        uint32_t w = j < R ? (uint32_t)workload[(size_t)j * E + e] : 0u;
+        if (local_first && (((j0 == 0 ? m0 : m1) >> lane) & 1u)) {     // this rank hosts e: its tokens stay
+            if (w) {
+                atomicAdd(disp_c + (size_t)j * R + j, (unsigned long long)w);
+                atomicAdd(load_c + j, (unsigned long long)w);
+            }
+            w = 0u;
+        }
         uint32_t incl = w;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -430,8 +450,23 @@ int launch_count_scan(director_ctx* ctx, const char* name, int T, const int32_t*
 
 }  // namespace
 
-int launch_dispatch(director_ctx* ctx, int T, const void* x, const int32_t* topk_idx, void* xp, int32_t* row_token,
-                    int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, cudaStream_t st) {
+int launch_scatter_rows(director_ctx* ctx, int T, const void* x, const int32_t* inv_row, void* xp, cudaStream_t st) {
+    const director_shape& s = ctx->shape;
+    const int row_vec = s.H * 2 / 16;
+    const int slices = (s.H * 2 + kSliceBytes - 1) / kSliceBytes;
+    const long long items = (long long)T * slices;
+    const unsigned grid = (unsigned)((items + kScatterWarps - 1) / kScatterWarps);
+    LaunchScope scope(ctx, st, "dispatch_scatter_rows_kernel");
+    scatter_rows_kernel<<<grid, kScatterWarps * 32, 0, st>>>(static_cast<const uint4*>(x), inv_row,
+                                                             static_cast<uint4*>(xp), T, s.K, row_vec, slices);
+    return cuda_status(cudaGetLastError());
+}
+
+int launch_dispatch(director_ctx* ctx, int T, const void* x, const int32_t* topk_idx, const int32_t* src_rank, void* xp,
+                    int32_t* row_token, int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, cudaStream_t st) {
+    if (ctx->replica_policy == DIRECTOR_REPLICA_LOCAL_FIRST)
+        return launch_dispatch_local_first(ctx, T, x, topk_idx, src_rank, xp, row_token, inv_row, dest_rank,
+                                           seg_offsets, st);
     const director_shape& s = ctx->shape;
     const int n_tiles = (T + kTokenTile - 1) / kTokenTile;
     int rc = launch_count_scan(ctx, "dispatch_count_scan_kernel", T, topk_idx, seg_offsets, ctx->d_seg_offsets, st);
@@ -444,16 +479,8 @@ int launch_dispatch(director_ctx* ctx, int T, const void* x, const int32_t* topk
         rc = cuda_status(cudaGetLastError());
         if (rc != DIRECTOR_OK) return rc;
     }
-    if (xp != nullptr) {      // xp == nullptr: indices only (the expert FFN then gathers its rows from x itself)
-        const int row_vec = s.H * 2 / 16;
-        const int slices = (s.H * 2 + kSliceBytes - 1) / kSliceBytes;
-        const long long items = (long long)T * slices;
-        const unsigned grid = (unsigned)((items + kScatterWarps - 1) / kScatterWarps);
-        LaunchScope scope(ctx, st, "dispatch_scatter_rows_kernel");
-        scatter_rows_kernel<<<grid, kScatterWarps * 32, 0, st>>>(static_cast<const uint4*>(x), inv_row,
-                                                                 static_cast<uint4*>(xp), T, s.K, row_vec, slices);
-        rc = cuda_status(cudaGetLastError());
-    }
+    // xp == nullptr: indices only (the expert FFN then gathers its rows from x itself)
+    if (xp != nullptr) rc = launch_scatter_rows(ctx, T, x, inv_row, xp, st);
     return rc;
 }
 
@@ -467,6 +494,7 @@ int launch_cost_batch(director_ctx* ctx, const int64_t* workload, int n, const u
         LaunchScope scope(ctx, st, "cost_batch_kernel");
         cost_batch_kernel<<<dim3((s.E + kCostWarps - 1) / kCostWarps, n), kCostWarps * 32, 0, st>>>(
             reinterpret_cast<const unsigned long long*>(workload), s.E, s.R, X,
+            ctx->replica_policy == DIRECTOR_REPLICA_LOCAL_FIRST ? 1 : 0,
             reinterpret_cast<unsigned long long*>(rank_load), reinterpret_cast<unsigned long long*>(dispatch_tokens));
         if (cudaGetLastError() != cudaSuccess) return DIRECTOR_ERR_CUDA;
     }
@@ -481,6 +509,9 @@ int launch_cost(director_ctx* ctx, int T, const int32_t* topk_idx, const int32_t
                 int64_t* rank_load, int64_t* dispatch_tokens, uint64_t* dispatch_bytes, cudaStream_t st) {
     const director_shape& s = ctx->shape;
     const int n_tiles = (T + kTokenTile - 1) / kTokenTile;
+    const bool local_first = ctx->replica_policy == DIRECTOR_REPLICA_LOCAL_FIRST;
+    if (local_first && src_rank != nullptr)
+        return launch_cost_local_first(ctx, T, topk_idx, src_rank, workload, rank_load, dispatch_tokens, dispatch_bytes, st);
     cudaError_t e;
     if ((e = cudaMemsetAsync(workload, 0, sizeof(int64_t) * s.R * s.E, st)) != cudaSuccess) return cuda_status(e);
     if (src_rank == nullptr) {
@@ -497,6 +528,7 @@ int launch_cost(director_ctx* ctx, int T, const int32_t* topk_idx, const int32_t
         LaunchScope scope(ctx, st, "cost_from_workload_kernel");
         cost_from_workload_kernel<<<(s.E + kCostWarps - 1) / kCostWarps, kCostWarps * 32, 0, st>>>(reinterpret_cast<const unsigned long long*>(workload), s.E, s.R,
                                                      s.C_max, ctx->d_rep_start, ctx->d_rep_slot,
+                                                     local_first ? ctx->d_host_mask : nullptr,
                                                      reinterpret_cast<unsigned long long*>(rank_load),
                                                      reinterpret_cast<unsigned long long*>(dispatch_tokens),
                                                      reinterpret_cast<unsigned long long*>(dispatch_bytes),

@@ -58,9 +58,25 @@ class MoELayer:
     def route(self, T, logits):
         self.d.route(T, logits, self.topk_idx, self.topk_w)
 
-    def dispatch(self, T, x, indices_only=False):
-        self.d.dispatch(T, x, self.topk_idx, None if indices_only else self.xp, self.row_token, self.inv_row,
-                        self.dest_rank, self.seg_offsets)
+    def set_replica_policy(self, policy: int):
+        """0: round-robin over an expert's replicas; 1: locality first (see director_set_replica_policy)."""
+        self.d.set_replica_policy(policy)
+
+    def dispatch(self, T, x, indices_only=False, token_src_rank=None):
+        xp = None if indices_only else self.xp
+        if token_src_rank is None:
+            self.d.dispatch(T, x, self.topk_idx, xp, self.row_token, self.inv_row, self.dest_rank, self.seg_offsets)
+        else:
+            self.d.dispatch_src(T, x, self.topk_idx, token_src_rank, xp, self.row_token, self.inv_row,
+                                self.dest_rank, self.seg_offsets)
+
+    def dedup_dispatch_tokens(self, T, token_src_rank=None):
+        """[R,R] int64: tokens each rank sends to each rank when a token goes to a rank once (after dispatch)."""
+        R = self.dims["R"]
+        if getattr(self, "dedup_tokens", None) is None:
+            self.dedup_tokens = torch.empty((R, R), dtype=torch.int64, device=self.topk_idx.device)
+        self.d.dedup_dispatch_tokens(T, self.dest_rank, token_src_rank, self.dedup_tokens)
+        return self.dedup_tokens
 
     def expert_ffn_gather(self, T, x):
         """The routed experts read their rows from x through row_token (no permuted copy)."""

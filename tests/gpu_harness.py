@@ -28,6 +28,7 @@ class GpuRun:
     dispatch_bytes: np.ndarray
     status: int
     launches: int
+    dedup_tokens: np.ndarray | None = None
 
 
 class GpuCase:
@@ -52,19 +53,24 @@ class GpuCase:
             sd = bf16_bits_to_tensor(synth.concat_shared_down(w.ws_down), dev)
         self.layer = MoELayer(T_max or s.T, s.H, s.F, s.E, s.K, s.S, s.R, self.C_max, wg, wu, wd, sg, su, sd, dev)
 
-    def run(self, X, T=None, src=None, stages="all") -> GpuRun:
+    def run(self, X, T=None, src=None, stages="all", policy=0) -> GpuRun:
         from paper_2607_08782_b200.layer import tensor_to_bf16_bits
         torch, L, s = self.torch, self.layer, self.shape
         T = T or s.T
         L.set_placement(X)
         n0 = L.d.launch_count()
         src_t = None if src is None else torch.from_numpy(np.ascontiguousarray(src, dtype=np.int32)).cuda()
-        L.route(T, self.logits)
-        L.dispatch(T, self.x)
-        if stages == "all":
-            L.expert_ffn(T, self.x)
-            L.combine(T)
-        L.placement_cost(T, src_t)
+        L.set_replica_policy(policy)
+        try:
+            L.route(T, self.logits)
+            L.dispatch(T, self.x, token_src_rank=src_t)       # the home ranks matter to the locality-first rule only
+            if stages == "all":
+                L.expert_ffn(T, self.x)
+                L.combine(T)
+            L.placement_cost(T, src_t)
+            dedup = L.dedup_dispatch_tokens(T, src_t).cpu().numpy()
+        finally:
+            L.set_replica_policy(0)
         torch.cuda.synchronize()
         status = L.d.last_status()
         A = T * s.K
@@ -78,7 +84,7 @@ class GpuCase:
             workload=L.workload.cpu().numpy(), rank_load=L.rank_load.cpu().numpy(),
             dispatch_tokens=L.dispatch_tokens.cpu().numpy(),
             dispatch_bytes=L.dispatch_bytes.cpu().numpy().view(np.uint64),
-            status=status, launches=L.d.launch_count() - n0)
+            status=status, launches=L.d.launch_count() - n0, dedup_tokens=dedup)
 
 
 def rel_l2(a: np.ndarray, b: np.ndarray) -> float:
