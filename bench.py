@@ -186,6 +186,8 @@ def build_layer(args, device):
     layer.set_placement(X)
     if args.ffn_variant is not None:
         layer.set_ffn_variant(args.ffn_variant)
+    if args.replica_policy == "local_first":
+        layer.set_replica_policy(1)
     return wl, layer, logits, x, X, pname
 
 
@@ -279,10 +281,12 @@ def run_reference(args):
 
 STAGE_KERNELS = {
     "route": ["route_topk_kernel"],
-    "dispatch": ["dispatch_count_scan_kernel", "dispatch_index_kernel", "dispatch_scatter_rows_kernel"],
+    "dispatch": ["dispatch_count_scan_kernel", "dispatch_index_kernel", "dispatch_scatter_rows_kernel",
+                 "dispatch_travel_count_scan_kernel", "dispatch_slot_count_scan_kernel", "dispatch_local_index_kernel"],
     "expert_ffn": ["grouped_gemm_swiglu_kernel", "grouped_gemm_down_kernel", "one_segment_kernel"],
     "combine": ["combine_kernel"],
-    "placement_cost": ["cost_workload_hist_kernel", "cost_from_workload_kernel", "cost_count_scan_kernel", "cost_kernel"],
+    "placement_cost": ["cost_workload_hist_kernel", "cost_from_workload_kernel", "cost_count_scan_kernel", "cost_kernel",
+                       "cost_travel_count_scan_kernel", "cost_local_kernel"],
 }
 
 
@@ -364,6 +368,8 @@ def main():
     ap.add_argument("--placement", default="auto", choices=["auto", "primary"])
     ap.add_argument("--ffn-variant", type=int, default=None, choices=[0, 1, 2],
                     help="expert-FFN tile scheme: 0 = one CTA per 128x256 tile, 1 = CTA pairs (256x256); default: library's")
+    ap.add_argument("--replica-policy", default="round_robin", choices=["round_robin", "local_first"],
+                    help="which replica of a replicated expert an assignment uses (the default is the headline setting)")
     ap.add_argument("--fused", action="store_true",
                     help="index-only dispatch + director_expert_ffn_gather (the GEMM gathers rows from x) instead of the "
                          "materialised permutation")
@@ -555,6 +561,7 @@ def main():
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": WORKLOAD_TEXT[args.config], "tokens": T, "placement": pname,
+                   "replica_policy": args.replica_policy,
                    "l2": "inputs larger than L2: every step streams the expert weights "
                          f"({3 * s.E * s.F * s.H * 2 / 1e9:.2f} GB) and activations through HBM",
                    "parallelism": "single GPU, logical ranks" if world == 1 else f"{world} independent replicas"},
