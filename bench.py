@@ -280,7 +280,7 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------------
 
 STAGE_KERNELS = {
-    "route": ["route_topk_kernel"],
+    "route": ["route_topk_kernel", "front_small_kernel"],   # the fused front end (T <= 256) is booked under route
     "dispatch": ["dispatch_count_scan_kernel", "dispatch_index_kernel", "dispatch_scatter_rows_kernel",
                  "dispatch_travel_count_scan_kernel", "dispatch_slot_count_scan_kernel", "dispatch_local_index_kernel"],
     "expert_ffn": ["grouped_gemm_swiglu_kernel", "grouped_gemm_down_kernel", "one_segment_kernel"],
@@ -357,6 +357,58 @@ def run_placement_search(args, device):
                    "lp_bound": res["lp_bound"]}}))
 
 
+def run_index_kernels(args, device):
+    """Extra measurement (not the headline): the routing and index kernels far above their launch latency.  At the
+    paper-shaped batch sizes these kernels move ~1-20 MB and finish in microseconds, so their bandwidth there says
+    little; here the same routing shape (E, K, R, C_max of --config) runs on 2^20 tokens (hidden size cut to 256:
+    neither kernel touches hidden states), logits tiled from the seeded generator."""
+    import numpy as np
+    import torch
+    from paper_2607_08782_b200 import placement, synth
+    from paper_2607_08782_b200.binding import Director
+    base = synth.shape_for(args.config, None)
+    T = args.tokens or (1 << 20)
+    s = base
+    block = torch.from_numpy(synth.make_logits(base)).to(device)
+    logits = block.repeat((T + base.T - 1) // base.T, 1)[:T].contiguous()
+    d = Director(T, 256, 128, s.E, s.K, 0, s.R, s.C_max)
+    d.set_placement(synth.placement_from_ranks(synth.primary_ranks(s), s.R))
+    A = T * s.K
+    i32 = dict(dtype=torch.int32, device=device)
+    idx, w = torch.empty((T, s.K), **i32), torch.empty((T, s.K), dtype=torch.float32, device=device)
+    row_token, inv_row, dest = torch.empty(A, **i32), torch.empty((T, s.K), **i32), torch.empty((T, s.K), **i32)
+    seg = torch.empty(s.R * s.C_max + 1, **i32)
+    peaks = measured_peaks()
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / args.steps
+
+    out = {}
+    ms = timed(lambda: d.route(T, logits, idx, w))
+    by = T * (4 * s.E + 8 * s.K)
+    out["route"] = {"ms": ms, "GB/s": by / ms / 1e6, "frac_of_peak": by / ms / 1e6 / peaks["hbm_gbs"]}
+    for policy, name in ((0, "dispatch_index_round_robin"), (1, "dispatch_index_local_first")):
+        d.set_replica_policy(policy)
+        ms = timed(lambda: d.dispatch(T, None, idx, None, row_token, inv_row, dest, seg))
+        by = T * 16 * s.K                                     # topk_idx read, inv_row / dest_rank / row_token written
+        out[name] = {"ms": ms, "GB/s": by / ms / 1e6, "frac_of_peak": by / ms / 1e6 / peaks["hbm_gbs"]}
+    d.set_replica_policy(0)
+    d.check_device_status()
+    print(json.dumps({"metric": "index_kernel_bandwidth", "unit": "GB/s", "n_gpus": 1, "steps": args.steps,
+                      "data": "synthetic", "peak": {"hbm_gbs": peaks["hbm_gbs"], "source": peaks["source"]},
+                      "config": {"workload": WORKLOAD_TEXT[args.config], "tokens": T, "E": s.E, "K": s.K, "R": s.R},
+                      "kernels": out}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -376,8 +428,9 @@ def main():
     ap.add_argument("--graph", action="store_true",
                     help="replay the device-resident step from a CUDA graph (decode-sized batches); no per-kernel timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--stage", default="layer", choices=["layer", "placement_search"],
-                    help="layer (default): the MoE layer step; placement_search: batched scoring of candidate placements")
+    ap.add_argument("--stage", default="layer", choices=["layer", "placement_search", "index_kernels"],
+                    help="layer (default): the MoE layer step; placement_search: batched scoring of candidate placements; "
+                         "index_kernels: routing and dispatch-index kernels on 2^20 tokens")
     ap.add_argument("--sample-clocks", nargs=2, metavar=("UUID", "PATH"), help=argparse.SUPPRESS)
     args = ap.parse_args()
     if args.sample_clocks:
@@ -402,6 +455,10 @@ def main():
 
     if args.stage == "placement_search":
         run_placement_search(args, device)
+        ranks.close()
+        return
+    if args.stage == "index_kernels":
+        run_index_kernels(args, device)
         ranks.close()
         return
     wl, layer, logits, x, X, pname = build_layer(args, device)

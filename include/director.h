@@ -98,6 +98,17 @@ int director_dispatch(director_ctx* ctx, int32_t T, const void* x, const int32_t
                       void* xp, int32_t* row_token, int32_t* inv_row, int32_t* dest_rank,
                       int32_t* seg_offsets, void* stream);
 
+/* (a1) + (a2) + (a5) in one call: the front end of the layer.  Same arguments, same results (bit for bit) as
+ * director_route, director_dispatch and director_placement_cost (token_src_rank = NULL) called in that order.
+ * For batches of at most 256 tokens under the ROUND_ROBIN replica policy - the decode steps of serving, where
+ * each of those stages moves a few KB - the gate, the counting sort and the histograms run in a single launch
+ * (plus the row copies if xp != NULL); larger batches run the separate kernels. */
+int director_route_dispatch_cost(director_ctx* ctx, int32_t T, const float* logits, const void* x,
+                                 int32_t* topk_idx, float* topk_w, void* xp, int32_t* row_token,
+                                 int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, int64_t* workload,
+                                 int64_t* rank_load, int64_t* dispatch_tokens, uint64_t* dispatch_bytes,
+                                 void* stream);
+
 /* Which replica of a replicated expert an assignment uses.  The paper replicates hot experts to shrink the
  * dispatch volume of Eq. 3 (Section III) without fixing this choice; both rules below are this library's.
  *   ROUND_ROBIN (default)  the n-th assignment of expert e (ascending token id) uses replica n mod r_e.

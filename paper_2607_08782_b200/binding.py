@@ -25,7 +25,7 @@ EXPORTED = (
     "director_status_string", "director_dispatch_index_static", "director_layer_submit_host",
     "director_layer_wait_host", "director_set_ffn_variant", "director_placement_cost_batch",
     "director_expert_ffn_gather", "director_set_replica_policy", "director_dispatch_src",
-    "director_dedup_dispatch_tokens",
+    "director_dedup_dispatch_tokens", "director_route_dispatch_cost",
 )
 
 REPLICA_ROUND_ROBIN, REPLICA_LOCAL_FIRST = 0, 1
@@ -73,6 +73,7 @@ def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.director_set_profiling.argtypes = [vp, c_int32]
     lib.director_set_ffn_variant.argtypes = [vp, c_int32]
     lib.director_set_replica_policy.argtypes = [vp, c_int32]
+    lib.director_route_dispatch_cost.argtypes = [vp, c_int32] + [vp] * 14
     lib.director_dispatch_src.argtypes = [vp, c_int32] + [vp] * 9
     lib.director_dedup_dispatch_tokens.argtypes = [vp, c_int32, vp, vp, vp, vp]
     lib.director_kernel_time.argtypes = [vp, c_char_p, POINTER(c_int64)]
@@ -143,6 +144,13 @@ class Director:
         _check(self.lib.director_dispatch(self._ctx, T, _ptr(x), _ptr(topk_idx), _ptr(xp), _ptr(row_token),
                                           _ptr(inv_row), _ptr(dest_rank), _ptr(seg_offsets), _stream()),
                "director_dispatch")
+
+    def route_dispatch_cost(self, T, logits, x, topk_idx, topk_w, xp, row_token, inv_row, dest_rank, seg_offsets,
+                            workload, rank_load, dispatch_tokens, dispatch_bytes):
+        _check(self.lib.director_route_dispatch_cost(
+            self._ctx, T, _ptr(logits), _ptr(x), _ptr(topk_idx), _ptr(topk_w), _ptr(xp), _ptr(row_token), _ptr(inv_row),
+            _ptr(dest_rank), _ptr(seg_offsets), _ptr(workload), _ptr(rank_load), _ptr(dispatch_tokens),
+            _ptr(dispatch_bytes), _stream()), "director_route_dispatch_cost")
 
     def dispatch_src(self, T, x, topk_idx, token_src_rank, xp, row_token, inv_row, dest_rank, seg_offsets):
         _check(self.lib.director_dispatch_src(self._ctx, T, _ptr(x), _ptr(topk_idx), _ptr(token_src_rank), _ptr(xp),

@@ -69,6 +69,24 @@ inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
         if (!(ctx)->placement_set) return DIRECTOR_ERR_PLACEMENT; \
     } while (0)
 
+// a1 + a2 + a5 on device buffers: one fused launch for decode-sized batches, the separate kernels otherwise
+int launch_front(director_ctx* ctx, int T, const float* logits, const void* x, int32_t* topk_idx, float* topk_w, void* xp,
+                 int32_t* row_token, int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, int64_t* workload,
+                 int64_t* rank_load, int64_t* dispatch_tokens, uint64_t* dispatch_bytes, cudaStream_t st) {
+    if (front_small_applies(ctx, T)) {
+        int rc = launch_front_small(ctx, T, logits, topk_idx, topk_w, row_token, inv_row, dest_rank, seg_offsets, workload,
+                                    rank_load, dispatch_tokens, dispatch_bytes, st);
+        if (rc == DIRECTOR_OK && xp != nullptr) rc = launch_scatter_rows(ctx, T, x, inv_row, xp, st);
+        return rc;
+    }
+    int rc = launch_route(ctx, T, logits, topk_idx, topk_w, st);
+    if (rc == DIRECTOR_OK)
+        rc = launch_dispatch(ctx, T, x, topk_idx, nullptr, xp, row_token, inv_row, dest_rank, seg_offsets, st);
+    if (rc == DIRECTOR_OK)
+        rc = launch_cost(ctx, T, topk_idx, nullptr, workload, rank_load, dispatch_tokens, dispatch_bytes, st);
+    return rc;
+}
+
 }  // namespace
 
 extern "C" {
@@ -248,6 +266,32 @@ int director_dispatch_src(director_ctx* ctx, int32_t T, const void* x, const int
                            as_stream(stream));
 }
 
+int director_route_dispatch_cost(director_ctx* ctx, int32_t T, const float* logits, const void* x, int32_t* topk_idx,
+                                 float* topk_w, void* xp, int32_t* row_token, int32_t* inv_row, int32_t* dest_rank,
+                                 int32_t* seg_offsets, int64_t* workload, int64_t* rank_load, int64_t* dispatch_tokens,
+                                 uint64_t* dispatch_bytes, void* stream) {
+    REQUIRE_CTX(ctx);
+    REQUIRE_T(ctx, T);
+    REQUIRE_PLACEMENT(ctx);
+    REQUIRE_PTR(logits);
+    REQUIRE_PTR(topk_idx);
+    REQUIRE_PTR(topk_w);
+    if (xp != nullptr) {
+        REQUIRE_PTR(x);
+        REQUIRE_PTR(xp);
+    }
+    REQUIRE_PTR(row_token);
+    REQUIRE_PTR(inv_row);
+    REQUIRE_PTR(dest_rank);
+    REQUIRE_PTR(seg_offsets);
+    if (!workload || !rank_load || !dispatch_tokens || !dispatch_bytes) return DIRECTOR_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(workload) | reinterpret_cast<uintptr_t>(rank_load) |
+         reinterpret_cast<uintptr_t>(dispatch_tokens) | reinterpret_cast<uintptr_t>(dispatch_bytes)) & 7u)
+        return DIRECTOR_ERR_INVALID_ARG;
+    return launch_front(ctx, T, logits, x, topk_idx, topk_w, xp, row_token, inv_row, dest_rank, seg_offsets, workload,
+                        rank_load, dispatch_tokens, dispatch_bytes, as_stream(stream));
+}
+
 int director_set_replica_policy(director_ctx* ctx, int32_t policy) {
     REQUIRE_CTX(ctx);
     if (policy != DIRECTOR_REPLICA_ROUND_ROBIN && policy != DIRECTOR_REPLICA_LOCAL_FIRST) return DIRECTOR_ERR_INVALID_ARG;
@@ -394,17 +438,15 @@ int director_layer_submit_host(director_ctx* ctx, int32_t T, const float* logits
     // the permuted rows are materialised once: the weight-stationary GEMM reads every token tile once per weight
     // block, so gathering inside it (director_expert_ffn_gather) repeats the gather 2F/256 times and measured slower
     const bool fused = false;
-    int rc = launch_route(ctx, T, d_logits, ctx->e_topk_idx, ctx->e_topk_w, st);
-    if (rc == DIRECTOR_OK)
-        rc = launch_dispatch(ctx, T, d_x, ctx->e_topk_idx, nullptr, fused ? nullptr : ctx->e_xp, ctx->e_row_token, ctx->e_inv_row,
-                             ctx->e_dest_rank, ctx->d_seg_offsets, st);
+    int rc = launch_front(ctx, T, d_logits, d_x, ctx->e_topk_idx, ctx->e_topk_w, fused ? nullptr : ctx->e_xp,
+                          ctx->e_row_token, ctx->e_inv_row, ctx->e_dest_rank, ctx->d_seg_offsets, c_w, c_load, c_tok,
+                          c_bytes, st);
     if (rc == DIRECTOR_OK)
         rc = launch_expert_ffn(ctx, T, ctx->e_xp, fused ? ctx->e_row_token : nullptr, ctx->d_seg_offsets, w_gate, w_up,
                                w_down, ctx->e_yp, (shared || fused) ? d_x : nullptr, ws_gate, ws_up, ws_down,
                                shared ? ctx->e_y_shared : nullptr, st);
     if (rc == DIRECTOR_OK)
         rc = launch_combine(ctx, T, ctx->e_yp, ctx->e_inv_row, ctx->e_topk_w, shared ? ctx->e_y_shared : nullptr, d_y, st);
-    if (rc == DIRECTOR_OK) rc = launch_cost(ctx, T, ctx->e_topk_idx, nullptr, c_w, c_load, c_tok, c_bytes, st);
     if (rc != DIRECTOR_OK) return rc;
     if (cudaEventRecord(ctx->ev_compute_done[slot], st) != cudaSuccess) return DIRECTOR_ERR_CUDA;
     // outputs

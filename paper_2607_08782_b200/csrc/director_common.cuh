@@ -123,6 +123,10 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // Stage launchers implemented in the individual translation units.  All validate nothing:
 // the extern "C" wrappers in director_api.cu check arguments first.
 int launch_route(director_ctx*, int T, const float* logits, int32_t* topk_idx, float* topk_w, cudaStream_t);
+bool front_small_applies(const director_ctx*, int T);
+int launch_front_small(director_ctx*, int T, const float* logits, int32_t* topk_idx, float* topk_w, int32_t* row_token,
+                       int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, int64_t* workload, int64_t* rank_load,
+                       int64_t* dispatch_tokens, uint64_t* dispatch_bytes, cudaStream_t);
 int launch_dispatch(director_ctx*, int T, const void* x, const int32_t* topk_idx, const int32_t* src_rank, void* xp,
                     int32_t* row_token, int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, cudaStream_t);
 int launch_scatter_rows(director_ctx*, int T, const void* x, const int32_t* inv_row, void* xp, cudaStream_t);

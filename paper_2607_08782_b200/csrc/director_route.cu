@@ -116,17 +116,13 @@ __device__ __noinline__ void exact_top8(const float* __restrict__ row, int E, rk
     }
 }
 
+// The gate of one token, computed by LPT adjacent lanes (sub = 0 .. LPT-1) that all call this together.
+// Returns true in the lane that holds the result (sub == 0): win_idx[0..K) / win_w[0..K) are the chosen experts
+// in descending logit order and their renormalised softmax weights.
 // VEC: the row can be read with 16-byte loads (E % 4 == 0; rows are then 16-byte aligned).
 template <bool VEC, int LPT>
-__global__ void __launch_bounds__(kRouteThreads)
-route_topk_kernel(const float* __restrict__ logits, int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
-                  int T, int E, int K, int32_t* __restrict__ status) {
-    const int tid = blockIdx.x * kRouteThreads + threadIdx.x;
-    const int t_raw = tid / LPT, sub = tid % LPT;
-    const bool live = t_raw < T;
-    const int t = live ? t_raw : T - 1;                // surplus lanes redo the last token (keeps shuffles full)
-    const float* row = logits + (size_t)t * E;
-
+__device__ __forceinline__ bool route_token(const float* __restrict__ row, int E, int K, int sub, bool live,
+                                            int32_t* __restrict__ status, int (&win_idx)[8], float (&win_w)[8]) {
     uint32_t top[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) top[i] = 0u;        // below every real key
@@ -173,7 +169,7 @@ route_topk_kernel(const float* __restrict__ logits, int32_t* __restrict__ topk_i
         max_abs = max(max_abs, __shfl_xor_sync(0xFFFFFFFFu, max_abs, step));
         merge_top8_32(top, other, rej);
     }
-    if (!live || sub != 0) return;
+    if (!live || sub != 0) return false;
     if (max_abs >= 0x7F800000u) director_set_status(status, DIRECTOR_ERR_NONFINITE);
 
     // the truncated keys decide exactly iff the K winners and the runner-up differ pairwise in the bits kept
@@ -184,7 +180,6 @@ route_topk_kernel(const float* __restrict__ logits, int32_t* __restrict__ topk_i
         if (s < K) exact = exact && ((top[s] >> 8) != (next >> 8));
     }
     uint32_t win_bits[8];
-    int win_idx[8];
     if (exact) {
 #pragma unroll
         for (int s = 0; s < 8; ++s) {
@@ -210,24 +205,187 @@ route_topk_kernel(const float* __restrict__ logits, int32_t* __restrict__ topk_i
         sum += p[s];
     }
     const float inv = 1.0f / sum;
-    int32_t* oi = topk_idx + (size_t)t * K;
-    float* ow = topk_w + (size_t)t * K;
+#pragma unroll
+    for (int s = 0; s < 8; ++s) win_w[s] = p[s] * inv;
+    return true;
+}
+
+__device__ __forceinline__ void store_gate(int32_t* __restrict__ oi, float* __restrict__ ow, int K, const int (&win_idx)[8],
+                                           const float (&win_w)[8]) {
     if (K == 8) {
         reinterpret_cast<int4*>(oi)[0] = make_int4(win_idx[0], win_idx[1], win_idx[2], win_idx[3]);
         reinterpret_cast<int4*>(oi)[1] = make_int4(win_idx[4], win_idx[5], win_idx[6], win_idx[7]);
-        reinterpret_cast<float4*>(ow)[0] = make_float4(p[0] * inv, p[1] * inv, p[2] * inv, p[3] * inv);
-        reinterpret_cast<float4*>(ow)[1] = make_float4(p[4] * inv, p[5] * inv, p[6] * inv, p[7] * inv);
+        reinterpret_cast<float4*>(ow)[0] = make_float4(win_w[0], win_w[1], win_w[2], win_w[3]);
+        reinterpret_cast<float4*>(ow)[1] = make_float4(win_w[4], win_w[5], win_w[6], win_w[7]);
     } else {
 #pragma unroll
         for (int s = 0; s < 8; ++s)
             if (s < K) {
                 oi[s] = win_idx[s];
-                ow[s] = p[s] * inv;
+                ow[s] = win_w[s];
             }
     }
 }
 
+template <bool VEC, int LPT>
+__global__ void __launch_bounds__(kRouteThreads)
+route_topk_kernel(const float* __restrict__ logits, int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
+                  int T, int E, int K, int32_t* __restrict__ status) {
+    const int tid = blockIdx.x * kRouteThreads + threadIdx.x;
+    const int t_raw = tid / LPT, sub = tid % LPT;
+    const bool live = t_raw < T;
+    const int t = live ? t_raw : T - 1;                // surplus lanes redo the last token (keeps shuffles full)
+    int win_idx[8];
+    float win_w[8];
+    if (route_token<VEC, LPT>(logits + (size_t)t * E, E, K, sub, live, status, win_idx, win_w))
+        store_gate(topk_idx + (size_t)t * K, topk_w + (size_t)t * K, K, win_idx, win_w);
+}
+
+// ---- decode-sized batches: gate, dispatch indices and placement cost in one CTA ----
+//
+// For T <= 256 the whole batch is one tile of the counting sort, every stage of the front end moves a few KB and
+// the five launches (route, count/scan, index, workload histogram, cost) cost more than their work.  One CTA of
+// 1024 threads does them back to back: four lanes per token compute the gate; then thread t < T is token t for the
+// counting sort (lane bitmasks per expert, popcounts; a single tile, so the tile prefix is zero), the slot lengths
+// are scanned by the block, and the histograms are accumulated per assignment in shared memory.  Same integer
+// arithmetic as the separate kernels, hence the same bits.  Round-robin replica rule, block partition of the
+// tokens over the source ranks.
+constexpr int kFrontThreads = 1024;
+constexpr int kFrontLpt = 4;
+constexpr int kFrontTokens = kFrontThreads / kFrontLpt;   // 256
+constexpr int kFrontWarps = kFrontTokens / 32;            // 8 warps of token threads
+
+template <bool VEC>
+__global__ void __launch_bounds__(kFrontThreads)
+front_small_kernel(const float* __restrict__ logits, int T, int E, int K, int R, int C_max, int G,
+                   const int32_t* __restrict__ rep_start, const int32_t* __restrict__ rep_slot,
+                   int32_t* __restrict__ topk_idx, float* __restrict__ topk_w, int32_t* __restrict__ row_token,
+                   int32_t* __restrict__ inv_row, int32_t* __restrict__ dest_rank, int32_t* __restrict__ seg_offsets_a,
+                   int32_t* __restrict__ seg_offsets_b, unsigned long long* __restrict__ workload,
+                   unsigned long long* __restrict__ rank_load, unsigned long long* __restrict__ dispatch_tokens,
+                   unsigned long long* __restrict__ dispatch_bytes, unsigned long long bytes_per_token,
+                   int32_t* __restrict__ status) {
+    __shared__ uint32_t mask[kMaxE][kFrontWarps];
+    __shared__ uint16_t warp_prefix[kMaxE][kFrontWarps];
+    __shared__ uint8_t s_idx[kFrontTokens][kMaxK];
+    __shared__ int32_t s_seg[kMaxG + 1];              // slot lengths, then their exclusive scan
+    __shared__ int32_t warp_sum[kFrontThreads / 32];
+    __shared__ uint32_t h_rr[kMaxR * kMaxR];          // [src][dest]
+    __shared__ uint32_t h_load[kMaxR];
+    const int tid = threadIdx.x;
+
+    for (int i = tid; i < E * kFrontWarps; i += kFrontThreads) (&mask[0][0])[i] = 0u;
+    for (int i = tid; i <= G; i += kFrontThreads) s_seg[i] = 0;
+    for (int i = tid; i < R * R; i += kFrontThreads) h_rr[i] = 0u;
+    for (int i = tid; i < R; i += kFrontThreads) h_load[i] = 0u;
+    for (int i = tid; i < R * E; i += kFrontThreads) workload[i] = 0ull;
+    for (int i = tid; i < R; i += kFrontThreads) rank_load[i] = 0ull;
+    for (int i = tid; i < R * R; i += kFrontThreads) { dispatch_tokens[i] = 0ull; dispatch_bytes[i] = 0ull; }
+
+    // ---- gate (a1) ----
+    {
+        const int t_raw = tid / kFrontLpt, sub = tid % kFrontLpt;
+        const bool live = t_raw < T;
+        const int t = live ? t_raw : T - 1;
+        int win_idx[8];
+        float win_w[8];
+        if (route_token<VEC, kFrontLpt>(logits + (size_t)t * E, E, K, sub, live, status, win_idx, win_w)) {
+            store_gate(topk_idx + (size_t)t * K, topk_w + (size_t)t * K, K, win_idx, win_w);
+#pragma unroll
+            for (int s = 0; s < 8; ++s)
+                if (s < K) s_idx[t][s] = (uint8_t)win_idx[s];
+        }
+    }
+    __syncthreads();
+
+    // ---- counting sort of the single tile (a2 indices) ----
+    const int w = tid >> 5, lane = tid & 31;
+    const bool token_thread = tid < T;                 // T <= 256: thread t is token t from here on
+    if (token_thread)
+        for (int s = 0; s < K; ++s) atomicOr(&mask[s_idx[tid][s]][w], 1u << lane);
+    __syncthreads();
+    for (int e = tid; e < E; e += kFrontThreads) {
+        int run = 0;
+#pragma unroll
+        for (int ww = 0; ww < kFrontWarps; ++ww) { warp_prefix[e][ww] = (uint16_t)run; run += __popc(mask[e][ww]); }
+        const int r0 = __ldg(rep_start + e), r_e = __ldg(rep_start + e + 1) - r0;
+        for (int q = 0; q < r_e; ++q)                   // replica q gets ceil((N_e - q) / r_e) rows
+            s_seg[__ldg(rep_slot + r0 + q)] = (run > q) ? (run - q + r_e - 1) / r_e : 0;
+    }
+    __syncthreads();
+    // exclusive scan of the G <= 1024 slot lengths: thread g owns slot g
+    {
+        const int len = tid < G ? s_seg[tid] : 0;
+        int incl = len;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) warp_sum[w] = incl;
+        __syncthreads();
+        int base = incl - len;
+        for (int i = 0; i < w; ++i) base += warp_sum[i];
+        __syncthreads();                                // every thread has read its slot length
+        if (tid < G) s_seg[tid] = base;
+        if (tid == G - 1) s_seg[G] = base + len;
+        __syncthreads();
+        for (int g = tid; g <= G; g += kFrontThreads) {
+            seg_offsets_a[g] = s_seg[g];
+            if (seg_offsets_b) seg_offsets_b[g] = s_seg[g];
+        }
+    }
+
+    // ---- rows (a2) and histograms (a5) per assignment ----
+    if (token_thread) {
+        const int t = tid;
+        const int src = (int)(((long long)t * R) / T);
+        for (int s = 0; s < K; ++s) {
+            const int e = s_idx[t][s];
+            const int n = warp_prefix[e][w] + __popc(mask[e][w] & ((1u << lane) - 1u));
+            const int r0 = __ldg(rep_start + e), r_e = __ldg(rep_start + e + 1) - r0;
+            const int slot = __ldg(rep_slot + r0 + n % r_e);
+            const int row = s_seg[slot] + n / r_e;
+            const int dest = slot / C_max;
+            row_token[row] = t;
+            inv_row[(size_t)t * K + s] = row;
+            dest_rank[(size_t)t * K + s] = dest;
+            atomicAdd(&h_rr[src * R + dest], 1u);
+            atomicAdd(&h_load[dest], 1u);
+            atomicAdd(workload + (size_t)src * E + e, 1ull);     // zeroed above, before the first barrier
+        }
+    }
+    __syncthreads();
+    for (int i = tid; i < R * R; i += kFrontThreads) {
+        const unsigned long long c = h_rr[i];
+        dispatch_tokens[i] = c;
+        dispatch_bytes[i] = c * bytes_per_token;
+    }
+    for (int i = tid; i < R; i += kFrontThreads) rank_load[i] = h_load[i];
+}
+
 }  // namespace
+
+bool front_small_applies(const director_ctx* ctx, int T) {
+    return T <= kFrontTokens && ctx->replica_policy == DIRECTOR_REPLICA_ROUND_ROBIN;
+}
+
+// Gate + dispatch indices + placement cost of a batch of at most 256 tokens in one launch.
+int launch_front_small(director_ctx* ctx, int T, const float* logits, int32_t* topk_idx, float* topk_w,
+                       int32_t* row_token, int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, int64_t* workload,
+                       int64_t* rank_load, int64_t* dispatch_tokens, uint64_t* dispatch_bytes, cudaStream_t st) {
+    const director_shape& s = ctx->shape;
+    LaunchScope scope(ctx, st, "front_small_kernel");
+#define FRONT_LAUNCH(VEC)                                                                                              \
+    front_small_kernel<VEC><<<1, kFrontThreads, 0, st>>>(                                                              \
+        logits, T, s.E, s.K, s.R, s.C_max, ctx->G, ctx->d_rep_start, ctx->d_rep_slot, topk_idx, topk_w, row_token,     \
+        inv_row, dest_rank, seg_offsets, ctx->d_seg_offsets, reinterpret_cast<unsigned long long*>(workload),          \
+        reinterpret_cast<unsigned long long*>(rank_load), reinterpret_cast<unsigned long long*>(dispatch_tokens),      \
+        reinterpret_cast<unsigned long long*>(dispatch_bytes), (unsigned long long)s.H * 2ull, ctx->d_status)
+    if (s.E % 4 == 0) FRONT_LAUNCH(true); else FRONT_LAUNCH(false);
+#undef FRONT_LAUNCH
+    return cuda_status(cudaGetLastError());
+}
 
 int launch_route(director_ctx* ctx, int T, const float* logits, int32_t* topk_idx, float* topk_w, cudaStream_t st) {
     const int E = ctx->shape.E, K = ctx->shape.K;
@@ -236,6 +394,7 @@ int launch_route(director_ctx* ctx, int T, const float* logits, int32_t* topk_id
     const int groups = (E + 7) / 8;
     int lpt = 1;
     while (lpt < 8 && 2 * lpt <= groups && ((long long)T * lpt < 131072 || groups > 4 * lpt)) lpt *= 2;
+    if (T >= (1 << 19)) lpt = 1;   // far above the launch-latency regime a lane per token executes the fewest instructions
     const long long threads = (long long)T * lpt;
     const dim3 grid((unsigned)((threads + kRouteThreads - 1) / kRouteThreads)), block(kRouteThreads);
     LaunchScope scope(ctx, st, "route_topk_kernel");

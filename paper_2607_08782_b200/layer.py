@@ -102,16 +102,19 @@ class MoELayer:
         fused: dispatch produces indices only and the expert GEMM gathers its rows from x.  Off by default: the
         weight-stationary GEMM re-reads a token tile once per weight block, so the gather is repeated 2F/256 times
         and costs more than the single row copy it saves."""
-        self.route(T, logits)
-        if fused and self.ffn_variant == 2:
-            self.dispatch(T, x, indices_only=True)
+        gather = fused and self.ffn_variant == 2
+        if with_cost:          # front end in one call (a single launch for decode-sized batches)
+            self.d.route_dispatch_cost(T, logits, x, self.topk_idx, self.topk_w, None if gather else self.xp,
+                                       self.row_token, self.inv_row, self.dest_rank, self.seg_offsets, self.workload,
+                                       self.rank_load, self.dispatch_tokens, self.dispatch_bytes)
+        else:
+            self.route(T, logits)
+            self.dispatch(T, x, indices_only=gather)
+        if gather:
             self.expert_ffn_gather(T, x)
         else:
-            self.dispatch(T, x)
             self.expert_ffn(T, x)
         self.combine(T)
-        if with_cost:
-            self.placement_cost(T)
         return self.y[:T]
 
     def capture(self, T, logits, x, with_cost=True, fused=False):

@@ -325,6 +325,34 @@ def test_k1_and_minimum_hidden_size_with_t_below_t_max():
     _check_outputs(shape, g, x, weights, idx, w, w64, d, c, np.arange(100), "k1")
 
 
+def test_routing_and_indices_at_half_a_million_tokens():
+    """Far above the paper's batch sizes: 2049 count tiles, the one-lane-per-token routing configuration."""
+    import torch
+    from paper_2607_08782_b200.binding import Director
+    T, E, K, R, C = (1 << 19) + 5, 24, 3, 4, 8
+    shape = synth.Shape("huge", T, 256, E, K, 128, 0, R, C, 1.2, 93)
+    logits = synth.make_logits(shape)
+    X = _random_placement(93, E, R, C, 5)
+    d = Director(T, 256, 128, E, K, 0, R, C)
+    d.set_placement(X)
+    i32 = dict(dtype=torch.int32, device="cuda")
+    idx, w = torch.empty((T, K), **i32), torch.empty((T, K), dtype=torch.float32, device="cuda")
+    row_token, inv_row, dest = torch.empty(T * K, **i32), torch.empty((T, K), **i32), torch.empty((T, K), **i32)
+    seg = torch.empty(R * C + 1, **i32)
+    d.route(T, torch.from_numpy(logits).cuda(), idx, w)
+    d.dispatch(T, None, idx, None, row_token, inv_row, dest, seg)
+    torch.cuda.synchronize()
+    assert d.last_status() == 0
+    idx_o, _, w64 = orc.route(logits, K)
+    assert np.array_equal(idx.cpu().numpy(), idx_o)
+    assert np.max(np.abs(w.cpu().numpy().astype(np.float64) - w64)) <= W_TOL
+    d_o = orc.dispatch(idx_o, X, C)
+    assert np.array_equal(seg.cpu().numpy(), d_o["seg_offsets"])
+    assert np.array_equal(inv_row.cpu().numpy(), d_o["inv_row"])
+    assert np.array_equal(dest.cpu().numpy(), d_o["dest_rank"])
+    assert np.array_equal(row_token.cpu().numpy(), d_o["row_token"])
+
+
 def test_cuda_graph_replay_reproduces_the_direct_pass():
     """Every entry point is capturable: a graph of the whole layer replays to the same bits, also after the
     inputs in the captured buffers have changed."""
@@ -377,3 +405,50 @@ def test_gathering_gemm_matches_the_materialised_permutation_bit_for_bit(seed, T
     assert np.array_equal(tensor_to_bf16_bits(L.y[:T]), g.y)
     assert np.array_equal(L.inv_row[:T].cpu().numpy(), g.inv_row)
     assert bool(torch.isnan(L.xp[:T * K]).all())
+
+
+@pytest.mark.parametrize("seed,T,H,E,K,F,R,C,extra", [
+    (61, 1, 256, 128, 8, 128, 16, 9, 16),       # one token
+    (62, 64, 256, 128, 8, 128, 16, 9, 16),      # a decode batch
+    (63, 255, 256, 13, 3, 128, 4, 5, 6),        # E not a multiple of 4 (scalar loads), ragged
+    (64, 256, 256, 256, 8, 128, 64, 4, 0),      # the largest fused batch, the largest E and R
+    (65, 200, 256, 7, 1, 128, 3, 16, 20),       # K = 1, heavy replication, the largest C_max
+    (66, 257, 256, 16, 2, 128, 4, 4, 0),        # one token too many for the fused kernel: the separate kernels run
+])
+def test_fused_front_end_matches_the_separate_stages_and_the_oracle(seed, T, H, E, K, F, R, C, extra):
+    import torch
+    shape, logits, x, weights = _custom(seed, T, H, E, K, F, 0, R, C)
+    X = _random_placement(seed, E, R, C, extra)
+    case = GpuCase(shape, logits, x, weights)
+    g = case.run(X, stages="front")                       # route, dispatch, placement_cost as separate calls
+    L = case.layer
+    i32 = dict(dtype=torch.int32, device="cuda")
+    i64 = dict(dtype=torch.int64, device="cuda")
+    A = T * K
+    o = dict(idx=torch.full((T, K), -7, **i32), w=torch.zeros((T, K), dtype=torch.float32, device="cuda"),
+             xp=torch.zeros_like(L.xp), row_token=torch.full((A,), -7, **i32), inv_row=torch.full((T, K), -7, **i32),
+             dest=torch.full((T, K), -7, **i32), seg=torch.full((R * C + 1,), -7, **i32),
+             W=torch.full((R, E), -7, **i64), load=torch.full((R,), -7, **i64), dt=torch.full((R, R), -7, **i64),
+             db=torch.full((R, R), -7, **i64))
+    n0 = L.d.launch_count()
+    L.d.route_dispatch_cost(T, case.logits, case.x, o["idx"], o["w"], o["xp"], o["row_token"], o["inv_row"], o["dest"],
+                            o["seg"], o["W"], o["load"], o["dt"], o["db"])
+    torch.cuda.synchronize()
+    assert L.d.last_status() == 0
+    assert L.d.launch_count() - n0 == (2 if T <= 256 else 6)
+    from paper_2607_08782_b200.layer import tensor_to_bf16_bits
+    assert np.array_equal(o["idx"].cpu().numpy(), g.topk_idx)
+    assert np.array_equal(o["w"].cpu().numpy(), g.topk_w)                # same arithmetic: same bits
+    assert np.array_equal(tensor_to_bf16_bits(o["xp"][:A]), g.xp)
+    for k, ref in (("row_token", g.row_token), ("inv_row", g.inv_row), ("dest", g.dest_rank), ("seg", g.seg_offsets),
+                   ("W", g.workload), ("load", g.rank_load), ("dt", g.dispatch_tokens)):
+        assert np.array_equal(o[k].cpu().numpy(), ref), k
+    assert np.array_equal(o["db"].cpu().numpy().view(np.uint64), g.dispatch_bytes)
+    idx, w, w64, d, c = _oracle_front(shape, logits, x, X, C)
+    check_integer_parity(g, idx, d, c, f"front{seed}")
+    # indices only
+    o["inv_row"].fill_(-7)
+    L.d.route_dispatch_cost(T, case.logits, None, o["idx"], o["w"], None, o["row_token"], o["inv_row"], o["dest"],
+                            o["seg"], o["W"], o["load"], o["dt"], o["db"])
+    torch.cuda.synchronize()
+    assert np.array_equal(o["inv_row"].cpu().numpy(), d["inv_row"])
