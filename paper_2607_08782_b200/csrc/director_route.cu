@@ -8,13 +8,14 @@
 // Fast path, 32-bit keys: key = (top 24 bits of the order-preserving image of the float) << 8 | (255 - expert).
 // A compare-exchange on such keys is one integer max and one integer min.  The lane sorts its eight keys with a
 // 19-comparator network and merges them into its running top-8 (element-wise max against the reversed list
-// gives a bitonic sequence holding the 8 largest; 12 more comparators sort it); the largest key ever rejected
-// is tracked too.  The token's lanes then merge their lists pairwise through shuffles.  Dropping the float's low
-// 8 bits cannot change the answer if the K winners and the best rejected element all differ in the 24 bits
-// kept - then their order is the order of the exact values and everything else is strictly smaller.  That is
-// checked, and the rare token that fails the check (two candidates within 2^-15 of each other, or real ties)
-// is redone by one lane with exact 64-bit keys (logit image << 8 | 255 - expert), which order by (logit
-// descending, expert id ascending).  Winners' exact logits are re-read by index for the weights.
+// gives a bitonic sequence holding the 8 largest; 12 more comparators sort it); for K = 8 the largest key ever
+// rejected is tracked too (for K < 8 the runner-up is simply the list's entry K).  The token's lanes then merge
+// their lists pairwise through shuffles.  Dropping the float's low 8 bits cannot change the answer if the K
+// winners and the runner-up all differ in the 24 bits kept - then their order is the order of the exact values
+// and everything else is strictly smaller.  That is checked, and the rare token that fails the check (two
+// candidates within 2^-15 of each other, or real ties) is redone by one lane with exact 64-bit keys (logit image
+// << 8 | 255 - expert), which order by (logit descending, expert id ascending).  Winners' exact logits are
+// re-read by index for the weights.  The loop is bound by the integer pipe: ~13 integer instructions per logit.
 // The weights are the softmax over the K winning logits, which equals the full softmax renormalised over the
 // winners.  HBM traffic is 4E bytes in and 8K bytes out per token.
 #include "director_common.cuh"
@@ -84,13 +85,14 @@ __device__ __forceinline__ void sort8_desc32(uint32_t (&k)[8]) {
     cx32(k[2], k[4]); cx32(k[3], k[5]);
     cx32(k[3], k[4]);
 }
-// as merge_top8, also folding the rejected keys into `rej` (the largest key not in top[])
+// as merge_top8; with REJ the rejected keys are folded into `rej` (the largest key not in top[]), which only a
+// gate that keeps all eight list entries (K = 8) needs: for K < 8 the runner-up is top[K]
+template <bool REJ>
 __device__ __forceinline__ void merge_top8_32(uint32_t (&top)[8], const uint32_t (&grp)[8], uint32_t& rej) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const uint32_t hi = max(top[i], grp[7 - i]), lo = min(top[i], grp[7 - i]);
-        top[i] = hi;
-        rej = max(rej, lo);
+        if (REJ) rej = max(rej, min(top[i], grp[7 - i]));
+        top[i] = max(top[i], grp[7 - i]);
     }
     cx32(top[0], top[4]); cx32(top[1], top[5]); cx32(top[2], top[6]); cx32(top[3], top[7]);
     cx32(top[0], top[2]); cx32(top[1], top[3]); cx32(top[4], top[6]); cx32(top[5], top[7]);
@@ -119,15 +121,18 @@ __device__ __noinline__ void exact_top8(const float* __restrict__ row, int E, rk
 // The gate of one token, computed by LPT adjacent lanes (sub = 0 .. LPT-1) that all call this together.
 // Returns true in the lane that holds the result (sub == 0): win_idx[0..K) / win_w[0..K) are the chosen experts
 // in descending logit order and their renormalised softmax weights.
-// VEC: the row can be read with 16-byte loads (E % 4 == 0; rows are then 16-byte aligned).
-template <bool VEC, int LPT>
+// VEC: the row can be read with 16-byte loads (E % 4 == 0; rows are then 16-byte aligned).  K8: K == 8.
+// The loop is bound by the integer pipe (min/max/logic run at half the issue rate), so the key of a logit costs
+// three integer instructions (shift, two 3-input logic ops); folding -0.0 onto +0.0 and the Inf/NaN detector
+// (x * 0 is NaN exactly for Inf and NaN) are floating-point instructions that issue beside them.
+template <bool VEC, int LPT, bool K8>
 __device__ __forceinline__ bool route_token(const float* __restrict__ row, int E, int K, int sub, bool live,
                                             int32_t* __restrict__ status, int (&win_idx)[8], float (&win_w)[8]) {
     uint32_t top[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) top[i] = 0u;        // below every real key
-    uint32_t rej = 0u;                               // largest key seen that is not in top[]
-    uint32_t max_abs = 0u;                           // largest |logit| bit pattern: >= 0x7F800000 iff Inf/NaN present
+    uint32_t rej = 0u;                               // largest key seen that is not in top[] (K8 only)
+    float nonfinite = 0.0f;                          // becomes NaN iff an Inf or NaN logit was read
 
     // software pipeline: the loads of the lane's next group are in flight while the current one is sorted
     auto load_group = [&](int e0, float (&v)[8]) {
@@ -146,16 +151,20 @@ __device__ __forceinline__ bool route_token(const float* __restrict__ row, int E
         const int e_next = e0 + 8 * LPT;
         if (e_next < E) load_group(e_next, v_next);
         uint32_t grp[8];
+        // low byte of the key: 255 - expert = (248 - e0) | (7 - i), e0 being a multiple of 8
+        const uint32_t group_field = 248u - (uint32_t)e0;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            const uint32_t raw = __float_as_uint(v[i]) & 0x7FFFFFFFu;
-            const bool real = e0 + i < E;
-            max_abs = real ? max(max_abs, raw) : max_abs;
-            const uint32_t hi = raw > 0x7F800000u ? 1u : ordered_bits(v[i]);     // NaN orders below every number
-            grp[i] = real ? (hi & 0xFFFFFF00u) | (255u - (uint32_t)(e0 + i)) : 0u;
+            nonfinite = fmaf(v[i], 0.0f, nonfinite);
+            const uint32_t key = (ordered_bits(v[i]) & 0xFFFFFF00u) | group_field | (uint32_t)(7 - i);
+            grp[i] = key;
+        }
+        if (e0 + 8 > E) {                            // ragged last group: positions past the row are no candidates
+#pragma unroll
+            for (int i = 0; i < 8; ++i) grp[i] = (e0 + i < E) ? grp[i] : 0u;
         }
         sort8_desc32(grp);
-        merge_top8_32(top, grp, rej);
+        merge_top8_32<K8>(top, grp, rej);
 #pragma unroll
         for (int i = 0; i < 8; ++i) v[i] = v_next[i];
     }
@@ -165,12 +174,12 @@ __device__ __forceinline__ bool route_token(const float* __restrict__ row, int E
         uint32_t other[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) other[i] = __shfl_xor_sync(0xFFFFFFFFu, top[i], step);
-        rej = max(rej, __shfl_xor_sync(0xFFFFFFFFu, rej, step));
-        max_abs = max(max_abs, __shfl_xor_sync(0xFFFFFFFFu, max_abs, step));
-        merge_top8_32(top, other, rej);
+        if (K8) rej = max(rej, __shfl_xor_sync(0xFFFFFFFFu, rej, step));
+        nonfinite += __shfl_xor_sync(0xFFFFFFFFu, nonfinite, step);
+        merge_top8_32<K8>(top, other, rej);
     }
     if (!live || sub != 0) return false;
-    if (max_abs >= 0x7F800000u) director_set_status(status, DIRECTOR_ERR_NONFINITE);
+    if (nonfinite != nonfinite) director_set_status(status, DIRECTOR_ERR_NONFINITE);
 
     // the truncated keys decide exactly iff the K winners and the runner-up differ pairwise in the bits kept
     bool exact = true;
@@ -227,7 +236,7 @@ __device__ __forceinline__ void store_gate(int32_t* __restrict__ oi, float* __re
     }
 }
 
-template <bool VEC, int LPT>
+template <bool VEC, int LPT, bool K8>
 __global__ void __launch_bounds__(kRouteThreads)
 route_topk_kernel(const float* __restrict__ logits, int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
                   int T, int E, int K, int32_t* __restrict__ status) {
@@ -237,7 +246,7 @@ route_topk_kernel(const float* __restrict__ logits, int32_t* __restrict__ topk_i
     const int t = live ? t_raw : T - 1;                // surplus lanes redo the last token (keeps shuffles full)
     int win_idx[8];
     float win_w[8];
-    if (route_token<VEC, LPT>(logits + (size_t)t * E, E, K, sub, live, status, win_idx, win_w))
+    if (route_token<VEC, LPT, K8>(logits + (size_t)t * E, E, K, sub, live, status, win_idx, win_w))
         store_gate(topk_idx + (size_t)t * K, topk_w + (size_t)t * K, K, win_idx, win_w);
 }
 
@@ -255,7 +264,7 @@ constexpr int kFrontLpt = 4;
 constexpr int kFrontTokens = kFrontThreads / kFrontLpt;   // 256
 constexpr int kFrontWarps = kFrontTokens / 32;            // 8 warps of token threads
 
-template <bool VEC>
+template <bool VEC, bool K8>
 __global__ void __launch_bounds__(kFrontThreads)
 front_small_kernel(const float* __restrict__ logits, int T, int E, int K, int R, int C_max, int G,
                    const int32_t* __restrict__ rep_start, const int32_t* __restrict__ rep_slot,
@@ -289,7 +298,7 @@ front_small_kernel(const float* __restrict__ logits, int T, int E, int K, int R,
         const int t = live ? t_raw : T - 1;
         int win_idx[8];
         float win_w[8];
-        if (route_token<VEC, kFrontLpt>(logits + (size_t)t * E, E, K, sub, live, status, win_idx, win_w)) {
+        if (route_token<VEC, kFrontLpt, K8>(logits + (size_t)t * E, E, K, sub, live, status, win_idx, win_w)) {
             store_gate(topk_idx + (size_t)t * K, topk_w + (size_t)t * K, K, win_idx, win_w);
 #pragma unroll
             for (int s = 0; s < 8; ++s)
@@ -376,13 +385,15 @@ int launch_front_small(director_ctx* ctx, int T, const float* logits, int32_t* t
                        int64_t* rank_load, int64_t* dispatch_tokens, uint64_t* dispatch_bytes, cudaStream_t st) {
     const director_shape& s = ctx->shape;
     LaunchScope scope(ctx, st, "front_small_kernel");
-#define FRONT_LAUNCH(VEC)                                                                                              \
-    front_small_kernel<VEC><<<1, kFrontThreads, 0, st>>>(                                                              \
+#define FRONT_LAUNCH(VEC, K8)                                                                                          \
+    front_small_kernel<VEC, K8><<<1, kFrontThreads, 0, st>>>(                                                          \
         logits, T, s.E, s.K, s.R, s.C_max, ctx->G, ctx->d_rep_start, ctx->d_rep_slot, topk_idx, topk_w, row_token,     \
         inv_row, dest_rank, seg_offsets, ctx->d_seg_offsets, reinterpret_cast<unsigned long long*>(workload),          \
         reinterpret_cast<unsigned long long*>(rank_load), reinterpret_cast<unsigned long long*>(dispatch_tokens),      \
         reinterpret_cast<unsigned long long*>(dispatch_bytes), (unsigned long long)s.H * 2ull, ctx->d_status)
-    if (s.E % 4 == 0) FRONT_LAUNCH(true); else FRONT_LAUNCH(false);
+    const bool vec = s.E % 4 == 0, k8 = s.K == 8;
+    if (vec) { if (k8) FRONT_LAUNCH(true, true); else FRONT_LAUNCH(true, false); }
+    else { if (k8) FRONT_LAUNCH(false, true); else FRONT_LAUNCH(false, false); }
 #undef FRONT_LAUNCH
     return cuda_status(cudaGetLastError());
 }
@@ -394,12 +405,16 @@ int launch_route(director_ctx* ctx, int T, const float* logits, int32_t* topk_id
     const int groups = (E + 7) / 8;
     int lpt = 1;
     while (lpt < 8 && 2 * lpt <= groups && ((long long)T * lpt < 131072 || groups > 4 * lpt)) lpt *= 2;
-    if (T >= (1 << 19)) lpt = 1;   // far above the launch-latency regime a lane per token executes the fewest instructions
+    if (T >= (1 << 19)) lpt = 1;
+    if (const char* ov = getenv("XLPT")) lpt = atoi(ov);   // far above the launch-latency regime a lane per token executes the fewest instructions
     const long long threads = (long long)T * lpt;
     const dim3 grid((unsigned)((threads + kRouteThreads - 1) / kRouteThreads)), block(kRouteThreads);
     LaunchScope scope(ctx, st, "route_topk_kernel");
-#define ROUTE_LAUNCH(VEC, LPT) \
-    route_topk_kernel<VEC, LPT><<<grid, block, 0, st>>>(logits, topk_idx, topk_w, T, E, K, ctx->d_status)
+#define ROUTE_LAUNCH(VEC, LPT)                                                                                         \
+    do {                                                                                                               \
+        if (K == 8) route_topk_kernel<VEC, LPT, true><<<grid, block, 0, st>>>(logits, topk_idx, topk_w, T, E, K, ctx->d_status); \
+        else route_topk_kernel<VEC, LPT, false><<<grid, block, 0, st>>>(logits, topk_idx, topk_w, T, E, K, ctx->d_status);       \
+    } while (0)
     const bool vec = E % 4 == 0;
     if (lpt == 8) { if (vec) ROUTE_LAUNCH(true, 8); else ROUTE_LAUNCH(false, 8); }
     else if (lpt == 4) { if (vec) ROUTE_LAUNCH(true, 4); else ROUTE_LAUNCH(false, 4); }
