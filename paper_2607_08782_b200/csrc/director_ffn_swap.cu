@@ -30,9 +30,15 @@ using namespace umma;
 
 namespace {
 
-constexpr int S_STAGES = 6;
 constexpr int S_STAGE_BYTES = A_BYTES + B_HALF_BYTES;          // 16 KB weights + 16 KB tokens per CTA per k-step
-constexpr int S_SMEM_BYTES = S_STAGES * S_STAGE_BYTES + 1024 + 256 + TABLE_INTS * 4;
+constexpr int S_HEADER_BYTES = 320;                            // barriers, scheduler ring, TMEM slot, scratch
+constexpr int S_MAX_SMEM = 232448;                             // opt-in shared memory per CTA on sm_100
+// Shared memory of a launch: alignment slack, the operand ring, the header, and the segment tables of its G slots
+// (seg_offsets and token-tile prefix as int32, expert ids as int16).
+constexpr int swap_smem_bytes(int stages, int G) { return 1024 + stages * S_STAGE_BYTES + S_HEADER_BYTES + (G + 1) * 10 + 6; }
+// The operand stream is latency-bound (a stage comes back ~2.5 us after it is released), so the ring is as deep as
+// shared memory allows: seven stages when the segment tables are small enough, else six.
+inline int swap_stages(int G) { return swap_smem_bytes(7, G) <= S_MAX_SMEM ? 7 : 6; }
 constexpr int TOKEN_TILE = 256;                                // tokens per full tile (N of the pair's MMA)
 constexpr int TOKEN_STEP = 32;                                 // granularity of N
 // Epilogue warps per TMEM lane quadrant.  The SwiGLU epilogue of GEMM-1 is long (shuffle, exp, reciprocal,
@@ -117,7 +123,7 @@ struct SwapTile {
 struct SwapWalker {
     const int32_t* seg_off;
     const int32_t* tt_start;    // prefix of token tiles per segment
-    const int32_t* expert;
+    const int16_t* expert;
     int w_blocks, w_rows_per_expert, rows_per_block, total, g = 0;
     __device__ bool get(int w, SwapTile& t) {
         if (w >= total) return false;
@@ -138,7 +144,7 @@ struct SwapWalker {
 // GATHER (GEMM-1 only): the token rows are not read from a permuted copy but gathered straight from the layer
 // input x through row_token - tm_x then describes x with a one-row box and the whole producer warp issues the
 // loads, four rows per lane - so the dispatch step needs no row copies at all.
-template <int MODE, int EPI_GROUPS, bool GATHER>
+template <int MODE, int EPI_GROUPS, bool GATHER, int S_STAGES>
 __global__ void __launch_bounds__(64 + 128 * EPI_GROUPS, 1)
 grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
                          const SwapParams p) {
@@ -146,32 +152,32 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     uint8_t* gen = smem_raw + (tiles - raw) + S_STAGES * S_STAGE_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(gen);             // full[6] empty[6] tfull[2] tempty[2]
-    // sched_full[4] at +128, sched_empty[4] at +160 (the leader's are the ones used)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + 192);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + 196);
-    volatile int* sched_item = reinterpret_cast<volatile int*>(gen + 200);   // [4]
-    int32_t* warp_sum = reinterpret_cast<int32_t*>(gen + 216);     // [10]
-    int32_t* s_seg = reinterpret_cast<int32_t*>(gen + 256);
-    int32_t* s_tt = s_seg + (kMaxG + 1);
-    int32_t* s_exp = s_tt + (kMaxG + 1);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(gen);             // full[8] empty[8] tfull[2] tempty[2]
+    // sched_full[4] at +160, sched_empty[4] at +192 (the leader's are the ones used)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + 224);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + 228);
+    volatile int* sched_item = reinterpret_cast<volatile int*>(gen + 232);   // [4]
+    int32_t* warp_sum = reinterpret_cast<int32_t*>(gen + 248);     // [10]
+    const int G = p.G;
+    int32_t* s_seg = reinterpret_cast<int32_t*>(gen + S_HEADER_BYTES);
+    int32_t* s_tt = s_seg + (G + 1);
+    int16_t* s_exp = reinterpret_cast<int16_t*>(s_tt + (G + 1));
 
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
-    auto empty_bar = [&](int s) { return bar0 + 8u * (S_STAGES + s); };
-    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * S_STAGES + a); };
-    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * S_STAGES + 2 + a); };
-    auto sched_full = [&](int q) { return bar0 + 128u + 8u * q; };
-    auto sched_empty = [&](int q) { return bar0 + 160u + 8u * q; };
+    auto empty_bar = [&](int s) { return bar0 + 64u + 8u * s; };
+    auto tfull_bar = [&](int a) { return bar0 + 128u + 8u * a; };
+    auto tempty_bar = [&](int a) { return bar0 + 144u + 8u * a; };
+    auto sched_full = [&](int q) { return bar0 + 160u + 8u * q; };
+    auto sched_empty = [&](int q) { return bar0 + 192u + 8u * q; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int G = p.G;
     const uint32_t rank = cluster_ctarank();
     const bool leader = rank == 0;
 
     constexpr int n_threads = 64 + 128 * EPI_GROUPS;               // producer warp + MMA warp + epilogue warps
     for (int g = threadIdx.x; g <= G; g += n_threads) s_seg[g] = __ldg(p.seg_offsets + g);
-    for (int g = threadIdx.x; g < G; g += n_threads) s_exp[g] = __ldg(p.slot_expert + g);
+    for (int g = threadIdx.x; g < G; g += n_threads) s_exp[g] = (int16_t)__ldg(p.slot_expert + g);
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         for (int s = 0; s < S_STAGES; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
@@ -506,13 +512,13 @@ bool map_interleaved(director_ctx* ctx, CUtensorMap* map, const void* first, uin
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int MODE, int EPI_GROUPS, bool GATHER>
-int launch_swap(director_ctx* ctx, const char* name, const CUtensorMap& w, const CUtensorMap& x, const SwapParams& p,
-                cudaStream_t st) {
+template <int MODE, int EPI_GROUPS, bool GATHER, int STAGES>
+int launch_swap_n(director_ctx* ctx, const char* name, const CUtensorMap& w, const CUtensorMap& x, const SwapParams& p,
+                  cudaStream_t st) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * ctx->pair_clusters));
     cfg.blockDim = dim3(64 + 128 * EPI_GROUPS);
-    cfg.dynamicSmemBytes = S_SMEM_BYTES;
+    cfg.dynamicSmemBytes = (size_t)swap_smem_bytes(STAGES, p.G);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -522,15 +528,29 @@ int launch_swap(director_ctx* ctx, const char* name, const CUtensorMap& w, const
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     LaunchScope scope(ctx, st, name);
-    return cuda_status(cudaLaunchKernelEx(&cfg, grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER>, w, x, p));
+    return cuda_status(cudaLaunchKernelEx(&cfg, grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, STAGES>, w, x, p));
+}
+
+template <int MODE, int EPI_GROUPS, bool GATHER>
+int launch_swap(director_ctx* ctx, const char* name, const CUtensorMap& w, const CUtensorMap& x, const SwapParams& p,
+                cudaStream_t st) {
+    return swap_stages(p.G) == 7 ? launch_swap_n<MODE, EPI_GROUPS, GATHER, 7>(ctx, name, w, x, p, st)
+                                 : launch_swap_n<MODE, EPI_GROUPS, GATHER, 6>(ctx, name, w, x, p, st);
+}
+
+template <int MODE, int EPI_GROUPS, bool GATHER>
+bool swap_opt_in() {
+    return cudaFuncSetAttribute(grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, 6>,
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, swap_smem_bytes(6, kMaxG)) == cudaSuccess &&
+           cudaFuncSetAttribute(grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, 7>,
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, S_MAX_SMEM) == cudaSuccess;
 }
 
 }  // namespace
 
 int ffn_swap_init(director_ctx*) {
-    if (cudaFuncSetAttribute(grouped_gemm_swap_kernel<0, EPI_GROUPS_GEMM1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, S_SMEM_BYTES) != cudaSuccess ||
-        cudaFuncSetAttribute(grouped_gemm_swap_kernel<0, EPI_GROUPS_GEMM1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, S_SMEM_BYTES) != cudaSuccess ||
-        cudaFuncSetAttribute(grouped_gemm_swap_kernel<1, EPI_GROUPS_GEMM2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, S_SMEM_BYTES) != cudaSuccess)
+    if (!swap_opt_in<0, EPI_GROUPS_GEMM1, false>() || !swap_opt_in<0, EPI_GROUPS_GEMM1, true>() ||
+        !swap_opt_in<1, EPI_GROUPS_GEMM2, false>())
         return DIRECTOR_ERR_CUDA;
     return DIRECTOR_OK;
 }
