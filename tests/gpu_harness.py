@@ -11,7 +11,7 @@ from paper_2607_08782_b200 import synth
 
 
 @dataclass
-class GpuRun:
+class GpuResult:
     topk_idx: np.ndarray
     topk_w: np.ndarray
     xp: np.ndarray           # bf16 bits
@@ -53,7 +53,7 @@ class GpuCase:
             sd = bf16_bits_to_tensor(synth.concat_shared_down(w.ws_down), dev)
         self.layer = MoELayer(T_max or s.T, s.H, s.F, s.E, s.K, s.S, s.R, self.C_max, wg, wu, wd, sg, su, sd, dev)
 
-    def run(self, X, T=None, src=None, stages="all", policy=0) -> GpuRun:
+    def run(self, X, T=None, src=None, stages="all", policy=0) -> GpuResult:
         from paper_2607_08782_b200.layer import tensor_to_bf16_bits
         torch, L, s = self.torch, self.layer, self.shape
         T = T or s.T
@@ -74,7 +74,7 @@ class GpuCase:
         torch.cuda.synchronize()
         status = L.d.last_status()
         A = T * s.K
-        return GpuRun(
+        return GpuResult(
             topk_idx=L.topk_idx[:T].cpu().numpy(), topk_w=L.topk_w[:T].cpu().numpy(),
             xp=tensor_to_bf16_bits(L.xp[:A]), yp=tensor_to_bf16_bits(L.yp[:A]),
             row_token=L.row_token[:A].cpu().numpy(), inv_row=L.inv_row[:T].cpu().numpy(),
@@ -96,7 +96,7 @@ def max_abs(a: np.ndarray, b: np.ndarray) -> float:
     return float(np.max(np.abs(a.astype(np.float64) - b))) if a.size else 0.0
 
 
-def check_integer_parity(g: GpuRun, idx_o, d_o, c_o, label=""):
+def check_integer_parity(g: GpuResult, idx_o, d_o, c_o, label=""):
     """Bit-exact comparison of everything integer against the oracle."""
     assert np.array_equal(g.topk_idx, idx_o), f"{label}: topk_idx differs"
     for name in ("row_token", "inv_row", "dest_rank", "seg_offsets"):
