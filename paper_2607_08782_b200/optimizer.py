@@ -4,9 +4,12 @@ What follows the paper: the cost model (Eq. 1-4: a layer's latency is the stragg
 straggler's communication), the LP relaxation of the placement problem with the max operators linearised by
 auxiliary variables (Eq. 6), and the binary search over the latency budget beta that Algorithm 1 wraps around
 the feasibility LP.  What does not: the profiled latency functions f_comp / f_comm are not published, so affine
-stand-ins are used (declared in `LatencyModel`), and the paper's iterative randomized rounding (whose constants are
-not given) is replaced by a deterministic rounding followed by a local search whose candidate batches are scored on
-the GPU by `director_placement_cost_batch` - the part of the search that is a data-parallel hot loop.
+stand-ins are used (declared in `LatencyModel`); and the rounding: the paper's iterative randomized rounding is
+here (`iterative_rounding`, with the constants the paper leaves open declared in `RoundingParams`), but at a vertex
+of the LP nearly every latency constraint is tight and its walk can hardly move inside the paper's polytope, so the
+search by default uses a deterministic rounding, or on request several randomized roundings that keep only the
+assignment and capacity constraints hard, and follows either with a local search.  All candidate batches are
+scored on the GPU by `director_placement_cost_batch` - the part of the search that is a data-parallel hot loop.
 
 The LP runs on the host with SciPy (as in the paper's prototype); everything that scores integer placements goes
 through an `evaluate(X_batch) -> summary` callable, by default the GPU evaluator below.
@@ -183,6 +186,204 @@ def round_placement(x_bar: np.ndarray, N: np.ndarray, C_max: int) -> np.ndarray:
     return X
 
 
+# ----------------------------------------------------------------------------------------------
+# iterative randomized rounding (Section VI-C, "Iterative Rounding")
+# ----------------------------------------------------------------------------------------------
+
+@dataclass(frozen=True)
+class RoundingParams:
+    """The constants the paper leaves open, as used here: alpha bounds how far a variable may drift inside one
+    macro-iteration (distance to its nearest integer at most alpha * scale), gamma is the step size of a micro-step
+    in units of the scale, t_micro the number of micro-steps per macro-iteration (None: 40 + 4 * active variables),
+    max_macro the number of macro-iterations (None: 4 + 2 * ceil(log2(number of variables)))."""
+    alpha: float = 2.0
+    gamma: float = 0.25
+    t_micro: int | None = None
+    max_macro: int | None = None
+    tol: float = 1e-6
+    # True: the walk also respects the latency constraints 6b-6d for the given budget (the paper's polytope Q).  At a
+    # vertex of the LP nearly all of them are tight and the walk can hardly move, so the search uses False: only the
+    # assignment and capacity constraints are hard, and the candidates the walk produces are scored afterwards.
+    respect_budget: bool = True
+
+
+def _scales(x: np.ndarray) -> np.ndarray:
+    """s_v = 2^-k with dist(x_v, {0,1}) in (2^-(k+1), 2^-k]  (k >= 1 since the distance is at most 1/2; the interval
+    is closed on the right, so a distance of exactly 2^-k has scale 2^-k)."""
+    d = np.minimum(x, 1.0 - x)
+    k = np.floor(-np.log2(np.maximum(d, 1e-300)))
+    return 2.0 ** -k
+
+
+def rounding_potential(x: np.ndarray, scale: np.ndarray) -> float:
+    """Phi(x) = sum over fractional v of s_v^-2 * dist(x_v, {0,1})^2."""
+    frac = (x > 0.0) & (x < 1.0)
+    d = np.minimum(x, 1.0 - x)
+    return float(np.sum((d[frac] / scale[frac]) ** 2))
+
+
+def iterative_rounding(x_bar: np.ndarray, W: np.ndarray, C_max: int, model: LatencyModel, beta: float,
+                       rng: np.random.Generator, params: RoundingParams = RoundingParams(), trace: list | None = None):
+    """From the fractional LP solution x_bar [E,R] (feasible for budget beta) to an integer placement by the paper's
+    constrained random walk:
+
+      macro-iteration: every fractional variable gets the scale s_v = 2^-k of its distance to the nearest integer.
+      The walk stays in the polytope Q cut out by (i) the LP's constraints 6b-6g, (ii) dist(x_v, {0,1}) <= alpha s_v
+      and (iii) the scale-preserving sums  sum_{v in U_k} x_v = const  over each scale class U_k.  A micro-step draws
+      a Gaussian direction with standard deviation s_v per variable, projects it onto the null space of the
+      constraints of Q that are tight, and moves by gamma along it (shortened so that no constraint of Q is
+      crossed).  A variable that reaches 0 or 1 is clamped there for good.
+
+    Returns (X uint8 [E,R], info).  Variables still fractional after the last macro-iteration are rounded by
+    `round_placement`'s rule; the result is repaired to satisfy the assignment and capacity constraints if the
+    clamping left it short (info counts both)."""
+    R, E = W.shape
+    Wf = W.astype(np.float64)
+    N = Wf.sum(axis=0)
+    tol = params.tol
+    x = np.clip(np.array(x_bar, dtype=np.float64), 0.0, 1.0)
+    x[x < tol] = 0.0
+    x[x > 1.0 - tol] = 1.0
+    nx = E * R
+
+    # gradients of the affine pieces of the objective in x (row-major [E,R] flattened): comp_j and comm_j
+    G_comp = np.zeros((R, nx))
+    G_comm = np.zeros((R, nx))
+    for j in range(R):
+        G_comp[j, np.arange(E) * R + j] = model.comp_per_token * N
+        for k in range(R):
+            if k != j:
+                G_comm[j, np.arange(E) * R + k] += model.comm_per_token * Wf[j]
+    A_assign = np.zeros((E, nx))
+    for i in range(E):
+        A_assign[i, i * R:(i + 1) * R] = 1.0
+    A_cap = np.zeros((R, nx))
+    for j in range(R):
+        A_cap[j, np.arange(E) * R + j] = 1.0
+
+    n_macro = params.max_macro if params.max_macro is not None else 4 + 2 * int(np.ceil(np.log2(max(nx, 2))))
+    info = dict(macro=0, micro=0, clamped=0, fallback=0, repaired=0)
+    xf = x.reshape(-1)
+    for _ in range(n_macro):
+        active = np.flatnonzero((xf > 0.0) & (xf < 1.0))
+        if active.size == 0:
+            break
+        info["macro"] += 1
+        scale = np.ones(nx)
+        scale[active] = _scales(xf[active])
+        classes = np.unique(scale[active])
+        A_scale = np.zeros((len(classes), nx))
+        for c, sc in enumerate(classes):
+            A_scale[c, active[scale[active] == sc]] = 1.0
+        frozen = np.zeros(nx, dtype=bool)                  # reached dist = alpha * s_v in this macro-iteration
+        if trace is not None:
+            trace.append(dict(fractional=int(active.size), potential=rounding_potential(xf, scale)))
+        steps = params.t_micro if params.t_micro is not None else 40 + 4 * int(active.size)
+        for _ in range(steps):
+            mov = active[(xf[active] > 0.0) & (xf[active] < 1.0) & ~frozen[active]]
+            if mov.size == 0:
+                break
+            info["micro"] += 1
+            comp = model.comp_fixed + G_comp @ xf
+            comm = G_comm @ xf
+            budget_slack = beta - (comp.max() + comm.max()) if params.respect_budget else np.inf
+            rows = [A_scale]
+            s_assign = A_assign @ xf - 1.0
+            s_cap = C_max - A_cap @ xf
+            rows.append(A_assign[s_assign <= tol])
+            rows.append(A_cap[s_cap <= tol])
+            scale_tol = tol * max(beta, 1.0)
+            if budget_slack <= scale_tol:
+                rows.append(G_comp[comp >= comp.max() - scale_tol])
+                rows.append(G_comm[comm >= comm.max() - scale_tol])
+            r = rng.standard_normal(mov.size) * scale[mov]
+
+            def project(row_blocks):
+                A = np.vstack(row_blocks)[:, mov]
+                A = A[np.abs(A).sum(axis=1) > 0]
+                if not A.shape[0]:
+                    return r
+                return r - A.T @ np.linalg.lstsq(A @ A.T, A @ r, rcond=None)[0]
+
+            g = project(rows)
+            if not np.any(np.abs(g) > 1e-9 * scale[mov]):
+                # the tight constraints leave no direction: the scale-preserving sums are a device of the analysis,
+                # not of feasibility, so they are the ones to give way
+                g = project(rows[1:])
+                if not np.any(np.abs(g) > 1e-9 * scale[mov]):
+                    break                                   # nothing can move in this macro-iteration any more
+            g[np.abs(g) <= 1e-12] = 0.0
+            # longest step <= gamma that keeps x inside Q
+            t = params.gamma
+            pos, neg = g > 1e-14, g < -1e-14
+            d = np.minimum(xf[mov], 1.0 - xf[mov])
+            toward_int = np.where(xf[mov] <= 0.5, neg, pos)            # moving towards the nearest integer
+            away = ~toward_int & (pos | neg)
+            lim = np.full(mov.size, np.inf)
+            lim[toward_int] = d[toward_int] / np.abs(g[toward_int])                           # reaches 0 or 1
+            # bound (ii): the distance grows until x passes 1/2, so it only binds where alpha * s_v < 1/2
+            room = np.where(params.alpha * scale[mov] >= 0.5, np.inf, params.alpha * scale[mov] - d)
+            lim[away] = np.maximum(room[away], 0.0) / np.abs(g[away])
+            t = min(t, float(lim.min()))
+            full = np.zeros(nx)
+            full[mov] = g
+            for Arow, slack in ((A_assign, s_assign), (-A_cap, s_cap)):                        # non-tight 6e, 6f
+                rate = -(Arow @ full)
+                m = (rate > 1e-9) & (slack > tol)
+                if m.any():
+                    t = min(t, float((np.maximum(slack[m], 0.0) / rate[m]).min()))
+            if budget_slack > scale_tol and params.respect_budget:                             # non-tight 6b-6d
+                rate = (G_comp @ full).max() + (G_comm @ full).max()
+                if rate > 1e-9:
+                    t = min(t, budget_slack / rate)
+            if t <= 0.0:
+                hit = np.zeros(mov.size, dtype=bool)
+                hit[away] = room[away] <= 0.0
+                frozen[mov[hit]] = True
+                if not hit.any():
+                    continue
+                continue
+            xf[mov] += t * g
+            snap0 = xf[mov] <= tol
+            snap1 = xf[mov] >= 1.0 - tol
+            xf[mov[snap0]] = 0.0
+            xf[mov[snap1]] = 1.0
+            info["clamped"] += int(snap0.sum() + snap1.sum())
+            d2 = np.minimum(xf[mov], 1.0 - xf[mov])
+            frozen[mov[(d2 >= params.alpha * scale[mov] - tol) & ~snap0 & ~snap1]] = True
+    x = xf.reshape(E, R)
+    frac_left = (x > 0.0) & (x < 1.0)
+    X = (x >= 1.0 - tol).astype(np.uint8)
+    if frac_left.any():                                    # deterministic finish for what the walk left fractional
+        info["fallback"] = int(frac_left.sum())
+        for i in np.flatnonzero(frac_left.any(axis=1)):
+            if X[i].sum() == 0:
+                free = np.flatnonzero(X.sum(axis=0) < C_max)
+                j = free[np.argmax(x[i, free])] if free.size else int(np.argmax(x[i]))
+                X[i, j] = 1
+    # repair: every expert hosted, no rank above capacity
+    for j in np.flatnonzero(X.sum(axis=0) > C_max):
+        hosted = sorted(np.flatnonzero(X[:, j]), key=lambda i: (X[i].sum() < 2, -N[i]))   # drop replicas first
+        for i in hosted:
+            if X[:, j].sum() <= C_max:
+                break
+            if X[i].sum() >= 2:
+                X[i, j] = 0
+                info["repaired"] += 1
+        for i in sorted(np.flatnonzero(X[:, j]), key=lambda i: N[i]):
+            if X[:, j].sum() <= C_max:
+                break
+            free = np.flatnonzero(X.sum(axis=0) < C_max)
+            X[i, j] = 0
+            X[i, free[np.argmin((X[:, free] * N[:, None]).sum(axis=0))]] = 1
+            info["repaired"] += 1
+    for i in np.flatnonzero(X.sum(axis=1) == 0):
+        free = np.flatnonzero(X.sum(axis=0) < C_max)
+        X[i, free[np.argmax(x_bar[i, free])]] = 1
+        info["repaired"] += 1
+    return X, info
+
+
 def _neighbours(X: np.ndarray, C_max: int):
     """All placements one step away: move one copy of an expert to a rank with a free slot, or swap the copies of
     two experts hosted on different ranks."""
@@ -244,9 +445,13 @@ def local_search(evaluate, X0: np.ndarray, C_max: int, model: LatencyModel, allo
 
 
 def optimize_placement(W: np.ndarray, C_max: int, model: LatencyModel, evaluate, allow_replicas: bool = False,
-                       use_binary_search: bool = True):
+                       use_binary_search: bool = True, rounding: str = "deterministic", n_roundings: int = 16,
+                       seed: int = 0):
     """Algorithm 1 with the stand-ins described in the module header.  W: int64 [R,E] workload matrix.
-    Returns dict(X, latency, lp_bound, x_bar, rounds)."""
+    rounding: "deterministic" (round_placement) or "randomized": n_roundings runs of the paper's iterative randomized
+    rounding (assignment and capacity hard, latency scored afterwards) plus the deterministic one, all scored in one
+    batch, the best one kept.  Either is followed by the local search.
+    Returns dict(X, latency, lp_bound, x_bar, rounds, start_latency)."""
     R, E = W.shape
     N = W.sum(axis=0)
     # a feasible starting budget: round-robin placement of the experts in order of load
@@ -259,12 +464,21 @@ def optimize_placement(W: np.ndarray, C_max: int, model: LatencyModel, evaluate,
         x_bar, bound = binary_search_budget(W, C_max, model, beta_high * (1.0 + 1e-9))
     else:
         x_bar, bound = lp_minimum(W, C_max, model)
-    X0 = round_placement(x_bar, N, C_max)
-    s0 = evaluate(X0[None])[0]
-    if s0[3] != 1 or model.latency(s0[0], s0[1]) > beta_high:
-        X0 = X_rr                                        # rounding never has to be worse than the trivial start
+    starts = [round_placement(x_bar, N, C_max)]
+    if rounding == "randomized":
+        rng = np.random.default_rng(seed)
+        soft = RoundingParams(respect_budget=False)
+        starts += [iterative_rounding(x_bar, W, C_max, model, bound, rng, soft)[0] for _ in range(n_roundings)]
+    elif rounding != "deterministic":
+        raise ValueError(rounding)
+    S = evaluate(np.stack(starts))
+    lat0 = np.where(S[:, 3] == 1, model.latency(S[:, 0], S[:, 1]), np.inf)
+    b = int(np.argmin(lat0))
+    X0, start = starts[b], float(lat0[b])
+    if not start <= beta_high:
+        X0, start = X_rr, beta_high                      # rounding never has to be worse than the trivial start
     X, lat, rounds = local_search(evaluate, X0, C_max, model, allow_replicas)
-    return dict(X=X, latency=lat, lp_bound=bound, x_bar=x_bar, rounds=rounds)
+    return dict(X=X, latency=lat, lp_bound=bound, x_bar=x_bar, rounds=rounds, start_latency=start)
 
 
 def enumerate_single_copy(E: int, R: int, C_max: int):

@@ -83,3 +83,82 @@ def test_rounding_gives_one_copy_per_expert_within_capacity():
     x_bar = rng.dirichlet(np.ones(4), size=10)
     X = opt.round_placement(x_bar, rng.integers(1, 100, size=10), 3)
     assert (X.sum(axis=1) == 1).all() and X.sum(axis=0).max() <= 3
+
+
+# ------------------------------------------------------------------ iterative randomized rounding (Section VI-C)
+
+def _fractional_case(seed, E=12, R=4, C=4, T=400, K=2):
+    shape = synth.Shape(f"round{seed}", T, 256, E, K, 128, 0, R, C, 1.3, 600 + seed)
+    idx, _, _ = orc.route(synth.make_logits(shape), K)
+    W = orc.placement_cost(idx, synth.placement_from_ranks(np.arange(E) % R, R), C, shape.H)["workload"]
+    model = opt.LatencyModel(1.0, 0.0, 0.3 / (2 * shape.H), 2 * shape.H)
+    x_bar, val = opt.lp_minimum(W, C, model)
+    return shape, idx, W, model, x_bar, val
+
+
+def test_scales_follow_the_dyadic_intervals():
+    x = np.array([0.5, 0.3, 0.25, 0.26, 0.1, 0.9, 0.999, 0.0625])
+    s = opt._scales(x)
+    d = np.minimum(x, 1 - x)
+    assert np.all(d <= s + 1e-15) and np.all(d > s / 2 - 1e-15)            # dist in (s/2, s]
+    assert s.tolist() == [0.5, 0.5, 0.25, 0.5, 0.125, 0.125, 2.0 ** -9, 0.0625]
+    assert opt.rounding_potential(np.array([0.0, 1.0, 0.5, 0.25]), np.array([1.0, 1.0, 0.5, 0.25])) == 2.0
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_randomized_rounding_gives_a_valid_placement_and_keeps_integral_entries(seed):
+    shape, idx, W, model, x_bar, val = _fractional_case(seed)
+    E, R, C = shape.E, shape.R, shape.C_max
+    was0, was1 = x_bar < 1e-6, x_bar > 1 - 1e-6
+    assert ((~was0) & (~was1)).sum() >= 4                                 # the case really is fractional
+    for respect in (False, True):
+        trace = []
+        X, info = opt.iterative_rounding(x_bar, W, C, model, val * 1.2, np.random.default_rng(seed),
+                                         opt.RoundingParams(respect_budget=respect), trace=trace)
+        orc.placement_tables(X, C)                                        # every expert hosted, capacity respected
+        assert set(np.unique(X)) <= {0, 1}
+        if info["repaired"] == 0 and info["fallback"] == 0:
+            assert np.all(X[was1] == 1) and np.all(X[was0] == 0)          # the walk never touches integral entries
+        fr = [t["fractional"] for t in trace]
+        assert all(b <= a for a, b in zip(fr, fr[1:]))                    # clamped variables stay clamped
+        if not respect:
+            assert info["fallback"] == 0 and fr[-1] <= fr[0]
+    # same seed, same walk
+    a = opt.iterative_rounding(x_bar, W, C, model, val, np.random.default_rng(9), opt.RoundingParams(respect_budget=False))[0]
+    b = opt.iterative_rounding(x_bar, W, C, model, val, np.random.default_rng(9), opt.RoundingParams(respect_budget=False))[0]
+    assert np.array_equal(a, b)
+
+
+def test_a_micro_step_stays_inside_the_polytope():
+    """One macro-iteration with few steps: assignment sums stay >= 1, rank sums <= C_max, and while nothing has been
+    clamped the scale-preserving sums are unchanged."""
+    shape, idx, W, model, x_bar, val = _fractional_case(1)
+    C = shape.C_max
+    params = opt.RoundingParams(respect_budget=True, t_micro=3, max_macro=1, gamma=0.05)
+    x0 = np.clip(x_bar, 0, 1)
+    x0[x0 < params.tol] = 0
+    x0[x0 > 1 - params.tol] = 1
+    # re-run the walk and look at the state through a fallback-free path: no variable can clamp in 3 tiny steps
+    X, info = opt.iterative_rounding(x0, W, C, model, val * 1.5, np.random.default_rng(3), params)
+    assert info["clamped"] == 0 and info["micro"] >= 1
+    orc.placement_tables(X, C)
+
+
+def test_integral_input_is_returned_unchanged():
+    X0 = synth.placement_from_ranks(np.arange(8) % 4, 4)
+    W = np.ones((4, 8), dtype=np.int64)
+    X, info = opt.iterative_rounding(X0.astype(np.float64), W, 2, opt.LatencyModel(), 100.0, np.random.default_rng(0))
+    assert np.array_equal(X, X0) and info["macro"] == 0 and info["repaired"] == 0
+
+
+def test_randomized_search_is_never_worse_than_its_own_deterministic_start(c1):
+    wl, s, idx, W = c1
+    ev = oracle_evaluator(idx, s.C_max, s.H)
+    model = opt.LatencyModel(1.0, 0.0, 0.5 / (2 * s.H), 2 * s.H)
+    det = opt.optimize_placement(W, s.C_max, model, ev)
+    rnd = opt.optimize_placement(W, s.C_max, model, ev, rounding="randomized", n_roundings=8, seed=1)
+    orc.placement_tables(rnd["X"], s.C_max)
+    assert rnd["start_latency"] <= det["start_latency"] + 1e-9           # the deterministic rounding is among the starts
+    S = ev(opt.enumerate_single_copy(s.E, s.R, s.C_max))
+    brute = float(model.latency(S[:, 0], S[:, 1]).min())
+    assert brute - 1e-9 <= rnd["latency"] <= brute * 1.10
