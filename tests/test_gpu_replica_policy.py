@@ -118,3 +118,30 @@ def test_policy_argument_is_checked():
         case.layer.set_replica_policy(2)
     case.layer.set_replica_policy(1)
     case.layer.set_replica_policy(0)
+
+
+def test_front_end_call_honours_the_policy_for_small_and_large_batches():
+    """director_route_dispatch_cost under LOCAL_FIRST: decode-sized batches may not take the fused round-robin kernel."""
+    import torch
+    for seed, T in ((41, 100), (42, 700)):
+        shape, logits, x, weights = _custom(seed, T, 256, 20, 3, 128, 0, 5, 6, 1.2)
+        X = _random_placement(seed, 20, 5, 6, 8)
+        case = GpuCase(shape, logits, x, weights)
+        L = case.layer
+        L.set_placement(X)
+        L.set_replica_policy(LOCAL_FIRST)
+        try:
+            L.d.route_dispatch_cost(T, case.logits, case.x, L.topk_idx, L.topk_w, L.xp, L.row_token, L.inv_row,
+                                    L.dest_rank, L.seg_offsets, L.workload, L.rank_load, L.dispatch_tokens,
+                                    L.dispatch_bytes)
+            torch.cuda.synchronize()
+        finally:
+            L.set_replica_policy(0)
+        idx, _, _ = orc.route(logits, shape.K)
+        d = orc.dispatch(idx, X, 6, x, policy="local_first")
+        c = orc.placement_cost(idx, X, 6, shape.H, policy="local_first")
+        assert np.array_equal(L.inv_row[:T].cpu().numpy(), d["inv_row"])
+        assert np.array_equal(L.dest_rank[:T].cpu().numpy(), d["dest_rank"])
+        assert np.array_equal(L.seg_offsets.cpu().numpy(), d["seg_offsets"])
+        assert np.array_equal(L.dispatch_tokens.cpu().numpy(), c["dispatch_tokens"])
+        assert np.array_equal(L.rank_load.cpu().numpy(), c["rank_load"])
