@@ -18,12 +18,13 @@
 //   cost_kernel        same ranks -> destination rank; shared-memory histograms flushed with
 //                      integer atomics (order independent, hence deterministic).
 #include "director_common.cuh"
+#include "director_sort.cuh"
 
 namespace director {
 
-namespace {
+using namespace sort;
 
-constexpr int kTileWarps = kTokenTile / 32;
+namespace {
 
 // Lane bitmasks: mask[e][w] has bit l set iff token (tile*256 + w*32 + l) chose expert e.
 __device__ __forceinline__ void build_masks(uint32_t (*mask)[kTileWarps], const int32_t* __restrict__ topk_idx,
@@ -61,77 +62,19 @@ count_scan_kernel(const int32_t* __restrict__ topk_idx, int T, int E, int K, int
         for (int w = 0; w < kTileWarps; ++w) c += __popc(mask[e][w]);
         tile_counts[(size_t)tile * E + e] = c;
     }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1u) == (unsigned)(n_tiles - 1));
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
+    if (!last_cta_done(ticket, n_tiles, &is_last)) return;
 
     // ---- last CTA: per-expert exclusive scan over tiles, replica split, slot scan ----
     for (int g = threadIdx.x; g < G; g += blockDim.x) slot_len[g] = 0;
     __syncthreads();
     for (int e = threadIdx.x; e < E; e += blockDim.x) {
-        int run = 0;
-        // chunks of 16 tiles: all loads of a chunk are issued before the first store, so the loop runs at
-        // memory throughput instead of one L2 round trip per tile
-        for (int i0 = 0; i0 < n_tiles; i0 += 16) {
-            int c[16];
-#pragma unroll
-            for (int k = 0; k < 16; ++k) c[k] = (i0 + k < n_tiles) ? __ldcg(tile_counts + (size_t)(i0 + k) * E + e) : 0;
-#pragma unroll
-            for (int k = 0; k < 16; ++k) {
-                if (i0 + k < n_tiles) tile_counts[(size_t)(i0 + k) * E + e] = run;
-                run += c[k];
-            }
-        }
+        const int run = scan_column(tile_counts, n_tiles, E, e);
         const int r0 = rep_start[e], r_e = rep_start[e + 1] - r0;
         for (int q = 0; q < r_e; ++q)               // replica q gets ceil((N_e - q) / r_e) rows
             slot_len[rep_slot[r0 + q]] = (run > q) ? (run - q + r_e - 1) / r_e : 0;
     }
     __syncthreads();
-    // exclusive scan of slot_len[0..G): each thread owns a contiguous chunk
-    const int per = (G + blockDim.x - 1) / blockDim.x;
-    const int lo = min(threadIdx.x * per, G), hi = min(lo + per, G);
-    int local = 0;
-    for (int g = lo; g < hi; ++g) local += slot_len[g];
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    int incl = local;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    if (lane == 31) warp_sum[w] = incl;
-    __syncthreads();
-    int base = incl - local;
-    for (int i = 0; i < w; ++i) base += warp_sum[i];
-    for (int g = lo; g < hi; ++g) {
-        seg_offsets_a[g] = base;
-        if (seg_offsets_b) seg_offsets_b[g] = base;
-        base += slot_len[g];
-    }
-    if (threadIdx.x == blockDim.x - 1) {
-        // the last thread's running total is the grand total T*K (minus skipped bad indices)
-        seg_offsets_a[G] = base;
-        if (seg_offsets_b) seg_offsets_b[G] = base;
-        *ticket = 0u;                                 // ready for the next call on this stream
-    }
-}
-
-// Stable rank of (token, expert e) among the tile's tokens that chose e.
-__device__ __forceinline__ int tile_rank(const uint32_t (*mask)[kTileWarps], const uint16_t (*warp_prefix)[kTileWarps],
-                                         int e, int w, int lane) {
-    return warp_prefix[e][w] + __popc(mask[e][w] & ((1u << lane) - 1u));
-}
-
-__device__ __forceinline__ void build_warp_prefix(const uint32_t (*mask)[kTileWarps], uint16_t (*warp_prefix)[kTileWarps], int E) {
-    for (int e = threadIdx.x; e < E; e += blockDim.x) {
-        int run = 0;
-#pragma unroll
-        for (int w = 0; w < kTileWarps; ++w) { warp_prefix[e][w] = (uint16_t)run; run += __popc(mask[e][w]); }
-    }
-    __syncthreads();
+    scan_slots(slot_len, G, warp_sum, seg_offsets_a, seg_offsets_b, ticket);
 }
 
 __global__ void __launch_bounds__(kTokenTile)

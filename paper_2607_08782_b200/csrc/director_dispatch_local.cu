@@ -16,12 +16,15 @@
 //   local_index_kernel        row = seg_offsets[slot] + tile prefix + stable rank inside the tile.
 // All counts come from lane bitmasks and popcounts: integer only, order independent, deterministic.
 #include "director_common.cuh"
+#include "director_sort.cuh"
 
 namespace director {
 
+using namespace sort;
+
 namespace {
 
-constexpr int kW = kTokenTile / 32;   // warps per tile
+constexpr int kW = kTileWarps;   // warps per tile
 
 __device__ __forceinline__ int home_rank(const int32_t* __restrict__ src_rank, int t, int T, int R, int32_t* status) {
     int src = src_rank ? __ldg(src_rank + t) : (int)(((long long)t * R) / T);
@@ -56,33 +59,6 @@ __device__ __forceinline__ void build_travel_masks(uint32_t (*travel)[kW], const
     __syncthreads();
 }
 
-// In-place exclusive scan of column `col` of counts[n_tiles][ncol] over the tiles; returns the column total.
-// Chunks of 16 tiles: all loads of a chunk are issued before the first store.
-__device__ __forceinline__ int scan_column(int32_t* __restrict__ counts, int n_tiles, int ncol, int col) {
-    int run = 0;
-    for (int i0 = 0; i0 < n_tiles; i0 += 16) {
-        int c[16];
-#pragma unroll
-        for (int k = 0; k < 16; ++k) c[k] = (i0 + k < n_tiles) ? __ldcg(counts + (size_t)(i0 + k) * ncol + col) : 0;
-#pragma unroll
-        for (int k = 0; k < 16; ++k) {
-            if (i0 + k < n_tiles) counts[(size_t)(i0 + k) * ncol + col] = run;
-            run += c[k];
-        }
-    }
-    return run;
-}
-
-// true in exactly one CTA of the grid: the last one to get here (no spinning)
-__device__ __forceinline__ bool last_cta_done(unsigned int* ticket, int n_tiles, bool* flag) {
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) *flag = (atomicAdd(ticket, 1u) == (unsigned)(n_tiles - 1));
-    __syncthreads();
-    if (*flag) __threadfence();
-    return *flag;
-}
-
 __global__ void __launch_bounds__(kTokenTile)
 travel_count_scan_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ src_rank,
                          const unsigned long long* __restrict__ host_mask, int T, int E, int K, int R, int n_tiles,
@@ -115,18 +91,8 @@ __device__ __forceinline__ int replica_of(const uint32_t (*travel)[kW], const ui
         if ((hm >> src) & 1ull) return r0 + __popcll(hm & ((1ull << src) - 1ull));   // replicas are in ascending rank
     }
     const int r_e = __ldg(rep_start + e + 1) - r0;
-    const int m = __ldg(tile_travel + (size_t)tile * E + e) + travel_prefix[e][w] +
-                  __popc(travel[e][w] & ((1u << lane) - 1u));
+    const int m = __ldg(tile_travel + (size_t)tile * E + e) + tile_rank(travel, travel_prefix, e, w, lane);
     return r0 + m % r_e;
-}
-
-__device__ __forceinline__ void build_prefix(const uint32_t (*mask)[kW], uint16_t (*prefix)[kW], int n) {
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        int run = 0;
-#pragma unroll
-        for (int w = 0; w < kW; ++w) { prefix[i][w] = (uint16_t)run; run += __popc(mask[i][w]); }
-    }
-    __syncthreads();
 }
 
 // dynamic shared memory of slot_count_scan_kernel: travel[E][kW] u32 | rep[NR][kW] u32 | slot_len[G] i32 |
@@ -154,7 +120,7 @@ slot_count_scan_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __re
     const int tile = blockIdx.x;
     for (int i = threadIdx.x; i < NR * kW; i += blockDim.x) (&rep[0][0])[i] = 0u;
     build_travel_masks(travel, topk_idx, src_rank, host_mask, tile, T, E, K, R, status);
-    build_prefix(travel, travel_prefix, E);
+    build_warp_prefix(travel, travel_prefix, E);
     const int t = tile * kTokenTile + threadIdx.x;
     const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (t < T) {
@@ -185,30 +151,7 @@ slot_count_scan_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __re
     __syncthreads();
     for (int ri = threadIdx.x; ri < NR; ri += blockDim.x) slot_len[__ldg(rep_slot + ri)] = scan_column(tile_rep, n_tiles, NR, ri);
     __syncthreads();
-    const int per = (G + blockDim.x - 1) / blockDim.x;
-    const int lo = min((int)threadIdx.x * per, G), hi = min(lo + per, G);
-    int local = 0;
-    for (int g = lo; g < hi; ++g) local += slot_len[g];
-    int incl = local;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    if (lane == 31) warp_sum[w] = incl;
-    __syncthreads();
-    int base = incl - local;
-    for (int i = 0; i < w; ++i) base += warp_sum[i];
-    for (int g = lo; g < hi; ++g) {
-        seg_offsets_a[g] = base;
-        if (seg_offsets_b) seg_offsets_b[g] = base;
-        base += slot_len[g];
-    }
-    if (threadIdx.x == blockDim.x - 1) {
-        seg_offsets_a[G] = base;
-        if (seg_offsets_b) seg_offsets_b[G] = base;
-        *ticket = 0u;
-    }
+    scan_slots(slot_len, G, warp_sum, seg_offsets_a, seg_offsets_b, ticket);
 }
 
 // dynamic shared memory of local_index_kernel: rep[NR][kW] u32 | rep_prefix[NR][kW] u16
@@ -233,7 +176,7 @@ local_index_kernel(int T, int K, int NR, const int32_t* __restrict__ rep_slot, c
         if (ri[s] >= 0) atomicOr(&rep[ri[s]][w], 1u << lane);
     }
     __syncthreads();
-    build_prefix(rep, rep_prefix, NR);
+    build_warp_prefix(rep, rep_prefix, NR);
     if (t >= T) return;
 #pragma unroll
     for (int s = 0; s < kMaxK; ++s) {
@@ -241,7 +184,7 @@ local_index_kernel(int T, int K, int NR, const int32_t* __restrict__ rep_slot, c
         int row = -1;
         if (ri[s] >= 0) {
             row = __ldg(seg_offsets + __ldg(rep_slot + ri[s])) + __ldg(tile_rep + (size_t)tile * NR + ri[s]) +
-                  rep_prefix[ri[s]][w] + __popc(rep[ri[s]][w] & ((1u << lane) - 1u));
+                  tile_rank(rep, rep_prefix, ri[s], w, lane);
             row_token[row] = t;
         }
         inv_row[(size_t)t * K + s] = row;
@@ -265,7 +208,7 @@ local_cost_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restric
     for (int i = threadIdx.x; i < R * R; i += blockDim.x) h_rr[i] = 0u;
     for (int i = threadIdx.x; i < R; i += blockDim.x) h_load[i] = 0u;
     build_travel_masks(travel, topk_idx, src_rank, host_mask, tile, T, E, K, R, status);
-    build_prefix(travel, travel_prefix, E);
+    build_warp_prefix(travel, travel_prefix, E);
     const int t = tile * kTokenTile + threadIdx.x;
     if (t < T) {
         const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
