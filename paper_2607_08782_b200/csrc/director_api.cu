@@ -437,13 +437,12 @@ int director_layer_submit_host(director_ctx* ctx, int32_t T, const float* logits
         return DIRECTOR_ERR_CUDA;
     // the permuted rows are materialised once: the weight-stationary GEMM reads every token tile once per weight
     // block, so gathering inside it (director_expert_ffn_gather) repeats the gather 2F/256 times and measured slower
-    const bool fused = false;
-    int rc = launch_front(ctx, T, d_logits, d_x, ctx->e_topk_idx, ctx->e_topk_w, fused ? nullptr : ctx->e_xp,
+    int rc = launch_front(ctx, T, d_logits, d_x, ctx->e_topk_idx, ctx->e_topk_w, ctx->e_xp,
                           ctx->e_row_token, ctx->e_inv_row, ctx->e_dest_rank, ctx->d_seg_offsets, c_w, c_load, c_tok,
                           c_bytes, st);
     if (rc == DIRECTOR_OK)
-        rc = launch_expert_ffn(ctx, T, ctx->e_xp, fused ? ctx->e_row_token : nullptr, ctx->d_seg_offsets, w_gate, w_up,
-                               w_down, ctx->e_yp, (shared || fused) ? d_x : nullptr, ws_gate, ws_up, ws_down,
+        rc = launch_expert_ffn(ctx, T, ctx->e_xp, nullptr, ctx->d_seg_offsets, w_gate, w_up,
+                               w_down, ctx->e_yp, shared ? d_x : nullptr, ws_gate, ws_up, ws_down,
                                shared ? ctx->e_y_shared : nullptr, st);
     if (rc == DIRECTOR_OK)
         rc = launch_combine(ctx, T, ctx->e_yp, ctx->e_inv_row, ctx->e_topk_w, shared ? ctx->e_y_shared : nullptr, d_y, st);
