@@ -229,6 +229,19 @@ int director_dispatch_index_static(int32_t T, int32_t K, int32_t E, int32_t R, i
                                    int32_t* row_token, int32_t* inv_row, int32_t* dest_rank,
                                    int32_t* seg_offsets, int32_t* device_status, void* stream);
 
+/* The whole layer (a1)-(a5) in one call on device buffers: the gate, the permutation, the expert FFNs and the
+ * combine run on the context's own workspace (the intermediates of the stage calls are not exposed), the layer
+ * output and the placement-cost histograms go to the caller's buffers.  Same results, bit for bit, as the stage
+ * calls in order.  logits: dev fp32 [T,E].  x: dev bf16 [T,H].  Weights as for director_expert_ffn (ws_* may be
+ * NULL when S == 0).  y: dev bf16 [T,H].  workload: dev int64 [R,E].  rank_load: dev int64 [R].
+ * dispatch_tokens: dev int64 [R,R].  dispatch_bytes: dev uint64 [R,R].  Shares the workspace with the host entry
+ * points below: do not run both at the same time on one context. */
+int director_layer_forward(director_ctx* ctx, int32_t T, const float* logits, const void* x,
+                           const void* w_gate, const void* w_up, const void* w_down,
+                           const void* ws_gate, const void* ws_up, const void* ws_down, void* y,
+                           int64_t* workload, int64_t* rank_load, int64_t* dispatch_tokens,
+                           uint64_t* dispatch_bytes, void* stream);
+
 /* The whole layer for callers that hold their batch in host memory: copies logits and x to the
  * device, runs (a1)-(a5) on context-owned buffers and copies y and the histograms back; returns
  * when the results are in the host buffers (director_layer_submit_host + director_layer_wait_host).

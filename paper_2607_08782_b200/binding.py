@@ -25,7 +25,7 @@ EXPORTED = (
     "director_status_string", "director_dispatch_index_static", "director_layer_submit_host",
     "director_layer_wait_host", "director_set_ffn_variant", "director_placement_cost_batch",
     "director_expert_ffn_gather", "director_set_replica_policy", "director_dispatch_src",
-    "director_dedup_dispatch_tokens", "director_route_dispatch_cost",
+    "director_dedup_dispatch_tokens", "director_route_dispatch_cost", "director_layer_forward",
 )
 
 REPLICA_ROUND_ROBIN, REPLICA_LOCAL_FIRST = 0, 1
@@ -63,6 +63,7 @@ def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.director_combine.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp]
     lib.director_placement_cost.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp, vp]
     lib.director_layer_forward_host.argtypes = [vp, c_int32] + [vp] * 12
+    lib.director_layer_forward.argtypes = [vp, c_int32] + [vp] * 14
     lib.director_placement_cost_batch.argtypes = [vp, vp, c_int32, vp, vp, vp, vp, vp]
     lib.director_layer_submit_host.argtypes = [vp, c_int32] + [vp] * 13
     lib.director_layer_wait_host.argtypes = [vp, c_int64]
@@ -192,6 +193,14 @@ class Director:
         _check(self.lib.director_placement_cost_batch(self._ctx, _ptr(workload), n, _ptr(X), _ptr(rank_load),
                                                       _ptr(dispatch_tokens), _ptr(summary), _stream()),
                "director_placement_cost_batch")
+
+    def layer_forward(self, T, logits, x, w_gate, w_up, w_down, ws_gate, ws_up, ws_down, y, workload, rank_load,
+                      dispatch_tokens, dispatch_bytes):
+        """The whole layer on device tensors in one call (intermediates stay in the context's workspace)."""
+        _check(self.lib.director_layer_forward(self._ctx, T, _ptr(logits), _ptr(x), _ptr(w_gate), _ptr(w_up),
+                                               _ptr(w_down), _ptr(ws_gate), _ptr(ws_up), _ptr(ws_down), _ptr(y),
+                                               _ptr(workload), _ptr(rank_load), _ptr(dispatch_tokens),
+                                               _ptr(dispatch_bytes), _stream()), "director_layer_forward")
 
     def layer_forward_host(self, T, logits, x, w_gate, w_up, w_down, ws_gate, ws_up, ws_down, y,
                            rank_load=None, dispatch_bytes=None):

@@ -470,6 +470,42 @@ int director_layer_wait_host(director_ctx* ctx, int64_t ticket) {
     return cuda_status(cudaEventSynchronize(ctx->ev_d2h_done[ticket & 1]));
 }
 
+int director_layer_forward(director_ctx* ctx, int32_t T, const float* logits, const void* x, const void* w_gate,
+                           const void* w_up, const void* w_down, const void* ws_gate, const void* ws_up,
+                           const void* ws_down, void* y, int64_t* workload, int64_t* rank_load, int64_t* dispatch_tokens,
+                           uint64_t* dispatch_bytes, void* stream) {
+    REQUIRE_CTX(ctx);
+    REQUIRE_T(ctx, T);
+    REQUIRE_PLACEMENT(ctx);
+    REQUIRE_PTR(logits);
+    REQUIRE_PTR(x);
+    REQUIRE_PTR(w_gate);
+    REQUIRE_PTR(w_up);
+    REQUIRE_PTR(w_down);
+    REQUIRE_PTR(y);
+    const director_shape& s = ctx->shape;
+    const bool shared = s.S > 0;
+    if (shared) {
+        REQUIRE_PTR(ws_gate);
+        REQUIRE_PTR(ws_up);
+        REQUIRE_PTR(ws_down);
+    }
+    if (!workload || !rank_load || !dispatch_tokens || !dispatch_bytes) return DIRECTOR_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(workload) | reinterpret_cast<uintptr_t>(rank_load) |
+         reinterpret_cast<uintptr_t>(dispatch_tokens) | reinterpret_cast<uintptr_t>(dispatch_bytes)) & 7u)
+        return DIRECTOR_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    int rc = launch_front(ctx, T, logits, x, ctx->e_topk_idx, ctx->e_topk_w, ctx->e_xp, ctx->e_row_token,
+                          ctx->e_inv_row, ctx->e_dest_rank, ctx->d_seg_offsets, workload, rank_load, dispatch_tokens,
+                          dispatch_bytes, st);
+    if (rc == DIRECTOR_OK)
+        rc = launch_expert_ffn(ctx, T, ctx->e_xp, nullptr, ctx->d_seg_offsets, w_gate, w_up, w_down, ctx->e_yp,
+                               shared ? x : nullptr, ws_gate, ws_up, ws_down, shared ? ctx->e_y_shared : nullptr, st);
+    if (rc == DIRECTOR_OK)
+        rc = launch_combine(ctx, T, ctx->e_yp, ctx->e_inv_row, ctx->e_topk_w, shared ? ctx->e_y_shared : nullptr, y, st);
+    return rc;
+}
+
 int director_layer_forward_host(director_ctx* ctx, int32_t T, const float* logits, const void* x, const void* w_gate,
                                 const void* w_up, const void* w_down, const void* ws_gate, const void* ws_up,
                                 const void* ws_down, void* y, int64_t* rank_load, uint64_t* dispatch_bytes, void* stream) {

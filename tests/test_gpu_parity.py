@@ -455,3 +455,25 @@ def test_fused_front_end_matches_the_separate_stages_and_the_oracle(seed, T, H, 
                             o["seg"], o["W"], o["load"], o["dt"], o["db"])
     torch.cuda.synchronize()
     assert np.array_equal(o["inv_row"].cpu().numpy(), d["inv_row"])
+
+
+@pytest.mark.parametrize("seed,T,S", [(71, 900, 1), (72, 64, 0), (73, 2048, 2)])
+def test_one_call_layer_matches_the_stage_calls(seed, T, S):
+    """director_layer_forward: same bits as route / dispatch / expert_ffn / combine / placement_cost in order."""
+    import torch
+    from paper_2607_08782_b200.layer import tensor_to_bf16_bits
+    shape, logits, x, weights = _custom(seed, T, 256, 12, 3, 256, S, 4, 4, 1.2)
+    X = _random_placement(seed, 12, 4, 4, 3)
+    case = GpuCase(shape, logits, x, weights)
+    g = case.run(X)
+    L = case.layer
+    y = torch.zeros_like(L.y)
+    W, load = torch.zeros_like(L.workload), torch.zeros_like(L.rank_load)
+    dt, db = torch.zeros_like(L.dispatch_tokens), torch.zeros_like(L.dispatch_bytes)
+    L.d.layer_forward(T, case.logits, case.x, *L.w, *(L.ws if S > 0 else (None, None, None)), y, W, load, dt, db)
+    torch.cuda.synchronize()
+    assert L.d.last_status() == 0
+    assert np.array_equal(tensor_to_bf16_bits(y[:T]), g.y)
+    assert np.array_equal(W.cpu().numpy(), g.workload) and np.array_equal(load.cpu().numpy(), g.rank_load)
+    assert np.array_equal(dt.cpu().numpy(), g.dispatch_tokens)
+    assert np.array_equal(db.cpu().numpy().view(np.uint64), g.dispatch_bytes)
