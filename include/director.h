@@ -23,7 +23,7 @@
  *   - Every pointer marked "dev" is caller-owned device memory on the context's device,
  *     16-byte aligned, valid until the stream has reached the call.  "host" pointers are
  *     ordinary host memory.  The context owns only its internal workspace, sized at create
- *     time; no entry point allocates after director_create.
+ *     time; no entry point allocates after director_create (except director_reserve_placements).
  *   - bf16 tensors are passed as void* (raw 16-bit patterns), row-major, innermost last.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - Calls are asynchronous on `stream` and never synchronise unless stated.  Every function
@@ -75,6 +75,16 @@ int director_destroy(director_ctx* ctx);
  * otherwise, previous placement kept), builds the slot tables and uploads them on `stream`.
  * X_host may be reused as soon as the call returns. */
 int director_set_placement(director_ctx* ctx, const uint8_t* X_host, void* stream);
+
+/* Several placements on one context (the placement map P(l, i) of Section VI-A has one placement per layer l;
+ * a model's layers can share one context's workspace and differ only in their tables).
+ * director_reserve_placements makes room for n table sets (slots 0..n-1; slot 0 exists from creation; this is the
+ * one call besides director_create that allocates).  director_select_placement makes a slot the current one: a
+ * host-side switch, no copy, no stream work; kernels already launched keep the tables they were launched with.
+ * director_set_placement fills the current slot; every entry point uses the current slot.  Selecting a slot that
+ * was never filled leaves the context without a placement (DIRECTOR_ERR_PLACEMENT from the calls that need one). */
+int director_reserve_placements(director_ctx* ctx, int32_t n);
+int director_select_placement(director_ctx* ctx, int32_t slot);
 
 /* (a1) Gating (Section II-A: relevance scores, top-k selection, scores used as weights).
  * logits: dev fp32 [T,E].  topk_idx: dev int32 [T,K], the K experts with the largest logits in

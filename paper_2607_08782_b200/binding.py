@@ -26,6 +26,7 @@ EXPORTED = (
     "director_layer_wait_host", "director_set_ffn_variant", "director_placement_cost_batch",
     "director_expert_ffn_gather", "director_set_replica_policy", "director_dispatch_src",
     "director_dedup_dispatch_tokens", "director_route_dispatch_cost", "director_layer_forward",
+    "director_reserve_placements", "director_select_placement",
 )
 
 REPLICA_ROUND_ROBIN, REPLICA_LOCAL_FIRST = 0, 1
@@ -74,6 +75,8 @@ def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.director_set_profiling.argtypes = [vp, c_int32]
     lib.director_set_ffn_variant.argtypes = [vp, c_int32]
     lib.director_set_replica_policy.argtypes = [vp, c_int32]
+    lib.director_reserve_placements.argtypes = [vp, c_int32]
+    lib.director_select_placement.argtypes = [vp, c_int32]
     lib.director_route_dispatch_cost.argtypes = [vp, c_int32] + [vp] * 14
     lib.director_dispatch_src.argtypes = [vp, c_int32] + [vp] * 9
     lib.director_dedup_dispatch_tokens.argtypes = [vp, c_int32, vp, vp, vp, vp]
@@ -157,6 +160,12 @@ class Director:
         _check(self.lib.director_dispatch_src(self._ctx, T, _ptr(x), _ptr(topk_idx), _ptr(token_src_rank), _ptr(xp),
                                               _ptr(row_token), _ptr(inv_row), _ptr(dest_rank), _ptr(seg_offsets),
                                               _stream()), "director_dispatch_src")
+
+    def reserve_placements(self, n: int):
+        _check(self.lib.director_reserve_placements(self._ctx, n), "director_reserve_placements")
+
+    def select_placement(self, slot: int):
+        _check(self.lib.director_select_placement(self._ctx, slot), "director_select_placement")
 
     def set_replica_policy(self, policy: int):
         _check(self.lib.director_set_replica_policy(self._ctx, policy), "director_set_replica_policy")

@@ -31,8 +31,14 @@ bool shape_supported(const director_shape& s) {
 }
 
 void free_all(director_ctx* c) {
-    void* ptrs[] = {c->d_rep_start, c->d_rep_slot, c->d_slot_expert, c->d_tile_counts, c->d_seg_offsets, c->d_ticket,
-                    c->d_host_mask, c->d_tile_rep,
+    if (c->bank.empty())        // creation failed before the bank took ownership of the first table set
+        c->bank.push_back({c->d_rep_start, c->d_rep_slot, c->d_slot_expert, c->d_host_mask, 0, false});
+    for (auto& t : c->bank) {
+        void* tables[] = {t.rep_start, t.rep_slot, t.slot_expert, t.host_mask};
+        for (void* p : tables)
+            if (p) cudaFree(p);
+    }
+    void* ptrs[] = {c->d_tile_counts, c->d_seg_offsets, c->d_ticket, c->d_tile_rep,
                     c->d_status, c->d_hidden, c->d_hidden_shared, c->d_one_seg, c->d_sched,
                     c->d_zero_expert, c->e_logits2[0], c->e_logits2[1], c->e_x2[0], c->e_x2[1], c->e_topk_idx,
                     c->e_topk_w, c->e_xp, c->e_yp, c->e_y2[0], c->e_y2[1], c->e_y_shared, c->e_row_token, c->e_inv_row,
@@ -137,6 +143,7 @@ int director_create(const director_shape* shape, director_ctx** out) {
         delete c;
         return DIRECTOR_ERR_WORKSPACE;
     }
+    c->bank.push_back({c->d_rep_start, c->d_rep_slot, c->d_slot_expert, c->d_host_mask, 0, false});
     ok = cudaMemset(c->d_ticket, 0, sizeof(unsigned int)) == cudaSuccess &&
          cudaMemset(c->d_status, 0, sizeof(int32_t)) == cudaSuccess &&
          cudaMemset(c->d_zero_expert, 0, sizeof(int32_t)) == cudaSuccess;
@@ -215,8 +222,44 @@ int director_set_placement(director_ctx* ctx, const uint8_t* X, void* stream) {
         cudaMemcpyAsync(ctx->d_host_mask, host_mask.data(), host_mask.size() * 8, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return DIRECTOR_ERR_CUDA;
     ctx->n_replicas = rep_start[E];
-    ctx->h_slot_expert = slot_expert;
     ctx->placement_set = true;
+    ctx->bank[ctx->active_placement].n_replicas = ctx->n_replicas;
+    ctx->bank[ctx->active_placement].set = true;
+    return DIRECTOR_OK;
+}
+
+int director_reserve_placements(director_ctx* ctx, int32_t n) {
+    REQUIRE_CTX(ctx);
+    if (n < 1 || n > 65536) return DIRECTOR_ERR_INVALID_ARG;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    const director_shape& s = ctx->shape;
+    while ((int)ctx->bank.size() < n) {
+        director_ctx::PlacementTables t{nullptr, nullptr, nullptr, nullptr, 0, false};
+        const bool ok = dev_alloc(&t.rep_start, s.E + 1) && dev_alloc(&t.rep_slot, (size_t)s.E * s.R) &&
+                        dev_alloc(&t.slot_expert, ctx->G) && dev_alloc(&t.host_mask, s.E);
+        if (!ok) {
+            cudaGetLastError();
+            void* tables[] = {t.rep_start, t.rep_slot, t.slot_expert, t.host_mask};
+            for (void* p : tables)
+                if (p) cudaFree(p);
+            return DIRECTOR_ERR_WORKSPACE;
+        }
+        ctx->bank.push_back(t);
+    }
+    return DIRECTOR_OK;
+}
+
+int director_select_placement(director_ctx* ctx, int32_t slot) {
+    REQUIRE_CTX(ctx);
+    if (slot < 0 || slot >= (int)ctx->bank.size()) return DIRECTOR_ERR_INVALID_ARG;
+    const auto& t = ctx->bank[slot];
+    ctx->d_rep_start = t.rep_start;
+    ctx->d_rep_slot = t.rep_slot;
+    ctx->d_slot_expert = t.slot_expert;
+    ctx->d_host_mask = t.host_mask;
+    ctx->n_replicas = t.n_replicas;
+    ctx->placement_set = t.set;
+    ctx->active_placement = slot;
     return DIRECTOR_OK;
 }
 

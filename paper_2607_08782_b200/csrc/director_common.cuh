@@ -38,7 +38,18 @@ struct director_ctx {
     int32_t* d_rep_start = nullptr;    // [E+1]
     int32_t* d_rep_slot = nullptr;     // [E*R] slot id of each replica, replicas by ascending rank
     int32_t* d_slot_expert = nullptr;  // [G] expert of each slot or -1
-    std::vector<int32_t> h_slot_expert;
+    // Placement bank: table sets for several placements (one per layer of a model, say) that share this context's
+    // workspace.  The d_* pointers above always alias the selected set; set 0 is allocated with the context.
+    struct PlacementTables {
+        int32_t* rep_start;
+        int32_t* rep_slot;
+        int32_t* slot_expert;
+        unsigned long long* host_mask;
+        int n_replicas;
+        bool set;
+    };
+    std::vector<PlacementTables> bank;
+    int active_placement = 0;
     unsigned long long* d_host_mask = nullptr;   // [E] bit j set iff rank j hosts the expert
     int n_replicas = 0;                // rep_start[E]: hosted (expert, rank) pairs of the current placement
     int replica_policy = 0;            // DIRECTOR_REPLICA_*: which replica an assignment uses

@@ -477,3 +477,42 @@ def test_one_call_layer_matches_the_stage_calls(seed, T, S):
     assert np.array_equal(W.cpu().numpy(), g.workload) and np.array_equal(load.cpu().numpy(), g.rank_load)
     assert np.array_equal(dt.cpu().numpy(), g.dispatch_tokens)
     assert np.array_equal(db.cpu().numpy().view(np.uint64), g.dispatch_bytes)
+
+
+def test_placement_bank_switches_between_layers_placements():
+    """Three placements kept on one context: selecting a slot gives the same bits as re-sending that placement."""
+    import torch
+    from paper_2607_08782_b200.binding import DirectorError
+    shape, logits, x, weights = _custom(81, 700, 256, 16, 2, 128, 0, 4, 6, 1.2)
+    case = GpuCase(shape, logits, x, weights)
+    L, d = case.layer, case.layer.d
+    Xs = [_random_placement(810 + i, 16, 4, 6, 3 * i) for i in range(3)]
+    ref = [case.run(X) for X in Xs]                       # slot 0, placement re-sent each time
+    d.reserve_placements(3)
+    d.reserve_placements(2)                                # shrinking is a no-op
+    for slot, X in enumerate(Xs):
+        d.select_placement(slot)
+        d.set_placement(X)
+    for rounds in range(2):
+        for slot in (2, 0, 1):
+            d.select_placement(slot)
+            L.route(shape.T, case.logits)
+            L.dispatch(shape.T, case.x)
+            L.expert_ffn(shape.T, case.x)
+            L.combine(shape.T)
+            L.placement_cost(shape.T)
+            torch.cuda.synchronize()
+            g = ref[slot]
+            assert np.array_equal(L.inv_row[:shape.T].cpu().numpy(), g.inv_row)
+            assert np.array_equal(L.seg_offsets.cpu().numpy(), g.seg_offsets)
+            assert np.array_equal(L.dispatch_tokens.cpu().numpy(), g.dispatch_tokens)
+            from paper_2607_08782_b200.layer import tensor_to_bf16_bits
+            assert np.array_equal(tensor_to_bf16_bits(L.y[:shape.T]), g.y)
+    with pytest.raises(DirectorError):
+        d.select_placement(3)
+    d.reserve_placements(4)
+    d.select_placement(3)                                  # reserved but never filled: no placement
+    with pytest.raises(DirectorError):
+        L.dispatch(shape.T, case.x)
+    d.select_placement(0)
+    assert d.last_status() == 0
