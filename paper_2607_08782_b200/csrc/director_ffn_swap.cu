@@ -95,7 +95,8 @@ __device__ __forceinline__ bool mbar_wait_acquire_cluster(uint32_t bar, uint32_t
     return true;
 }
 
-constexpr int SCHED_SLOTS = 4;      // ring through which the leader's producer hands work items to the other roles
+constexpr int SCHED_SLOTS = 4;      // ring through which the scheduler thread hands work items to the other roles
+constexpr int SCHED_AHEAD = 1;      // items the scheduler may claim beyond the one after the producer's current item
 
 struct SwapParams {
     const int32_t* seg_offsets;
@@ -145,7 +146,7 @@ struct SwapWalker {
 // input x through row_token - tm_x then describes x with a one-row box and the whole producer warp issues the
 // loads, four rows per lane - so the dispatch step needs no row copies at all.
 template <int MODE, int EPI_GROUPS, bool GATHER, int S_STAGES>
-__global__ void __launch_bounds__(64 + 128 * EPI_GROUPS, 1)
+__global__ void __launch_bounds__(96 + 128 * EPI_GROUPS, 1)
 grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
                          const SwapParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -153,11 +154,12 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     uint8_t* gen = smem_raw + (tiles - raw) + S_STAGES * S_STAGE_BYTES;
     uint64_t* bars = reinterpret_cast<uint64_t*>(gen);             // full[8] empty[8] tfull[2] tempty[2]
-    // sched_full[4] at +160, sched_empty[4] at +192 (the leader's are the ones used)
+    // sched_full[4] at +160, sched_empty[4] at +192 (sched_empty: the scheduler CTA's are the ones used)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + 224);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + 228);
     volatile int* sched_item = reinterpret_cast<volatile int*>(gen + 232);   // [4]
-    int32_t* warp_sum = reinterpret_cast<int32_t*>(gen + 248);     // [10]
+    int32_t* warp_sum = reinterpret_cast<int32_t*>(gen + 248);     // [11]
+    volatile int* prod_taken = reinterpret_cast<volatile int*>(gen + 292);   // items the scheduler CTA's producer has taken
     const int G = p.G;
     int32_t* s_seg = reinterpret_cast<int32_t*>(gen + S_HEADER_BYTES);
     int32_t* s_tt = s_seg + (G + 1);
@@ -175,15 +177,16 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     const uint32_t rank = cluster_ctarank();
     const bool leader = rank == 0;
 
-    constexpr int n_threads = 64 + 128 * EPI_GROUPS;               // producer warp + MMA warp + epilogue warps
+    constexpr int n_threads = 96 + 128 * EPI_GROUPS;               // producer, MMA and scheduler warps + epilogue warps
     for (int g = threadIdx.x; g <= G; g += n_threads) s_seg[g] = __ldg(p.seg_offsets + g);
     for (int g = threadIdx.x; g < G; g += n_threads) s_exp[g] = (int16_t)__ldg(p.slot_expert + g);
     if (threadIdx.x == 0) {
         *abort_flag = 0;
+        *prod_taken = 0;
         for (int s = 0; s < S_STAGES; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8 * EPI_GROUPS); }
-        // a slot is free again once every consumer has read it: MMA thread, peer producer, all epilogue warps
-        for (int q = 0; q < SCHED_SLOTS; ++q) { mbar_init(sched_full(q), 1); mbar_init(sched_empty(q), 2 + 8 * EPI_GROUPS); }
+        // a slot is free again once every reader has read it: MMA thread, both producers, all epilogue warps
+        for (int q = 0; q < SCHED_SLOTS; ++q) { mbar_init(sched_full(q), 1); mbar_init(sched_empty(q), 3 + 8 * EPI_GROUPS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -225,65 +228,42 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     SwapTile t;
 
     // Work items (segment, weight block, token tile) are handed out dynamically, in their natural order, from a
-    // global counter: the leader's producer claims the next item whenever it is ready for one (it claims one
-    // ahead, so the atomic's latency hides behind the current item's loads) and publishes it through a small ring
-    // in both CTAs' shared memory.  Tail tiles are cheaper than full ones, so fixed assignments leave 6-15 % of
-    // imbalance between clusters; and since the items are still taken in order, clusters running at the same
-    // time keep working on neighbouring items and share their weight tiles in L2.
+    // global counter.  A scheduler thread - lane 0 of a warp of its own in the leader CTA, next to the MMA thread that
+    // reads its ring most urgently - claims items and publishes them through a small ring in both CTAs' shared
+    // memory; every other role (both producers, the MMA thread, all epilogue warps) reads the ring.  Claiming and publishing take ~2000 cycles per item (a global atomic, a remote
+    // store and a remote arrive with cluster-scope release); on a thread of its own that latency is off the load
+    // path.  Tail tiles are cheaper than full ones, so fixed assignments leave 6-15 % of imbalance between clusters;
+    // and since the items are still taken in order, clusters running at the same time keep working on neighbouring
+    // items and share their weight tiles in L2.
     const int total_items = walker.total;
+    constexpr uint32_t SCHED_RANK = 0;                             // CTA of the pair that owns the ring's barriers
+    const bool sched_local = rank == SCHED_RANK;
     // consumer side of the ring: wait for item i, read it, hand the slot back
     auto take_item = [&](int i, int& w) -> bool {
         const int q = i & (SCHED_SLOTS - 1);
         const uint32_t par = ((uint32_t)i / SCHED_SLOTS) & 1u;
-        const bool ok = leader ? mbar_wait(sched_full(q), par, abort_flag)
-                               : mbar_wait_acquire_cluster(sched_full(q), par, abort_flag);
+        const bool ok = sched_local ? mbar_wait(sched_full(q), par, abort_flag)
+                                    : mbar_wait_acquire_cluster(sched_full(q), par, abort_flag);
         if (ok) w = sched_item[q];
         return ok;
     };
     auto release_item = [&](int i) {
         const int q = i & (SCHED_SLOTS - 1);
-        if (leader) mbar_arrive(sched_empty(q));
-        else mbar_arrive_cluster(map_to_cta(sched_empty(q), 0));
+        if (sched_local) mbar_arrive(sched_empty(q));
+        else mbar_arrive_cluster(map_to_cta(sched_empty(q), SCHED_RANK));
     };
 
     if (warp == 0 && GATHER) {
-        // whole warp: lane 0 schedules and loads the weight tile, every lane gathers four token rows per k-step
+        // whole warp: lane 0 loads the weight tile, every lane gathers four token rows per k-step
         int stage = 0;
         uint32_t phase = 0;
         int ok = 1;
-        auto publish = [&](int i, int w) -> bool {
-            const int q = i & (SCHED_SLOTS - 1);
-            if (!mbar_wait(sched_empty(q), (((uint32_t)i / SCHED_SLOTS) & 1u) ^ 1u, abort_flag)) return false;
-            sched_item[q] = w;
-            st_cluster_u32(map_to_cta(smem_u32(const_cast<int*>(&sched_item[q])), 1), (uint32_t)w);
-            mbar_arrive(sched_full(q));
-            mbar_arrive_cluster_release(map_to_cta(sched_full(q), 1));
-            return true;
-        };
-        auto clamp_item = [&](unsigned int c) { return c < (unsigned)total_items ? (int)c : total_items; };
-        int w_cur = total_items;
-        unsigned int claim_ahead = 0u;
-        if (lane == 0 && leader) {
-            w_cur = clamp_item(atomicAdd(p.counter, 1u));
-            claim_ahead = w_cur < total_items ? atomicAdd(p.counter, 1u) : (unsigned)total_items;
-            ok = publish(0, w_cur) ? 1 : 0;
-        }
-        ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
         for (int i = 0; ok; ++i) {
             int w = 0;
             if (lane == 0) {
-                if (leader) {
-                    w = w_cur;
-                    if (w < total_items) {
-                        const int w_next = clamp_item(claim_ahead);
-                        ok = publish(i + 1, w_next) ? 1 : 0;
-                        if (ok && w_next < total_items) claim_ahead = atomicAdd(p.counter, 1u);
-                        w_cur = w_next;
-                    }
-                } else {
-                    ok = take_item(i, w) ? 1 : 0;
-                    if (ok) release_item(i);
-                }
+                ok = take_item(i, w) ? 1 : 0;
+                if (ok) release_item(i);
+                if (ok && sched_local) *prod_taken = i + 1;
             }
             ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
             w = __shfl_sync(0xFFFFFFFFu, w, 0);
@@ -323,39 +303,11 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            // leader: item i+1 is published (and item i+2 claimed) when item i starts, so neither the atomic's
-            // latency nor the trip to the peer's shared memory ever sits in front of a load
-            auto publish = [&](int i, int w) -> bool {
-                const int q = i & (SCHED_SLOTS - 1);
-                if (!mbar_wait(sched_empty(q), (((uint32_t)i / SCHED_SLOTS) & 1u) ^ 1u, abort_flag)) return false;
-                sched_item[q] = w;
-                st_cluster_u32(map_to_cta(smem_u32(const_cast<int*>(&sched_item[q])), 1), (uint32_t)w);
-                mbar_arrive(sched_full(q));
-                mbar_arrive_cluster_release(map_to_cta(sched_full(q), 1));
-                return true;
-            };
-            auto clamp_item = [&](unsigned int c) { return c < (unsigned)total_items ? (int)c : total_items; };
-            int w_cur = total_items;
-            unsigned int claim_ahead = 0u;
-            if (leader) {
-                w_cur = clamp_item(atomicAdd(p.counter, 1u));
-                claim_ahead = w_cur < total_items ? atomicAdd(p.counter, 1u) : (unsigned)total_items;
-                ok = publish(0, w_cur);
-            }
             for (int i = 0; ok; ++i) {
                 int w;
-                if (leader) {
-                    w = w_cur;
-                    if (w < total_items) {
-                        const int w_next = clamp_item(claim_ahead);
-                        if (!(ok = publish(i + 1, w_next))) break;
-                        if (w_next < total_items) claim_ahead = atomicAdd(p.counter, 1u);
-                        w_cur = w_next;
-                    }
-                } else {
-                    if (!(ok = take_item(i, w))) break;
-                    release_item(i);
-                }
+                if (!(ok = take_item(i, w))) break;
+                release_item(i);
+                if (sched_local) *prod_taken = i + 1;
                 if (w >= total_items) break;
                 walker.get(w, t);
                 const int x_row = t.row0 + (int)rank * (t.n >> 1);          // this CTA's half of the tile's tokens
@@ -402,9 +354,38 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 if (ok) umma_commit_both(tfull_bar(acc));
             }
         }
+    } else if (warp == 2) {
+        if (lane == 0 && rank == SCHED_RANK) {
+            // scheduler: claim the next item, wait until every reader is done with the slot's previous item, write
+            // the item into both CTAs' rings, signal both.  The item past the end is published once: it ends every
+            // role's loop.
+            for (int i = 0;; ++i) {
+                // stay SCHED_AHEAD items ahead of this CTA's producer, no more: items held back by a cluster that is
+                // not ready for them are imbalance at the end of the kernel
+                if (i > *prod_taken + SCHED_AHEAD) {
+                    const unsigned long long t0 = global_ns();
+                    uint32_t n = 0;
+                    bool give_up = false;
+                    while (i > *prod_taken + SCHED_AHEAD) {
+                        __nanosleep(256);            // an item lasts microseconds: poll gently, this SM has an epilogue to run
+                        if ((++n & 63u) == 0u && (*abort_flag || global_ns() - t0 > WAIT_LIMIT_NS)) { give_up = true; break; }
+                    }
+                    if (give_up) { *abort_flag = 1; break; }
+                }
+                const unsigned int c = atomicAdd(p.counter, 1u);
+                const int w = c < (unsigned)total_items ? (int)c : total_items;
+                const int q = i & (SCHED_SLOTS - 1);
+                if (!mbar_wait(sched_empty(q), (((uint32_t)i / SCHED_SLOTS) & 1u) ^ 1u, abort_flag)) break;
+                sched_item[q] = w;
+                st_cluster_u32(map_to_cta(smem_u32(const_cast<int*>(&sched_item[q])), 1u - SCHED_RANK), (uint32_t)w);
+                mbar_arrive(sched_full(q));
+                mbar_arrive_cluster_release(map_to_cta(sched_full(q), 1u - SCHED_RANK));
+                if (w >= total_items) break;
+            }
+        }
     } else {
         const int quad = warp & 3;                                 // TMEM lane quadrant this warp may read
-        const int cgroup = EPI_GROUPS == 1 ? 0 : (warp - 2) >> 2;  // which of the 32-token chunks this warp takes
+        const int cgroup = EPI_GROUPS == 1 ? 0 : (warp - 3) >> 2;  // which of the 32-token chunks this warp takes
         constexpr int CSTEP = 32 * EPI_GROUPS;
         const int c_first = 32 * cgroup;
         uint16_t* out = static_cast<uint16_t*>(p.out);
@@ -517,7 +498,7 @@ int launch_swap_n(director_ctx* ctx, const char* name, const CUtensorMap& w, con
                   cudaStream_t st) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * ctx->pair_clusters));
-    cfg.blockDim = dim3(64 + 128 * EPI_GROUPS);
+    cfg.blockDim = dim3(96 + 128 * EPI_GROUPS);
     cfg.dynamicSmemBytes = (size_t)swap_smem_bytes(STAGES, p.G);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
