@@ -31,7 +31,7 @@ using namespace umma;
 namespace {
 
 constexpr int S_STAGE_BYTES = A_BYTES + B_HALF_BYTES;          // 16 KB weights + 16 KB tokens per CTA per k-step
-constexpr int S_HEADER_BYTES = 320;                            // barriers, scheduler ring, TMEM slot, scratch
+constexpr int S_HEADER_BYTES = 384;                            // barriers, scheduler ring, TMEM slot, scratch
 constexpr int S_MAX_SMEM = 232448;                             // opt-in shared memory per CTA on sm_100
 // Shared memory of a launch: alignment slack, the operand ring, the header, and the segment tables of its G slots
 // (seg_offsets and token-tile prefix as int32, expert ids as int16).
@@ -66,8 +66,9 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(cluster_bar), "r"(x), "r"(y), "r"(z) : "memory");
 }
 
-__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
-    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+__device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, int4 v) {
+    asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
 }
 // remote arrive that publishes this thread's earlier (remote) stores to the waiting CTA
 __device__ __forceinline__ void mbar_arrive_cluster_release(uint32_t cluster_bar) {
@@ -157,7 +158,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     // sched_full[4] at +160, sched_empty[4] at +192 (sched_empty: the scheduler CTA's are the ones used)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + 224);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + 228);
-    volatile int* sched_item = reinterpret_cast<volatile int*>(gen + 232);   // [4]
+    int4* sched_item = reinterpret_cast<int4*>(gen + 304);         // [4] decoded work items {row0, valid, w_row, wb}
     int32_t* warp_sum = reinterpret_cast<int32_t*>(gen + 248);     // [11]
     volatile int* prod_taken = reinterpret_cast<volatile int*>(gen + 292);   // items the scheduler CTA's producer has taken
     const int G = p.G;
@@ -230,7 +231,8 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     // Work items (segment, weight block, token tile) are handed out dynamically, in their natural order, from a
     // global counter.  A scheduler thread - lane 0 of a warp of its own in the leader CTA, next to the MMA thread that
     // reads its ring most urgently - claims items and publishes them through a small ring in both CTAs' shared
-    // memory; every other role (both producers, the MMA thread, all epilogue warps) reads the ring.  Claiming and publishing take ~2000 cycles per item (a global atomic, a remote
+    // memory, already decoded into tile coordinates; every other role (both producers, the MMA thread, all epilogue
+    // warps) reads the ring.  Claiming and publishing take ~2000 cycles per item (a global atomic, a remote
     // store and a remote arrive with cluster-scope release); on a thread of its own that latency is off the load
     // path.  Tail tiles are cheaper than full ones, so fixed assignments leave 6-15 % of imbalance between clusters;
     // and since the items are still taken in order, clusters running at the same time keep working on neighbouring
@@ -239,12 +241,20 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     constexpr uint32_t SCHED_RANK = 0;                             // CTA of the pair that owns the ring's barriers
     const bool sched_local = rank == SCHED_RANK;
     // consumer side of the ring: wait for item i, read it, hand the slot back
-    auto take_item = [&](int i, int& w) -> bool {
+    // (valid == 0 marks the item past the end)
+    auto take_item = [&](int i, SwapTile& tile) -> bool {
         const int q = i & (SCHED_SLOTS - 1);
         const uint32_t par = ((uint32_t)i / SCHED_SLOTS) & 1u;
         const bool ok = sched_local ? mbar_wait(sched_full(q), par, abort_flag)
                                     : mbar_wait_acquire_cluster(sched_full(q), par, abort_flag);
-        if (ok) w = sched_item[q];
+        if (ok) {
+            const int4 v = sched_item[q];
+            tile.row0 = v.x;
+            tile.valid = v.y;
+            tile.n = (v.y + TOKEN_STEP - 1) / TOKEN_STEP * TOKEN_STEP;
+            tile.w_row = v.z;
+            tile.wb = v.w;
+        }
         return ok;
     };
     auto release_item = [&](int i) {
@@ -259,16 +269,18 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
         uint32_t phase = 0;
         int ok = 1;
         for (int i = 0; ok; ++i) {
-            int w = 0;
             if (lane == 0) {
-                ok = take_item(i, w) ? 1 : 0;
+                ok = take_item(i, t) ? 1 : 0;
                 if (ok) release_item(i);
                 if (ok && sched_local) *prod_taken = i + 1;
             }
             ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-            w = __shfl_sync(0xFFFFFFFFu, w, 0);
-            if (!ok || w >= total_items) break;
-            walker.get(w, t);
+            t.row0 = __shfl_sync(0xFFFFFFFFu, t.row0, 0);
+            t.valid = __shfl_sync(0xFFFFFFFFu, t.valid, 0);
+            t.n = __shfl_sync(0xFFFFFFFFu, t.n, 0);
+            t.w_row = __shfl_sync(0xFFFFFFFFu, t.w_row, 0);
+            t.wb = __shfl_sync(0xFFFFFFFFu, t.wb, 0);
+            if (!ok || t.valid == 0) break;
             const int half = t.n >> 1;                                  // token rows this CTA supplies (multiple of 16)
             const int x_row = t.row0 + (int)rank * half;
             const int w_row = t.w_row + (int)rank * (ROWS_PER_BLOCK / 2);
@@ -304,12 +316,10 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
             uint32_t phase = 0;
             bool ok = true;
             for (int i = 0; ok; ++i) {
-                int w;
-                if (!(ok = take_item(i, w))) break;
+                if (!(ok = take_item(i, t))) break;
                 release_item(i);
                 if (sched_local) *prod_taken = i + 1;
-                if (w >= total_items) break;
-                walker.get(w, t);
+                if (t.valid == 0) break;
                 const int x_row = t.row0 + (int)rank * (t.n >> 1);          // this CTA's half of the tile's tokens
                 const int w_row = t.w_row + (int)rank * (ROWS_PER_BLOCK / 2);
                 for (int kb = 0; kb < p.k_steps; ++kb) {
@@ -330,11 +340,9 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
             uint32_t phase = 0;
             bool ok = true;
             for (int it = 0; ok; ++it) {
-                int w;
-                if (!(ok = take_item(it, w))) break;
+                if (!(ok = take_item(it, t))) break;
                 release_item(it);
-                if (w >= total_items) break;
-                walker.get(w, t);
+                if (t.valid == 0) break;
                 const int acc = it & 1;
                 if (!(ok = mbar_wait(tempty_bar(acc), (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag))) break;
                 tc_fence_after();
@@ -376,8 +384,13 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 const int w = c < (unsigned)total_items ? (int)c : total_items;
                 const int q = i & (SCHED_SLOTS - 1);
                 if (!mbar_wait(sched_empty(q), (((uint32_t)i / SCHED_SLOTS) & 1u) ^ 1u, abort_flag)) break;
-                sched_item[q] = w;
-                st_cluster_u32(map_to_cta(smem_u32(const_cast<int*>(&sched_item[q])), 1u - SCHED_RANK), (uint32_t)w);
+                int4 item = make_int4(0, 0, 0, 0);
+                if (w < total_items) {
+                    walker.get(w, t);
+                    item = make_int4(t.row0, t.valid, t.w_row, t.wb);
+                }
+                sched_item[q] = item;
+                st_cluster_v4(map_to_cta(smem_u32(&sched_item[q]), 1u - SCHED_RANK), item);
                 mbar_arrive(sched_full(q));
                 mbar_arrive_cluster_release(map_to_cta(sched_full(q), 1u - SCHED_RANK));
                 if (w >= total_items) break;
@@ -392,12 +405,10 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
         const int lane_row = quad * 32 + lane;                     // weight row of this thread inside the CTA's 128
         bool ok = true;
         for (int it = 0; ok; ++it) {
-            int w;
-            if (!(ok = take_item(it, w))) break;
+            if (!(ok = take_item(it, t))) break;
             __syncwarp();
             if (lane == 0) release_item(it);
-            if (w >= total_items) break;
-            walker.get(w, t);
+            if (t.valid == 0) break;
             const int acc = it & 1;
             if (!(ok = mbar_wait(tfull_bar(acc), ((uint32_t)it >> 1) & 1u, abort_flag))) break;
             tc_fence_after();
