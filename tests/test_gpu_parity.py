@@ -79,8 +79,8 @@ def _random_placement(seed, E, R, C, extra):
     (14, 1, 256, 8, 2, 128, 1, 4, 2, 0),         # a single token
     (15, 513, 768, 128, 8, 256, 0, 16, 9, 16),   # Qwen3-like routing sizes, many empty segments
     (16, 260, 256, 256, 8, 128, 0, 64, 4, 0),    # the largest supported E and R
-    (17, 300, 256, 40, 4, 128, 0, 19, 9, 5),     # 171 slots: the most for which the GEMM's operand ring has 7 stages
-    (18, 300, 256, 40, 4, 128, 0, 43, 4, 5),     # 172 slots: the first size with 6 stages
+    (17, 300, 256, 40, 4, 128, 0, 41, 4, 5),     # 164 slots: the most for which the GEMM's operand ring has 7 stages
+    (18, 300, 256, 40, 4, 128, 0, 33, 5, 5),     # 165 slots: the first size with 6 stages
     (19, 300, 256, 40, 4, 128, 2, 64, 16, 200),  # 1024 slots: the largest segment table
 ])
 def test_small_cases_full_tensor_parity(seed, T, H, E, K, F, S, R, C, extra):
