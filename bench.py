@@ -279,6 +279,8 @@ def run_reference(args):
 # main (CUDA arm)
 # ------------------------------------------------------------------------------------------------
 
+DOMINANT_KERNEL = "grouped_gemm_swiglu_kernel"      # the gate||up grouped GEMM: ~63 % of a step
+
 STAGE_KERNELS = {
     "route": ["route_topk_kernel", "front_small_kernel"],   # the fused front end (T <= 256) is booked under route
     "dispatch": ["dispatch_count_scan_kernel", "dispatch_index_kernel", "dispatch_scatter_rows_kernel",
@@ -490,7 +492,9 @@ def main():
         graph = layer.capture(T, logits, x, fused=args.fused)
         launches_per_pass = (layer.d.launch_count() - n_c) // 2      # capture() runs the pass twice (warm-up + record)
     else:
-        layer.d.set_profiling(True)
+        # inside the timed region only the dominant kernel is bracketed by events (its live duration is what the
+        # roofline object needs); the other kernels are timed in a pass of their own afterwards
+        layer.d.set_profiling(True, only=DOMINANT_KERNEL)
     n0 = layer.d.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     wall0 = time.time()
@@ -510,11 +514,22 @@ def main():
     ms_total = ev0.elapsed_time(ev1)
     clocks = sampler.stop(wall0, wall1) if sampler else {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
     kernel_ms = {}
-    for names in STAGE_KERNELS.values():
-        for k in names:
-            ms, n = layer.d.kernel_time(k)
-            if n:
-                kernel_ms[k] = (ms / n, n // args.steps)
+    if graph is None:
+        ms, n = layer.d.kernel_time(DOMINANT_KERNEL)
+        dominant = (ms / n, n // args.steps) if n else None
+        # every kernel, in an extra pass outside the timed region (same steps, events around every launch)
+        extra = min(args.steps, 100)
+        layer.d.set_profiling(True)
+        for _ in range(extra):
+            layer.forward(T, logits, x, fused=args.fused)
+        torch.cuda.synchronize()
+        for names in STAGE_KERNELS.values():
+            for k in names:
+                ms, n = layer.d.kernel_time(k)
+                if n:
+                    kernel_ms[k] = (ms / n, n // extra)
+        if dominant:
+            kernel_ms[DOMINANT_KERNEL] = dominant        # the figure from the timed region itself
     layer.d.set_profiling(False)
     layer.d.check_device_status()
     ms_total = ranks.max_over_ranks(ms_total)
@@ -572,7 +587,7 @@ def main():
 
     # ---- roofline of the dominant kernel and per-stage figures ----
     work = algorithmic_work(s, T)
-    dom = "grouped_gemm_swiglu_kernel"
+    dom = DOMINANT_KERNEL
     dom_ms, dom_per_step = kernel_ms.get(dom, (None, 0))
     shared_frac = work["shared_flop"] / work["ffn_flop"] if work["ffn_flop"] else 0.0
     # with shared experts the kernel is launched twice per step (routed + shared); flops per launch averaged

@@ -300,6 +300,10 @@ int64_t director_launch_count(const director_ctx* ctx);
  * milliseconds and the number of launches of the kernels whose name contains `name_substr`
  * since profiling was last enabled; returns a negative value on error. */
 int director_set_profiling(director_ctx* ctx, int32_t enabled);
+/* Restricts the timing to kernels whose name contains `name_substr` (NULL or "" = all kernels): two event records
+ * per launch are cheap but not free, and a measurement that wants one kernel's duration inside an otherwise
+ * undisturbed run times only that kernel. */
+int director_set_profiling_filter(director_ctx* ctx, const char* name_substr);
 double director_kernel_time(director_ctx* ctx, const char* name_substr, int64_t* launches);
 
 const char* director_status_string(int status);

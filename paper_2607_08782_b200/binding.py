@@ -26,7 +26,7 @@ EXPORTED = (
     "director_layer_wait_host", "director_set_ffn_variant", "director_placement_cost_batch",
     "director_expert_ffn_gather", "director_set_replica_policy", "director_dispatch_src",
     "director_dedup_dispatch_tokens", "director_route_dispatch_cost", "director_layer_forward",
-    "director_reserve_placements", "director_select_placement",
+    "director_reserve_placements", "director_select_placement", "director_set_profiling_filter",
 )
 
 REPLICA_ROUND_ROBIN, REPLICA_LOCAL_FIRST = 0, 1
@@ -73,6 +73,7 @@ def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.director_launch_count.argtypes = [vp]
     lib.director_launch_count.restype = c_int64
     lib.director_set_profiling.argtypes = [vp, c_int32]
+    lib.director_set_profiling_filter.argtypes = [vp, c_char_p]
     lib.director_set_ffn_variant.argtypes = [vp, c_int32]
     lib.director_set_replica_policy.argtypes = [vp, c_int32]
     lib.director_reserve_placements.argtypes = [vp, c_int32]
@@ -246,7 +247,10 @@ class Director:
     def launch_count(self) -> int:
         return int(self.lib.director_launch_count(self._ctx))
 
-    def set_profiling(self, enabled: bool):
+    def set_profiling(self, enabled: bool, only: str | None = None):
+        """Per-kernel device timing on/off; `only`: time just the kernels whose name contains this string."""
+        _check(self.lib.director_set_profiling_filter(self._ctx, only.encode() if only else None),
+               "director_set_profiling_filter")
         _check(self.lib.director_set_profiling(self._ctx, 1 if enabled else 0), "director_set_profiling")
 
     def kernel_time(self, name_substr: str):

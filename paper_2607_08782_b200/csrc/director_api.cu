@@ -589,6 +589,12 @@ int director_set_profiling(director_ctx* ctx, int32_t enabled) {
     return DIRECTOR_OK;
 }
 
+int director_set_profiling_filter(director_ctx* ctx, const char* name_substr) {
+    REQUIRE_CTX(ctx);
+    ctx->profile_filter = name_substr ? name_substr : "";
+    return DIRECTOR_OK;
+}
+
 double director_kernel_time(director_ctx* ctx, const char* name_substr, int64_t* launches) {
     if (ctx == nullptr || name_substr == nullptr) return -1.0;
     if (cudaDeviceSynchronize() != cudaSuccess) return -1.0;

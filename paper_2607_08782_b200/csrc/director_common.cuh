@@ -5,6 +5,7 @@
 #include <cuda.h>
 #include <stdint.h>
 
+#include <cstring>
 #include <string>
 #include <vector>
 
@@ -93,6 +94,7 @@ struct director_ctx {
 
     int64_t launches = 0;
     bool profiling = false;
+    std::string profile_filter;         // when not empty, only kernels whose name contains it are timed
     std::vector<director::KernelEvent> events;
     std::vector<director::KernelEvent> free_events;
 };
@@ -107,7 +109,7 @@ struct LaunchScope {
     bool timed = false;
     LaunchScope(director_ctx* c, cudaStream_t s, const char* name) : ctx(c), stream(s) {
         ctx->launches++;
-        if (ctx->profiling) {
+        if (ctx->profiling && (ctx->profile_filter.empty() || strstr(name, ctx->profile_filter.c_str()) != nullptr)) {
             if (!ctx->free_events.empty()) {
                 ev = ctx->free_events.back();
                 ctx->free_events.pop_back();
