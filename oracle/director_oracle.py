@@ -12,8 +12,9 @@ replicas, "sum_i x_{i,j} <= C_max" is the capacity), workload matrix W[j, i] = t
 j routed to expert i.
 
 Where the paper fixes no detail, the reading taken is stated at the function.  Those readings
-(tie-breaks, renormalised top-k softmax, round-robin replica choice, block partition of tokens
-over source ranks, shared experts, SwiGLU) are **parity unpinned by the paper**: they are
+(tie-breaks, renormalised top-k softmax, round-robin and locality-first replica choice, the
+de-duplicated dispatch volume, block partition of tokens over source ranks, shared experts,
+SwiGLU) are **parity unpinned by the paper**: they are
 pinned only by the invariants in the CPU tests (weights sum to one, identity round trip,
 loads sum to T*K, capacity, brute-force counts, scalar-loop FFN, closed forms).
 """
