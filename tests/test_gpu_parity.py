@@ -516,3 +516,22 @@ def test_placement_bank_switches_between_layers_placements():
         L.dispatch(shape.T, case.x)
     d.select_placement(0)
     assert d.last_status() == 0
+
+
+@pytest.mark.parametrize("T", [1, 200, 1500])
+def test_many_steps_stay_bitwise_identical(T):
+    """The dynamic work-item scheduling of the GEMMs and the atomics of the counting sort must not leak into the
+    results: 300 passes of the whole layer, compared every 25th."""
+    import torch
+    shape, logits, x, weights = _custom(95, T, 256, 24, 4, 256, 1, 6, 6, 1.3)
+    X = _random_placement(95, 24, 6, 6, 7)
+    case = GpuCase(shape, logits, x, weights)
+    L = case.layer
+    L.set_placement(X)
+    y0 = L.forward(T, case.logits, case.x).clone()
+    inv0, W0 = L.inv_row.clone(), L.workload.clone()
+    for i in range(300):
+        y = L.forward(T, case.logits, case.x)
+        if i % 25 == 24:
+            assert torch.equal(y, y0) and torch.equal(L.inv_row, inv0) and torch.equal(L.workload, W0), i
+    assert L.d.last_status() == 0
