@@ -155,6 +155,17 @@ int launch_cost(director_ctx*, int T, const int32_t* topk_idx, const int32_t* sr
                 int64_t* rank_load, int64_t* dispatch_tokens, uint64_t* dispatch_bytes, cudaStream_t);
 int launch_cost_batch(director_ctx*, const int64_t* workload, int n, const uint8_t* X, int64_t* rank_load,
                       int64_t* dispatch_tokens, int64_t* summary, cudaStream_t);
+// A dense SwiGLU FFN over one segment (the shared experts as one wide FFN), see ffn_pass_swap.
+struct DenseFfn {
+    const void* in;        // bf16 [rows, H]
+    uint64_t rows;
+    const void* w_gate;    // bf16 [Fw, H]
+    const void* w_up;      // bf16 [Fw, H]
+    const void* w_down;    // bf16 [H, Fw]
+    int Fw;
+    void* hidden;          // bf16 [rows, Fw]
+    void* out;             // bf16 [rows, H]
+};
 int launch_expert_ffn(director_ctx*, int T, const void* xp, const int32_t* row_token, const int32_t* seg_offsets,
                       const void* w_gate, const void* w_up, const void* w_down, void* yp, const void* x,
                       const void* ws_gate, const void* ws_up, const void* ws_down, void* y_shared, cudaStream_t);

@@ -29,7 +29,7 @@ int ffn_swap_init(director_ctx* ctx);   // director_ffn_swap.cu
 int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int32_t* gather_rows, uint64_t rows,
                   const int32_t* seg_offsets, const int32_t* slot_expert, int G, const void* w_gate, const void* w_up,
                   const void* w_down, uint64_t n_experts, int Fw, void* hidden, void* out, unsigned int* counters,
-                  cudaStream_t st);
+                  const DenseFfn* dense, cudaStream_t st);
 int ffn_pair_init(director_ctx* ctx);   // director_ffn_pair.cu
 int launch_gemm_pair(director_ctx* ctx, int mode, const char* name, const CUtensorMap& a, const CUtensorMap& b0,
                      const CUtensorMap& b1, const umma::GroupedGemmParams& p, cudaStream_t st);
@@ -280,7 +280,7 @@ int ffn_pass(director_ctx* ctx, const void* in, uint64_t in_rows, const int32_t*
              cudaStream_t st) {
     if (ctx->ffn_variant == 2) {
         const int rc = ffn_pass_swap(ctx, in, in_rows, gather_rows, rows, seg_offsets, slot_expert, G, w_gate, w_up, w_down,
-                                     n_experts, Fw, hidden, out, counters, st);
+                                     n_experts, Fw, hidden, out, counters, nullptr, st);
         if (rc != DIRECTOR_ERR_UNSUPPORTED) return rc;   // weight arrays not expressible as one map: tile scheme 0
     }
     if (gather_rows != nullptr) return DIRECTOR_ERR_UNSUPPORTED;   // only the weight-stationary scheme gathers
@@ -321,11 +321,19 @@ int launch_expert_ffn(director_ctx* ctx, int T, const void* xp, const int32_t* r
     // work-item counters of the (up to four) GEMM launches below
     if (cudaMemsetAsync(ctx->d_sched, 0, 4 * sizeof(unsigned int), st) != cudaSuccess) return DIRECTOR_ERR_CUDA;
     const uint64_t A = (uint64_t)T * s.K;
+    const bool shared = s.S > 0 && x != nullptr && y_shared != nullptr;
+    if (shared && row_token == nullptr && ctx->ffn_variant == 2) {
+        // routed and shared experts in the same two launches: the shared experts' work items follow the routed ones
+        const DenseFfn dense{x, (uint64_t)T, ws_gate, ws_up, ws_down, s.S * s.F, ctx->d_hidden_shared, y_shared};
+        const int rc = ffn_pass_swap(ctx, xp, A, nullptr, A, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up, w_down,
+                                     s.E, s.F, ctx->d_hidden, yp, ctx->d_sched, &dense, st);
+        if (rc != DIRECTOR_ERR_UNSUPPORTED) return rc;    // a weight pair not expressible as one map: separate passes
+    }
     int rc = row_token ? ffn_pass(ctx, x, (uint64_t)T, row_token, A, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up,
                                   w_down, s.E, s.F, ctx->d_hidden, yp, ctx->d_sched, st)
                        : ffn_pass(ctx, xp, A, nullptr, A, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up, w_down,
                                   s.E, s.F, ctx->d_hidden, yp, ctx->d_sched, st);
-    if (rc != DIRECTOR_OK || s.S == 0 || x == nullptr || y_shared == nullptr) return rc;
+    if (rc != DIRECTOR_OK || !shared) return rc;
     {
         LaunchScope scope(ctx, st, "one_segment_kernel");
         one_segment_kernel<<<1, 1, 0, st>>>(ctx->d_one_seg, T);

@@ -112,9 +112,19 @@ struct SwapParams {
     int32_t* status;
     unsigned int* counter;     // next unclaimed work item of this launch (zero when the kernel starts)
     const int32_t* row_token;  // GATHER only: token of every permuted row (the tokens operand is gathered from x)
+    // Optional second problem of the same launch: one dense segment of `dense_rows` rows against a single weight
+    // set (the shared experts run as one wide FFN over all tokens).  Its items follow the grouped problem's in the
+    // work-item order, so the two share the launch, its prologue and its tail.  dense_rows == 0: absent.
+    int dense_rows;
+    int dense_w_blocks;
+    int dense_k_steps;
+    int dense_out_pitch;
+    int dense_gate_first;
+    void* dense_out;
 };
 
 struct SwapTile {
+    int prob;      // 0: grouped problem, 1: dense problem
     int row0;      // first token row of the tile
     int valid;     // tokens of the tile that belong to the segment (1..256)
     int n;         // valid rounded up to a multiple of 32: N of the MMA
@@ -132,6 +142,7 @@ struct SwapWalker {
         while (w >= tt_start[g + 1] * w_blocks) ++g;
         const int nt = tt_start[g + 1] - tt_start[g];
         const int local = w - tt_start[g] * w_blocks;
+        t.prob = 0;
         t.wb = local / nt;
         const int tt = local - t.wb * nt;
         t.row0 = seg_off[g] + tt * TOKEN_TILE;
@@ -149,7 +160,8 @@ struct SwapWalker {
 template <int MODE, int EPI_GROUPS, bool GATHER, int S_STAGES>
 __global__ void __launch_bounds__(96 + 128 * EPI_GROUPS, 1)
 grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
-                         const SwapParams p) {
+                         const __grid_constant__ CUtensorMap tm_w2 /* dense problem */,
+                         const __grid_constant__ CUtensorMap tm_x2, const SwapParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
@@ -237,7 +249,8 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     // path.  Tail tiles are cheaper than full ones, so fixed assignments leave 6-15 % of imbalance between clusters;
     // and since the items are still taken in order, clusters running at the same time keep working on neighbouring
     // items and share their weight tiles in L2.
-    const int total_items = walker.total;
+    const int dense_tiles = (p.dense_rows + TOKEN_TILE - 1) / TOKEN_TILE;
+    const int total_items = walker.total + dense_tiles * p.dense_w_blocks;
     constexpr uint32_t SCHED_RANK = 0;                             // CTA of the pair that owns the ring's barriers
     const bool sched_local = rank == SCHED_RANK;
     // consumer side of the ring: wait for item i, read it, hand the slot back
@@ -253,7 +266,8 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
             tile.valid = v.y;
             tile.n = (v.y + TOKEN_STEP - 1) / TOKEN_STEP * TOKEN_STEP;
             tile.w_row = v.z;
-            tile.wb = v.w;
+            tile.wb = v.w & 0x3FFFFFFF;
+            tile.prob = (v.w >> 30) & 1;
         }
         return ok;
     };
@@ -280,6 +294,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
             t.n = __shfl_sync(0xFFFFFFFFu, t.n, 0);
             t.w_row = __shfl_sync(0xFFFFFFFFu, t.w_row, 0);
             t.wb = __shfl_sync(0xFFFFFFFFu, t.wb, 0);
+            t.prob = 0;                                                 // a gathering launch has no dense problem
             if (!ok || t.valid == 0) break;
             const int half = t.n >> 1;                                  // token rows this CTA supplies (multiple of 16)
             const int x_row = t.row0 + (int)rank * half;
@@ -322,14 +337,17 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 if (t.valid == 0) break;
                 const int x_row = t.row0 + (int)rank * (t.n >> 1);          // this CTA's half of the tile's tokens
                 const int w_row = t.w_row + (int)rank * (ROWS_PER_BLOCK / 2);
-                for (int kb = 0; kb < p.k_steps; ++kb) {
+                const CUtensorMap* mw = t.prob ? &tm_w2 : &tm_w;
+                const CUtensorMap* mx = t.prob ? &tm_x2 : &tm_x;
+                const int k_steps = t.prob ? p.dense_k_steps : p.k_steps;
+                for (int kb = 0; kb < k_steps; ++kb) {
                     if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag))) break;
                     const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
                     const uint32_t a_dst = tiles + stage * S_STAGE_BYTES;
                     mbar_expect_tx_cluster(leader_full, S_STAGE_BYTES);
-                    if (MODE == 0) tma_load_3d_pair(a_dst, &tm_w, leader_full, kb * BLOCK_K, 0, w_row);
-                    else tma_load_2d_pair(a_dst, &tm_w, leader_full, kb * BLOCK_K, w_row);
-                    tma_load_2d_pair(a_dst + A_BYTES, &tm_x, leader_full, kb * BLOCK_K, x_row);
+                    if (MODE == 0) tma_load_3d_pair(a_dst, mw, leader_full, kb * BLOCK_K, 0, w_row);
+                    else tma_load_2d_pair(a_dst, mw, leader_full, kb * BLOCK_K, w_row);
+                    tma_load_2d_pair(a_dst + A_BYTES, mx, leader_full, kb * BLOCK_K, x_row);
                     if (++stage == S_STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -348,7 +366,8 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TOKEN_TILE);
                 const uint32_t idesc = S_IDESC_BASE | ((uint32_t)(t.n >> 3) << 17);
-                for (int kb = 0; kb < p.k_steps; ++kb) {
+                const int k_steps = t.prob ? p.dense_k_steps : p.k_steps;
+                for (int kb = 0; kb < k_steps; ++kb) {
                     if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag))) break;
                     tc_fence_after();
                     const uint32_t a_src = tiles + stage * S_STAGE_BYTES;
@@ -385,9 +404,13 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 const int q = i & (SCHED_SLOTS - 1);
                 if (!mbar_wait(sched_empty(q), (((uint32_t)i / SCHED_SLOTS) & 1u) ^ 1u, abort_flag)) break;
                 int4 item = make_int4(0, 0, 0, 0);
-                if (w < total_items) {
+                if (w < walker.total) {
                     walker.get(w, t);
                     item = make_int4(t.row0, t.valid, t.w_row, t.wb);
+                } else if (w < total_items) {          // dense problem: (weight block, token tile) over one segment
+                    const int local = w - walker.total;
+                    const int wb = local / dense_tiles, row0 = (local - wb * dense_tiles) * TOKEN_TILE;
+                    item = make_int4(row0, min(TOKEN_TILE, p.dense_rows - row0), wb * ROWS_PER_BLOCK, wb | (1 << 30));
                 }
                 sched_item[q] = item;
                 st_cluster_v4(map_to_cta(smem_u32(&sched_item[q]), 1u - SCHED_RANK), item);
@@ -401,7 +424,8 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
         const int cgroup = EPI_GROUPS == 1 ? 0 : (warp - 3) >> 2;  // which of the 32-token chunks this warp takes
         constexpr int CSTEP = 32 * EPI_GROUPS;
         const int c_first = 32 * cgroup;
-        uint16_t* out = static_cast<uint16_t*>(p.out);
+        uint16_t* const out_a = static_cast<uint16_t*>(p.out);
+        uint16_t* const out_b = static_cast<uint16_t*>(p.dense_out);
         const int lane_row = quad * 32 + lane;                     // weight row of this thread inside the CTA's 128
         bool ok = true;
         for (int it = 0; ok; ++it) {
@@ -413,6 +437,8 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
             if (!(ok = mbar_wait(tfull_bar(acc), ((uint32_t)it >> 1) & 1u, abort_flag))) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * TOKEN_TILE);
+            uint16_t* const out = t.prob ? out_b : out_a;
+            const int out_pitch = t.prob ? p.dense_out_pitch : p.out_pitch;
             if constexpr (MODE == 0) {
                 // even lane: one of (gate, up) for feature f, odd lane: the other; column = token.
                 // The two lanes of a pair split the tokens: the even lane finishes the even tokens, the odd lane
@@ -420,15 +446,15 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 // 32 lanes stay active and no branch separates the shuffles.
                 const int f = t.wb * 128 + (int)rank * 64 + (lane_row >> 1);
                 const bool odd = (lane & 1) != 0;
-                const bool i_am_gate = (!odd) == (p.gate_first != 0);
-                uint16_t* ocol = out + (size_t)(t.row0 + (odd ? 1 : 0)) * p.out_pitch + f;
-                const size_t two_rows = 2 * (size_t)p.out_pitch;
+                const bool i_am_gate = (!odd) == ((t.prob ? p.dense_gate_first : p.gate_first) != 0);
+                uint16_t* ocol = out + (size_t)(t.row0 + (odd ? 1 : 0)) * out_pitch + f;
+                const size_t two_rows = 2 * (size_t)out_pitch;
 #pragma unroll 1
                 for (int c = c_first; c < t.n; c += CSTEP) {
                     uint32_t v[32];
                     tmem_ld32(taddr + c, v);
                     tmem_ld_wait();
-                    uint16_t* ptr = ocol + (size_t)c * p.out_pitch;     // my token of pair m is row c + 2m (+1 if odd)
+                    uint16_t* ptr = ocol + (size_t)c * out_pitch;       // my token of pair m is row c + 2m (+1 if odd)
                     const int rem = t.valid - c - (odd ? 1 : 0);        // store pair m iff 2m < rem
 #pragma unroll
                     for (int m = 0; m < 16; ++m) {
@@ -443,18 +469,18 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 }
             } else {
                 const int h_col = t.wb * 256 + (int)rank * 128 + lane_row;
-                uint16_t* ocol = out + (size_t)t.row0 * p.out_pitch + h_col;
+                uint16_t* ocol = out + (size_t)t.row0 * out_pitch + h_col;
 #pragma unroll 1
                 for (int c = c_first; c < t.n; c += CSTEP) {
                     uint32_t v[32];
                     tmem_ld32(taddr + c, v);
                     tmem_ld_wait();
-                    uint16_t* ptr = ocol + (size_t)c * p.out_pitch;
+                    uint16_t* ptr = ocol + (size_t)c * out_pitch;
                     const int rem = t.valid - c;
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         if (j < rem) *ptr = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[j])));
-                        ptr += p.out_pitch;
+                        ptr += out_pitch;
                     }
                 }
             }
@@ -505,8 +531,8 @@ bool map_interleaved(director_ctx* ctx, CUtensorMap* map, const void* first, uin
 }
 
 template <int MODE, int EPI_GROUPS, bool GATHER, int STAGES>
-int launch_swap_n(director_ctx* ctx, const char* name, const CUtensorMap& w, const CUtensorMap& x, const SwapParams& p,
-                  cudaStream_t st) {
+int launch_swap_n(director_ctx* ctx, const char* name, const CUtensorMap& w, const CUtensorMap& x, const CUtensorMap& w2,
+                  const CUtensorMap& x2, const SwapParams& p, cudaStream_t st) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * ctx->pair_clusters));
     cfg.blockDim = dim3(96 + 128 * EPI_GROUPS);
@@ -520,14 +546,15 @@ int launch_swap_n(director_ctx* ctx, const char* name, const CUtensorMap& w, con
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     LaunchScope scope(ctx, st, name);
-    return cuda_status(cudaLaunchKernelEx(&cfg, grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, STAGES>, w, x, p));
+    return cuda_status(cudaLaunchKernelEx(&cfg, grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, STAGES>, w, x, w2, x2, p));
 }
 
+// w2 / x2: the dense problem's maps (any valid map when the launch has none)
 template <int MODE, int EPI_GROUPS, bool GATHER>
-int launch_swap(director_ctx* ctx, const char* name, const CUtensorMap& w, const CUtensorMap& x, const SwapParams& p,
-                cudaStream_t st) {
-    return swap_stages(p.G) == 7 ? launch_swap_n<MODE, EPI_GROUPS, GATHER, 7>(ctx, name, w, x, p, st)
-                                 : launch_swap_n<MODE, EPI_GROUPS, GATHER, 6>(ctx, name, w, x, p, st);
+int launch_swap(director_ctx* ctx, const char* name, const CUtensorMap& w, const CUtensorMap& x, const CUtensorMap& w2,
+                const CUtensorMap& x2, const SwapParams& p, cudaStream_t st) {
+    return swap_stages(p.G) == 7 ? launch_swap_n<MODE, EPI_GROUPS, GATHER, 7>(ctx, name, w, x, w2, x2, p, st)
+                                 : launch_swap_n<MODE, EPI_GROUPS, GATHER, 6>(ctx, name, w, x, w2, x2, p, st);
 }
 
 template <int MODE, int EPI_GROUPS, bool GATHER>
@@ -550,29 +577,50 @@ int ffn_swap_init(director_ctx*) {
 // in [rows, H] -> hidden [rows, Fw] -> out [rows, H] over a segment table, weight-stationary pair kernels.
 // With gather_rows != nullptr, `in` is the un-permuted layer input [in_rows, H] and row i of the segment table
 // is in[gather_rows[i]].
-// Returns DIRECTOR_ERR_UNSUPPORTED if the two weight arrays cannot be described by one interleaving map.
+// dense (optional, not with gather_rows): a second FFN over ONE segment of dense->rows rows of dense->in with a single
+// weight set - the shared experts - whose work items ride in the same two launches.
+// Returns DIRECTOR_ERR_UNSUPPORTED if a pair of weight arrays cannot be described by one interleaving map.
 int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int32_t* gather_rows, uint64_t rows,
                   const int32_t* seg_offsets, const int32_t* slot_expert, int G, const void* w_gate, const void* w_up,
                   const void* w_down, uint64_t n_experts, int Fw, void* hidden, void* out,
-                  unsigned int* counters /* 2 zeroed work-item counters */, cudaStream_t st) {
+                  unsigned int* counters /* 2 zeroed work-item counters */, const DenseFfn* dense, cudaStream_t st) {
     const int H = ctx->shape.H;
-    const uintptr_t pg = reinterpret_cast<uintptr_t>(w_gate), pu = reinterpret_cast<uintptr_t>(w_up);
-    if (pg == pu) return DIRECTOR_ERR_UNSUPPORTED;
-    const bool gate_first = pg < pu;
-    const uint64_t delta = gate_first ? pu - pg : pg - pu;
-    if (delta % 16 != 0 || delta >= (1ull << 40)) return DIRECTOR_ERR_UNSUPPORTED;
+    struct Interleave { bool ok; bool gate_first; const void* first; uint64_t delta; };
+    auto interleave = [](const void* g, const void* u) {
+        const uintptr_t pg = reinterpret_cast<uintptr_t>(g), pu = reinterpret_cast<uintptr_t>(u);
+        Interleave r{false, pg < pu, pg < pu ? g : u, pg < pu ? pu - pg : pg - pu};
+        r.ok = pg != pu && r.delta % 16 == 0 && r.delta < (1ull << 40);
+        return r;
+    };
+    const Interleave ia = interleave(w_gate, w_up);
+    if (!ia.ok) return DIRECTOR_ERR_UNSUPPORTED;
+    if (dense && gather_rows) return DIRECTOR_ERR_INVALID_ARG;
     CUtensorMap m_in, m_gu, m_h, m_d;
     if (!map_2d(ctx, &m_in, in, in_rows, H, gather_rows ? 1 : 128) || !map_2d(ctx, &m_h, hidden, rows, Fw) ||
         !map_2d(ctx, &m_d, w_down, n_experts * H, Fw))
         return DIRECTOR_ERR_CUDA;
-    if (!map_interleaved(ctx, &m_gu, gate_first ? w_gate : w_up, delta, n_experts * Fw, H)) return DIRECTOR_ERR_UNSUPPORTED;
-    SwapParams p1{seg_offsets, slot_expert, G, Fw / 128, H / BLOCK_K, Fw, Fw, gate_first ? 1 : 0, hidden, ctx->d_status,
-                  counters, gather_rows};
-    int rc = gather_rows ? launch_swap<0, EPI_GROUPS_GEMM1, true>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, p1, st)
-                         : launch_swap<0, EPI_GROUPS_GEMM1, false>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, p1, st);
+    if (!map_interleaved(ctx, &m_gu, ia.first, ia.delta, n_experts * Fw, H)) return DIRECTOR_ERR_UNSUPPORTED;
+    // the dense problem's maps default to the grouped problem's (never used then)
+    CUtensorMap d_in = m_in, d_gu = m_gu, d_h = m_h, d_d = m_d;
+    Interleave id{true, true, nullptr, 0};
+    if (dense) {
+        id = interleave(dense->w_gate, dense->w_up);
+        if (!id.ok) return DIRECTOR_ERR_UNSUPPORTED;
+        if (!map_2d(ctx, &d_in, dense->in, dense->rows, H) || !map_2d(ctx, &d_h, dense->hidden, dense->rows, dense->Fw) ||
+            !map_2d(ctx, &d_d, dense->w_down, H, dense->Fw))
+            return DIRECTOR_ERR_CUDA;
+        if (!map_interleaved(ctx, &d_gu, id.first, id.delta, dense->Fw, H)) return DIRECTOR_ERR_UNSUPPORTED;
+    }
+    const int d_rows = dense ? (int)dense->rows : 0, d_Fw = dense ? dense->Fw : 0;
+    SwapParams p1{seg_offsets, slot_expert, G, Fw / 128, H / BLOCK_K, Fw, Fw, ia.gate_first ? 1 : 0, hidden, ctx->d_status,
+                  counters, gather_rows, d_rows, d_Fw / 128, H / BLOCK_K, d_Fw, id.gate_first ? 1 : 0,
+                  dense ? dense->hidden : nullptr};
+    int rc = gather_rows ? launch_swap<0, EPI_GROUPS_GEMM1, true>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, d_gu, d_in, p1, st)
+                         : launch_swap<0, EPI_GROUPS_GEMM1, false>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, d_gu, d_in, p1, st);
     if (rc != DIRECTOR_OK) return rc;
-    SwapParams p2{seg_offsets, slot_expert, G, H / 256, Fw / BLOCK_K, H, H, 1, out, ctx->d_status, counters + 1, nullptr};
-    return launch_swap<1, EPI_GROUPS_GEMM2, false>(ctx, "grouped_gemm_down_kernel", m_d, m_h, p2, st);
+    SwapParams p2{seg_offsets, slot_expert, G, H / 256, Fw / BLOCK_K, H, H, 1, out, ctx->d_status, counters + 1, nullptr,
+                  d_rows, H / 256, d_Fw / BLOCK_K, H, 1, dense ? dense->out : nullptr};
+    return launch_swap<1, EPI_GROUPS_GEMM2, false>(ctx, "grouped_gemm_down_kernel", m_d, m_h, d_d, d_h, p2, st);
 }
 
 }  // namespace director
