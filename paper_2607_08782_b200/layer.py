@@ -120,7 +120,7 @@ class MoELayer:
     def capture(self, T, logits, x, with_cost=True, fused=False):
         """Records one pass of the layer (fixed T, fixed input and output buffers) into a CUDA graph and returns it;
         `graph.replay()` re-runs the pass with a single launch, which matters for decode-sized batches where the
-        nine kernel launches cost more than the kernels.  Per-kernel profiling must be off while capturing."""
+        handful of kernel launches cost more than the kernels.  Per-kernel profiling must be off while capturing."""
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):                      # first pass outside the capture: lazy module loading
