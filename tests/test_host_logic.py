@@ -89,3 +89,20 @@ def test_expert_counts_and_loads():
     assert placement.expert_counts(W).tolist() == [5, 7, 9]
     X = np.array([[1, 0], [0, 1], [1, 0]], dtype=np.uint8)
     assert placement.single_copy_loads([5, 7, 9], X).tolist() == [14, 7]
+
+
+def test_the_header_is_plain_c(tmp_path):
+    """include/director.h is the C ABI: it must compile as C99 with warnings on, without any CUDA header."""
+    import os
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        import pytest
+        pytest.skip("no C compiler")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = tmp_path / "use_header.c"
+    src.write_text('#include "director.h"\nint main(void) { director_shape s = {0}; (void)s; return DIRECTOR_OK; }\n')
+    r = subprocess.run([gcc, "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-I", os.path.join(root, "include"),
+                        "-fsyntax-only", str(src)], capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
