@@ -535,3 +535,36 @@ def test_many_steps_stay_bitwise_identical(T):
         if i % 25 == 24:
             assert torch.equal(y, y0) and torch.equal(L.inv_row, inv0) and torch.equal(L.workload, W0), i
     assert L.d.last_status() == 0
+
+
+def test_argument_errors_of_the_newer_entry_points():
+    """Host-side checks return a status before anything is launched."""
+    import torch
+    from paper_2607_08782_b200.binding import DirectorError
+    shape, logits, x, weights = _custom(97, 64, 256, 8, 2, 128, 0, 4, 2, 1.2)
+    case = GpuCase(shape, logits, x, weights)
+    L, d = case.layer, case.layer.d
+    L.set_placement(_random_placement(97, 8, 4, 2, 0))
+    n0 = d.launch_count()
+    W, load, dt, db = L.workload, L.rank_load, L.dispatch_tokens, L.dispatch_bytes
+    for bad_call in (
+        lambda: d.layer_forward(64, None, case.x, *L.w, None, None, None, L.y, W, load, dt, db),          # no logits
+        lambda: d.layer_forward(65, case.logits, case.x, *L.w, None, None, None, L.y, W, load, dt, db),   # T > T_max
+        lambda: d.layer_forward(64, case.logits, case.x, *L.w, None, None, None, L.y, None, load, dt, db),
+        lambda: d.route_dispatch_cost(64, case.logits, case.x, L.topk_idx, L.topk_w, L.xp, None, L.inv_row, L.dest_rank,
+                                      L.seg_offsets, W, load, dt, db),
+        lambda: d.dedup_dispatch_tokens(64, None, None, dt),
+        lambda: d.reserve_placements(0),
+        lambda: d.select_placement(-1),
+        lambda: d.set_replica_policy(7),
+    ):
+        with pytest.raises(DirectorError):
+            bad_call()
+    assert d.launch_count() == n0                         # nothing was launched
+    d.set_profiling(True, only="combine")
+    L.forward(64, case.logits, case.x)
+    ms_all, n_all = d.kernel_time("kernel")
+    ms_c, n_c = d.kernel_time("combine_kernel")
+    d.set_profiling(False)
+    assert n_all == n_c == 1 and ms_c > 0                 # the filter timed the combine kernel only
+    assert d.last_status() == 0
