@@ -287,7 +287,7 @@ STAGE_KERNELS = {
                  "dispatch_travel_count_scan_kernel", "dispatch_slot_count_scan_kernel", "dispatch_local_index_kernel"],
     "expert_ffn": ["grouped_gemm_swiglu_kernel", "grouped_gemm_down_kernel", "one_segment_kernel"],
     "combine": ["combine_kernel"],
-    "placement_cost": ["cost_workload_kernel", "cost_count_scan_kernel", "cost_kernel",
+    "placement_cost": ["cost_workload_hist_kernel", "cost_from_workload_kernel", "cost_count_scan_kernel", "cost_kernel",
                        "cost_travel_count_scan_kernel", "cost_local_kernel"],
 }
 

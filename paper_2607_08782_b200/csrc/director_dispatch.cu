@@ -188,28 +188,67 @@ cost_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ sr
 // an expert is numbered in ascending token order, so the assignments that rank j sends to expert e occupy a
 // contiguous range [a, b) of n.  Round-robin over r replicas gives replica q exactly
 //     f(b) - f(a),  f(x) = max(0, ceil((x - q) / r))
-// of them.  The whole cost therefore follows from the workload matrix W alone: a histogram over the tiles and,
-// in the last CTA to finish, one warp per expert - a single kernel, no per-assignment ranks.  Under the locality-first rule the ranks that host e keep their
+// of them.  The whole cost therefore follows from the workload matrix W alone: one histogram kernel and one
+// warp-per-expert kernel, no per-assignment ranks.  Under the locality-first rule the ranks that host e keep their
 // own W[j][e] assignments and the same closed form runs over the remaining (travelling) ranks' counts.
 
-constexpr int kCostWarps = 8;
+constexpr int kHistSmemInts = 4096;
+
+__global__ void __launch_bounds__(kTokenTile)
+workload_hist_kernel(const int32_t* __restrict__ topk_idx, int T, int E, int K, int R,
+                     unsigned long long* __restrict__ workload, unsigned long long* __restrict__ rank_load,
+                     unsigned long long* __restrict__ dispatch_tokens, unsigned long long* __restrict__ dispatch_bytes,
+                     int32_t* __restrict__ status) {
+    __shared__ uint32_t hist[kHistSmemInts];
+    if (blockIdx.x == 0) {      // the other outputs are accumulated by the next kernel: clear them here
+        for (int i = threadIdx.x; i < R * R; i += blockDim.x) { dispatch_tokens[i] = 0ull; dispatch_bytes[i] = 0ull; }
+        for (int i = threadIdx.x; i < R; i += blockDim.x) rank_load[i] = 0ull;
+    }
+    const int t0 = blockIdx.x * kTokenTile, t1 = min(t0 + kTokenTile, T) - 1;
+    const int src_lo = (int)(((long long)t0 * R) / T), src_hi = (int)(((long long)t1 * R) / T);
+    const int n_src = src_hi - src_lo + 1;
+    const bool use_smem = n_src * E <= kHistSmemInts;
+    if (use_smem) {
+        for (int i = threadIdx.x; i < n_src * E; i += blockDim.x) hist[i] = 0u;
+        __syncthreads();
+    }
+    const int t = t0 + threadIdx.x;
+    if (t < T) {
+        const int src = (int)(((long long)t * R) / T);
+        for (int s = 0; s < K; ++s) {
+            const int e = __ldg(topk_idx + (size_t)t * K + s);
+            if ((unsigned)e >= (unsigned)E) { director_set_status(status, DIRECTOR_ERR_BAD_INDEX); continue; }
+            if (use_smem) atomicAdd(&hist[(src - src_lo) * E + e], 1u);
+            else atomicAdd(workload + (size_t)src * E + e, 1ull);
+        }
+    }
+    if (use_smem) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < n_src * E; i += blockDim.x)
+            if (hist[i]) atomicAdd(workload + (size_t)src_lo * E + i, (unsigned long long)hist[i]);
+    }
+}
 
 // One warp per expert, lanes over the source ranks: prefix-scan the expert's column of W over the ranks
 // (the start a_j of rank j's range of n), split each range over the replicas, add into the outputs
-// (zeroed by the first CTA of workload_cost_kernel) with 64-bit global atomics.
+// (zeroed by workload_hist_kernel) with 64-bit global atomics.
+constexpr int kCostWarps = 8;
 
-__device__ __forceinline__ void cost_of_expert(int e, int lane, const unsigned long long* workload, int E, int R, int C_max,
-                                               const int32_t* __restrict__ rep_start, const int32_t* __restrict__ rep_slot,
-                                               const unsigned long long* __restrict__ host_mask /* non-null: locality-first rule */,
-                                               unsigned long long* rank_load, unsigned long long* dispatch_tokens,
-                                               unsigned long long* dispatch_bytes, unsigned long long bytes_per_token) {
+__global__ void __launch_bounds__(kCostWarps * 32)
+cost_from_workload_kernel(const unsigned long long* __restrict__ workload, int E, int R, int C_max,
+                          const int32_t* __restrict__ rep_start, const int32_t* __restrict__ rep_slot,
+                          const unsigned long long* __restrict__ host_mask /* non-null: locality-first rule */,
+                          unsigned long long* __restrict__ rank_load, unsigned long long* __restrict__ dispatch_tokens,
+                          unsigned long long* __restrict__ dispatch_bytes, unsigned long long bytes_per_token) {
+    const int e = blockIdx.x * kCostWarps + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (e >= E) return;
     const int r0 = __ldg(rep_start + e);
     const uint32_t r = (uint32_t)(__ldg(rep_start + e + 1) - r0);
     const unsigned long long hm = host_mask ? __ldg(host_mask + e) : 0ull;
     uint32_t carry = 0;                                        // assignments of e sent by ranks before this chunk
     for (int j0 = 0; j0 < R; j0 += 32) {
         const int j = j0 + lane;
-        uint32_t w = j < R ? (uint32_t)__ldcg(workload + (size_t)j * E + e) : 0u;   // counts fit 32 bits: T*K < 2^31
+        uint32_t w = j < R ? (uint32_t)workload[(size_t)j * E + e] : 0u;   // counts fit 32 bits: T*K < 2^31
         if (j < R && ((hm >> j) & 1ull)) {
             // locality first: a rank that hosts e serves its own tokens; only the others' assignments are numbered
             if (w) {
@@ -241,55 +280,6 @@ __device__ __forceinline__ void cost_of_expert(int e, int lane, const unsigned l
         carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
 }
-
-constexpr int kHistSmemInts = 4096;
-
-__global__ void __launch_bounds__(kTokenTile)
-workload_cost_kernel(const int32_t* __restrict__ topk_idx, int T, int E, int K, int R, int C_max, int n_tiles,
-                     const int32_t* __restrict__ rep_start, const int32_t* __restrict__ rep_slot,
-                     const unsigned long long* __restrict__ host_mask /* non-null: locality-first rule */,
-                     unsigned long long* workload, unsigned long long* rank_load, unsigned long long* dispatch_tokens,
-                     unsigned long long* dispatch_bytes, unsigned long long bytes_per_token,
-                     unsigned int* __restrict__ ticket, int32_t* __restrict__ status) {
-    __shared__ uint32_t hist[kHistSmemInts];
-    __shared__ bool is_last;
-    if (blockIdx.x == 0) {      // the other outputs are accumulated by the last CTA: clear them here
-        for (int i = threadIdx.x; i < R * R; i += blockDim.x) { dispatch_tokens[i] = 0ull; dispatch_bytes[i] = 0ull; }
-        for (int i = threadIdx.x; i < R; i += blockDim.x) rank_load[i] = 0ull;
-    }
-    const int t0 = blockIdx.x * kTokenTile, t1 = min(t0 + kTokenTile, T) - 1;
-    const int src_lo = (int)(((long long)t0 * R) / T), src_hi = (int)(((long long)t1 * R) / T);
-    const int n_src = src_hi - src_lo + 1;
-    const bool use_smem = n_src * E <= kHistSmemInts;
-    if (use_smem) {
-        for (int i = threadIdx.x; i < n_src * E; i += blockDim.x) hist[i] = 0u;
-        __syncthreads();
-    }
-    const int t = t0 + threadIdx.x;
-    if (t < T) {
-        const int src = (int)(((long long)t * R) / T);
-        for (int s = 0; s < K; ++s) {
-            const int e = __ldg(topk_idx + (size_t)t * K + s);
-            if ((unsigned)e >= (unsigned)E) { director_set_status(status, DIRECTOR_ERR_BAD_INDEX); continue; }
-            if (use_smem) atomicAdd(&hist[(src - src_lo) * E + e], 1u);
-            else atomicAdd(workload + (size_t)src * E + e, 1ull);
-        }
-    }
-    if (use_smem) {
-        __syncthreads();
-        for (int i = threadIdx.x; i < n_src * E; i += blockDim.x)
-            if (hist[i]) atomicAdd(workload + (size_t)src_lo * E + i, (unsigned long long)hist[i]);
-    }
-    // the last CTA to finish holds the complete W: one warp per expert turns it into load and dispatch volume
-    if (!last_cta_done(ticket, n_tiles, &is_last)) return;
-    const int lane = threadIdx.x & 31;
-    for (int e = threadIdx.x >> 5; e < E; e += kTileWarps)
-        cost_of_expert(e, lane, workload, E, R, C_max, rep_start, rep_slot, host_mask, rank_load, dispatch_tokens,
-                       dispatch_bytes, bytes_per_token);
-    if (threadIdx.x == 0) *ticket = 0u;
-}
-
-
 
 // ---- batched placement cost: many candidate placements against one workload matrix ----
 //
@@ -468,13 +458,24 @@ int launch_cost(director_ctx* ctx, int T, const int32_t* topk_idx, const int32_t
     cudaError_t e;
     if ((e = cudaMemsetAsync(workload, 0, sizeof(int64_t) * s.R * s.E, st)) != cudaSuccess) return cuda_status(e);
     if (src_rank == nullptr) {
-        LaunchScope scope(ctx, st, "cost_workload_kernel");
-        workload_cost_kernel<<<n_tiles, kTokenTile, 0, st>>>(
-            topk_idx, T, s.E, s.K, s.R, s.C_max, n_tiles, ctx->d_rep_start, ctx->d_rep_slot,
-            local_first ? ctx->d_host_mask : nullptr, reinterpret_cast<unsigned long long*>(workload),
-            reinterpret_cast<unsigned long long*>(rank_load), reinterpret_cast<unsigned long long*>(dispatch_tokens),
-            reinterpret_cast<unsigned long long*>(dispatch_bytes), (unsigned long long)s.H * 2ull, ctx->d_ticket,
-            ctx->d_status);
+        {
+            LaunchScope scope(ctx, st, "cost_workload_hist_kernel");
+            workload_hist_kernel<<<n_tiles, kTokenTile, 0, st>>>(topk_idx, T, s.E, s.K, s.R,
+                                                                 reinterpret_cast<unsigned long long*>(workload),
+                                                                 reinterpret_cast<unsigned long long*>(rank_load),
+                                                                 reinterpret_cast<unsigned long long*>(dispatch_tokens),
+                                                                 reinterpret_cast<unsigned long long*>(dispatch_bytes),
+                                                                 ctx->d_status);
+            if (cudaGetLastError() != cudaSuccess) return DIRECTOR_ERR_CUDA;
+        }
+        LaunchScope scope(ctx, st, "cost_from_workload_kernel");
+        cost_from_workload_kernel<<<(s.E + kCostWarps - 1) / kCostWarps, kCostWarps * 32, 0, st>>>(reinterpret_cast<const unsigned long long*>(workload), s.E, s.R,
+                                                     s.C_max, ctx->d_rep_start, ctx->d_rep_slot,
+                                                     local_first ? ctx->d_host_mask : nullptr,
+                                                     reinterpret_cast<unsigned long long*>(rank_load),
+                                                     reinterpret_cast<unsigned long long*>(dispatch_tokens),
+                                                     reinterpret_cast<unsigned long long*>(dispatch_bytes),
+                                                     (unsigned long long)s.H * 2ull);
         return cuda_status(cudaGetLastError());
     }
     if ((e = cudaMemsetAsync(rank_load, 0, sizeof(int64_t) * s.R, st)) != cudaSuccess) return cuda_status(e);
