@@ -125,7 +125,10 @@ __device__ __noinline__ void exact_top8(const float* __restrict__ row, int E, rk
 // The loop is bound by the integer pipe (min/max/logic run at half the issue rate), so the key of a logit costs
 // three integer instructions (shift, two 3-input logic ops); folding -0.0 onto +0.0 and the Inf/NaN detector
 // (x * 0 is NaN exactly for Inf and NaN) are floating-point instructions that issue beside them.
-template <bool VEC, int LPT, bool K8>
+// PRE > 0: the lane's (at most PRE) groups are all loaded before the first is sorted - one memory round trip instead of
+// one per group - for launches too small to hide a load's latency behind other warps; PRE == 0: the loads of the
+// lane's next group are in flight while the current one is sorted (fewer registers).
+template <bool VEC, int LPT, bool K8, int PRE = 0>
 __device__ __forceinline__ bool route_token(const float* __restrict__ row, int E, int K, int sub, bool live,
                                             int32_t* __restrict__ status, int (&win_idx)[8], float (&win_w)[8]) {
     uint32_t top[8];
@@ -134,7 +137,6 @@ __device__ __forceinline__ bool route_token(const float* __restrict__ row, int E
     uint32_t rej = 0u;                               // largest key seen that is not in top[] (K8 only)
     float nonfinite = 0.0f;                          // becomes NaN iff an Inf or NaN logit was read
 
-    // software pipeline: the loads of the lane's next group are in flight while the current one is sorted
     auto load_group = [&](int e0, float (&v)[8]) {
         if (VEC && e0 + 8 <= E) {
             const float4 a = __ldg(reinterpret_cast<const float4*>(row + e0));
@@ -145,11 +147,8 @@ __device__ __forceinline__ bool route_token(const float* __restrict__ row, int E
             for (int i = 0; i < 8; ++i) v[i] = (e0 + i < E) ? __ldg(row + e0 + i) : 0.0f;
         }
     };
-    float v[8], v_next[8];
-    if (8 * sub < E) load_group(8 * sub, v);
-    for (int e0 = 8 * sub; e0 < E; e0 += 8 * LPT) {
-        const int e_next = e0 + 8 * LPT;
-        if (e_next < E) load_group(e_next, v_next);
+    // keys of one group, sorted and merged into the running top-8
+    auto take_group = [&](int e0, const float (&v)[8]) {
         uint32_t grp[8];
         // low byte of the key: 255 - expert = (248 - e0) | (7 - i), e0 being a multiple of 8
         const uint32_t group_field = 248u - (uint32_t)e0;
@@ -165,8 +164,25 @@ __device__ __forceinline__ bool route_token(const float* __restrict__ row, int E
         }
         sort8_desc32(grp);
         merge_top8_32<K8>(top, grp, rej);
+    };
+    if constexpr (PRE > 0) {
+        float va[PRE][8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = v_next[i];
+        for (int g = 0; g < PRE; ++g)
+            if (8 * (sub + g * LPT) < E) load_group(8 * (sub + g * LPT), va[g]);
+#pragma unroll
+        for (int g = 0; g < PRE; ++g)
+            if (8 * (sub + g * LPT) < E) take_group(8 * (sub + g * LPT), va[g]);
+    } else {
+        float v[8], v_next[8];
+        if (8 * sub < E) load_group(8 * sub, v);
+        for (int e0 = 8 * sub; e0 < E; e0 += 8 * LPT) {
+            const int e_next = e0 + 8 * LPT;
+            if (e_next < E) load_group(e_next, v_next);
+            take_group(e0, v);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = v_next[i];
+        }
     }
     // merge the lists of the token's lanes (butterfly: afterwards every lane holds the token's top 8)
 #pragma unroll
@@ -254,19 +270,20 @@ route_topk_kernel(const float* __restrict__ logits, int32_t* __restrict__ topk_i
 //
 // For T <= 256 the whole batch is one tile of the counting sort, every stage of the front end moves a few KB and
 // the five launches (route, count/scan, index, workload histogram, cost) cost more than their work.  One CTA of
-// 1024 threads does them back to back: four lanes per token compute the gate; then thread t < T is token t for the
+// 1024 threads does them back to back: eight lanes per token compute the gate (all of a lane's logits are loaded
+// before the first is sorted: with a single CTA there is nothing else to hide a load behind); then thread t < T is token t for the
 // counting sort (lane bitmasks per expert, popcounts; a single tile, so the tile prefix is zero), the slot lengths
 // are scanned by the block, and the histograms are accumulated per assignment in shared memory.  Same integer
 // arithmetic as the separate kernels, hence the same bits.  Round-robin replica rule, block partition of the
 // tokens over the source ranks.
 constexpr int kFrontThreads = 1024;
-constexpr int kFrontLpt = 4;
-constexpr int kFrontTokens = kFrontThreads / kFrontLpt;   // 256
+constexpr int kFrontLpt = 8;                              // at most four groups of logits per lane (E <= 256)
+constexpr int kFrontTokens = 256;                         // largest batch: two passes of 128 tokens through the gate
 constexpr int kFrontWarps = kFrontTokens / 32;            // 8 warps of token threads
 
 template <bool VEC, bool K8>
 __global__ void __launch_bounds__(kFrontThreads)
-front_small_kernel(const float* __restrict__ logits, int T, int E, int K, int R, int C_max, int G,
+front_small_kernel(const float* __restrict__ logits, int T, int E, int K, int R, int C_max, int G, int n_replicas,
                    const int32_t* __restrict__ rep_start, const int32_t* __restrict__ rep_slot,
                    int32_t* __restrict__ topk_idx, float* __restrict__ topk_w, int32_t* __restrict__ row_token,
                    int32_t* __restrict__ inv_row, int32_t* __restrict__ dest_rank, int32_t* __restrict__ seg_offsets_a,
@@ -281,7 +298,11 @@ front_small_kernel(const float* __restrict__ logits, int T, int E, int K, int R,
     __shared__ int32_t warp_sum[kFrontThreads / 32];
     __shared__ uint32_t h_rr[kMaxR * kMaxR];          // [src][dest]
     __shared__ uint32_t h_load[kMaxR];
+    __shared__ int32_t s_rep_start[kMaxE + 1];        // the placement tables, fetched while the gate runs
+    __shared__ int16_t s_rep_slot[kMaxG];
     const int tid = threadIdx.x;
+    for (int i = tid; i <= E; i += kFrontThreads) s_rep_start[i] = __ldg(rep_start + i);
+    for (int i = tid; i < n_replicas; i += kFrontThreads) s_rep_slot[i] = (int16_t)__ldg(rep_slot + i);
 
     for (int i = tid; i < E * kFrontWarps; i += kFrontThreads) (&mask[0][0])[i] = 0u;
     for (int i = tid; i <= G; i += kFrontThreads) s_seg[i] = 0;
@@ -292,13 +313,13 @@ front_small_kernel(const float* __restrict__ logits, int T, int E, int K, int R,
     for (int i = tid; i < R * R; i += kFrontThreads) { dispatch_tokens[i] = 0ull; dispatch_bytes[i] = 0ull; }
 
     // ---- gate (a1) ----
-    {
-        const int t_raw = tid / kFrontLpt, sub = tid % kFrontLpt;
+    for (int t0 = 0; t0 < T; t0 += kFrontThreads / kFrontLpt) {
+        const int t_raw = t0 + tid / kFrontLpt, sub = tid % kFrontLpt;
         const bool live = t_raw < T;
         const int t = live ? t_raw : T - 1;
         int win_idx[8];
         float win_w[8];
-        if (route_token<VEC, kFrontLpt, K8>(logits + (size_t)t * E, E, K, sub, live, status, win_idx, win_w)) {
+        if (route_token<VEC, kFrontLpt, K8, 4>(logits + (size_t)t * E, E, K, sub, live, status, win_idx, win_w)) {
             store_gate(topk_idx + (size_t)t * K, topk_w + (size_t)t * K, K, win_idx, win_w);
 #pragma unroll
             for (int s = 0; s < 8; ++s)
@@ -317,9 +338,9 @@ front_small_kernel(const float* __restrict__ logits, int T, int E, int K, int R,
         int run = 0;
 #pragma unroll
         for (int ww = 0; ww < kFrontWarps; ++ww) { warp_prefix[e][ww] = (uint16_t)run; run += __popc(mask[e][ww]); }
-        const int r0 = __ldg(rep_start + e), r_e = __ldg(rep_start + e + 1) - r0;
+        const int r0 = s_rep_start[e], r_e = s_rep_start[e + 1] - r0;
         for (int q = 0; q < r_e; ++q)                   // replica q gets ceil((N_e - q) / r_e) rows
-            s_seg[__ldg(rep_slot + r0 + q)] = (run > q) ? (run - q + r_e - 1) / r_e : 0;
+            s_seg[s_rep_slot[r0 + q]] = (run > q) ? (run - q + r_e - 1) / r_e : 0;
     }
     __syncthreads();
     // exclusive scan of the G <= 1024 slot lengths: thread g owns slot g
@@ -352,8 +373,8 @@ front_small_kernel(const float* __restrict__ logits, int T, int E, int K, int R,
         for (int s = 0; s < K; ++s) {
             const int e = s_idx[t][s];
             const int n = warp_prefix[e][w] + __popc(mask[e][w] & ((1u << lane) - 1u));
-            const int r0 = __ldg(rep_start + e), r_e = __ldg(rep_start + e + 1) - r0;
-            const int slot = __ldg(rep_slot + r0 + n % r_e);
+            const int r0 = s_rep_start[e], r_e = s_rep_start[e + 1] - r0;
+            const int slot = s_rep_slot[r0 + n % r_e];
             const int row = s_seg[slot] + n / r_e;
             const int dest = slot / C_max;
             row_token[row] = t;
@@ -387,7 +408,8 @@ int launch_front_small(director_ctx* ctx, int T, const float* logits, int32_t* t
     LaunchScope scope(ctx, st, "front_small_kernel");
 #define FRONT_LAUNCH(VEC, K8)                                                                                          \
     front_small_kernel<VEC, K8><<<1, kFrontThreads, 0, st>>>(                                                          \
-        logits, T, s.E, s.K, s.R, s.C_max, ctx->G, ctx->d_rep_start, ctx->d_rep_slot, topk_idx, topk_w, row_token,     \
+        logits, T, s.E, s.K, s.R, s.C_max, ctx->G, ctx->n_replicas, ctx->d_rep_start, ctx->d_rep_slot, topk_idx, topk_w, \
+        row_token,                                                                                                     \
         inv_row, dest_rank, seg_offsets, ctx->d_seg_offsets, reinterpret_cast<unsigned long long*>(workload),          \
         reinterpret_cast<unsigned long long*>(rank_load), reinterpret_cast<unsigned long long*>(dispatch_tokens),      \
         reinterpret_cast<unsigned long long*>(dispatch_bytes), (unsigned long long)s.H * 2ull, ctx->d_status)
