@@ -93,7 +93,7 @@ int director_select_placement(director_ctx* ctx, int32_t slot);
 int director_route(director_ctx* ctx, int32_t T, const float* logits,
                    int32_t* topk_idx, float* topk_w, void* stream);
 
-/* (a2) Dispatch (Section II-B: tokens are packaged and sent to the ranks hosting their experts;
+/* (a2) Dispatch (Section II-B: the first all-to-all moves every token to the ranks that host its experts;
  * here an on-device permutation, the bytes that would cross ranks are counted by
  * director_placement_cost).  Under the default replica policy (see director_set_replica_policy) the n-th
  * assignment of expert e in ascending token order goes to

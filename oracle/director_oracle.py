@@ -45,7 +45,7 @@ def f64_to_bf16_bits(v: np.ndarray) -> np.ndarray:
 
 
 # ----------------------------------------------------------------------------------------------
-# (a1) gating: Section II-A "relevance scores ... top-k routing ... weighted summation"
+# (a1) gating: Section II-A (the gate scores the experts per token, keeps the k best, their scores weight the sum)
 # ----------------------------------------------------------------------------------------------
 
 def route(logits: np.ndarray, K: int):
@@ -73,7 +73,7 @@ def route(logits: np.ndarray, K: int):
 
 
 # ----------------------------------------------------------------------------------------------
-# source ranks: Section VI-A "tokens on GPU j"
+# source ranks: Section VI-A (every token lives on one GPU; W counts tokens per GPU and expert)
 # ----------------------------------------------------------------------------------------------
 
 def source_ranks(T: int, R: int) -> np.ndarray:
@@ -120,7 +120,7 @@ def _slot_of(hosted, C_max: int, rank: int, e: int) -> int:
 
 
 # ----------------------------------------------------------------------------------------------
-# (a2) dispatch: Section II-B "tokens are packaged and sent to the GPUs hosting their experts"
+# (a2) dispatch: Section II-B (first all-to-all: every token travels to the GPUs that host its chosen experts)
 # ----------------------------------------------------------------------------------------------
 
 def dispatch(topk_idx: np.ndarray, X: np.ndarray, C_max: int, x_bits: np.ndarray | None = None,
@@ -255,7 +255,7 @@ def dedup_dispatch_tokens(dest_rank: np.ndarray, src: np.ndarray, R: int) -> np.
 
 
 # ----------------------------------------------------------------------------------------------
-# (a3) expert FFN: Section II-A "experts are FFN sub-networks" (SwiGLU, no bias)
+# (a3) expert FFN: Section II-A (an expert is a feed-forward sub-network; here SwiGLU, no bias)
 # ----------------------------------------------------------------------------------------------
 
 def swiglu_ffn_rows(rows_f64: np.ndarray, wg_bits, wu_bits, wd_bits) -> np.ndarray:

@@ -1,6 +1,5 @@
-// (a4) Weighted un-permute / combine: Section II-A "outputs of these experts are aggregated ...
-// weighted summation based on the scores"; Section II-B: the second all-to-all returns the token
-// outputs to their origin.
+// (a4) Weighted un-permute / combine (Section II-A: a token's result is the sum of its experts' outputs weighted by
+// the gate's scores; Section II-B: the second all-to-all brings those outputs back to the token's rank).
 //
 //   y[t,:] = bf16( sum_s w[t,s] * float(yp[inv_row[t,s],:]) (+ float(y_shared[t,:])) )
 //

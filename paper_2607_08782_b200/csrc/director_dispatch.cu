@@ -1,6 +1,6 @@
 // (a2) Placement-aware dispatch and (a5) placement cost.
 //
-// Dispatch (Section II-B: tokens are packaged and sent to the ranks hosting their experts) is an
+// Dispatch (Section II-B: the first all-to-all moves every token to the ranks that host its experts) is an
 // on-device stable counting sort of the T*K (token, choice) assignments by (destination rank,
 // expert id, token id), followed by the row copies.  The same counting front-end feeds the
 // placement-cost histograms (Section VI-A: workload matrix W, Eq. 1 load, Eq. 3 dispatch volume).

@@ -1,5 +1,5 @@
-// (a1) Top-k softmax gating: Section II-A "the gating network computes relevance scores and
-// selects a small subset of experts ... weighted summation based on the scores".
+// (a1) Top-k softmax gating (Section II-A): the gate scores every expert for a token, the k best are kept and
+// their scores weight the sum of the experts' outputs.
 //
 // LPT lanes per token (1, 2, 4 or 8, chosen from E and T), no data-dependent branches on the common path.
 // A lane streams every LPT-th group of eight logits of its token's row (two 16-byte loads, the next group
