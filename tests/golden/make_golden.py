@@ -31,7 +31,24 @@ def compute() -> dict:
     c = orc.placement_cost(idx, wl.X_primary, s.C_max, s.H)
     yp = orc.expert_ffn(d["xp"], d["seg_offsets"], d["slot_expert"], w.w_gate, w.w_up, w.w_down)
     y = orc.combine(yp, d["inv_row"], w64)
+    # the same routing under a placement with replicas (one more slot per rank), both replica rules
+    N = np.bincount(idx.ravel(), minlength=s.E)
+    Xr = orc.replicate_hottest(N, wl.X_primary, 3)
+    src = orc.source_ranks(s.T, s.R)
+    rr = orc.dispatch(idx, Xr, s.C_max + 1)
+    lf = orc.dispatch(idx, Xr, s.C_max + 1, policy="local_first")
+    replicated = {
+        "placement": Xr.tolist(),
+        "round_robin": {"seg_offsets": rr["seg_offsets"].tolist(), "inv_row_sha256": sha(rr["inv_row"]),
+                        "dispatch_tokens": orc.placement_cost(idx, Xr, s.C_max + 1, s.H)["dispatch_tokens"].tolist(),
+                        "dedup_tokens": orc.dedup_dispatch_tokens(rr["dest_rank"], src, s.R).tolist()},
+        "local_first": {"seg_offsets": lf["seg_offsets"].tolist(), "inv_row_sha256": sha(lf["inv_row"]),
+                        "dispatch_tokens": orc.placement_cost(idx, Xr, s.C_max + 1, s.H,
+                                                              policy="local_first")["dispatch_tokens"].tolist(),
+                        "dedup_tokens": orc.dedup_dispatch_tokens(lf["dest_rank"], src, s.R).tolist()},
+    }
     return {
+        "replicated": replicated,
         "inputs": {"logits_sha256": sha(wl.logits), "x_sha256": sha(wl.x), "w_gate_sha256": sha(w.w_gate),
                    "w_down_sha256": sha(w.w_down), "placement": wl.X_primary.tolist()},
         "topk_idx_first4": idx[:4].tolist(),
