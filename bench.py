@@ -34,10 +34,10 @@ if ROOT not in sys.path:
 METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
-# from the ncu captures summarised under profiles/ (None until a capture for that workload exists).
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from the
+# committed ncu summary of that kernel on that workload (None until a capture for the workload exists).
 NCU_TRAFFIC_BYTES = {
-    # profiles/grouped_gemm_dram_c2_mixtral.md: gate||up GEMM, full-size workload, 2 424 978 176 B read + 230 159 360 B written
+    # gate||up GEMM, full-size workload: 2 420 504 576 B read + 229 234 176 B written
     "c2_mixtral": 2649738752,
 }
 
@@ -53,7 +53,7 @@ REASON_BITS = {
 }
 
 
-def _sample_clocks_main(uuid: str, out_path: str, period_s: float = 0.02):
+def _sample_clocks_main(uuid: str, out_path: str, period_s: float = 0.001):
     """Child process: polls SM clock, power and clock-event reasons of one GPU until SIGTERM."""
     import pynvml
     pynvml.nvmlInit()
@@ -74,7 +74,6 @@ def _sample_clocks_main(uuid: str, out_path: str, period_s: float = 0.02):
             except Exception:
                 power = -1.0
             f.write(f"{time.time():.4f} {sm} {reasons} {power:.1f}\n")
-            f.flush()
             time.sleep(period_s)
 
 
@@ -88,31 +87,38 @@ class ClockSampler:
                 break
             time.sleep(0.02)
 
-    def stop(self, t0: float, t1: float) -> dict:
+    def stop(self) -> None:
+        """Ends the child and reads its samples; window() then summarises any time interval."""
         self.proc.send_signal(signal.SIGTERM)
         try:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.max_mhz, self.samples = None, []
         try:
             lines = open(self.path).read().split("\n")
             os.unlink(self.path)
         except OSError:
-            return out
-        sm, bits, power = [], 0, []
+            return
         for ln in lines:
             p = ln.split()
             if len(p) == 2 and p[0] == "max":
-                out["sm_max_mhz"] = int(p[1])
-            elif len(p) == 4 and t0 <= float(p[0]) <= t1:
-                sm.append(int(p[1]))
-                bits |= int(p[2])
-                power.append(float(p[3]))
-        if sm:
-            out["sm_mhz"] = statistics.median(sm)
-            out["samples"] = len(sm)
-            out["power_w_max"] = max(power)
+                self.max_mhz = int(p[1])
+            elif len(p) == 4:
+                self.samples.append((float(p[0]), int(p[1]), int(p[2]), float(p[3])))
+
+    def window(self, t0: float, t1: float) -> dict:
+        """Median SM clock, clock-event reasons and peak power of the samples taken in [t0, t1] (wall clock)."""
+        out = {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        sel = [smp for smp in self.samples if t0 <= smp[0] <= t1]
+        if sel:
+            bits = 0
+            for smp in sel:
+                bits |= smp[2]
+            out["sm_mhz"] = statistics.median(smp[1] for smp in sel)
+            out["sm_mhz_min"] = min(smp[1] for smp in sel)
+            out["samples"] = len(sel)
+            out["power_w_max"] = max(smp[3] for smp in sel)
             out["reasons"] = [name for bit, name in REASON_BITS.items() if bits & bit and name != "gpu_idle"]
         return out
 
@@ -296,9 +302,33 @@ def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         p = json.load(open(path))
+        under_load = p.get("clocks_under_load", {})
         return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
-                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
-    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                "sm_max_mhz": p.get("sm_max_mhz", 1965.0),
+                "sustained_sm_mhz": under_load.get("sm_mhz_median", 1342.0), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0,
+            "sustained_sm_mhz": 1300.0, "source": "fallback"}
+
+
+def tensor_peak_for_clock(peaks, sm_mhz):
+    """The cuBLAS bf16 ceiling that belongs to the clock regime a kernel was timed in.
+
+    The two measured ceilings were taken at two clocks: the burst figure at the maximum SM clock (a kernel timed
+    alone, before the power cap bites) and the sustained figure at the clock the GPU settles to under the 1 kW cap.
+    A timed region whose median SM clock is within 5 % of the maximum is compared with the burst ceiling, one at or
+    below the sustained clock with the sustained ceiling, and one in between with the straight line between the two
+    points.  Without clock samples the burst ceiling (the stricter one) is used.
+    Returns (peak TFLOP/s, regime name)."""
+    burst, sust = peaks["bf16_tflops"], peaks["bf16_tflops_sustained"]
+    f_max, f_sust = float(peaks["sm_max_mhz"]), float(peaks["sustained_sm_mhz"])
+    if sm_mhz is None:
+        return burst, "burst (no clock samples)"
+    if sm_mhz >= 0.95 * f_max:
+        return burst, "burst"
+    if sm_mhz <= f_sust or f_max <= f_sust:
+        return sust, "sustained"
+    return sust + (burst - sust) * (sm_mhz - f_sust) / (f_max - f_sust), "between"
 
 
 def run_placement_search(args, device):
@@ -512,17 +542,19 @@ def main():
     if graph is not None:                                  # replays launch the kernels recorded in the graph
         launches = args.steps * launches_per_pass
     ms_total = ev0.elapsed_time(ev1)
-    clocks = sampler.stop(wall0, wall1) if sampler else {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
     kernel_ms = {}
+    wallx0 = wallx1 = None
     if graph is None:
         ms, n = layer.d.kernel_time(DOMINANT_KERNEL)
         dominant = (ms / n, n // args.steps) if n else None
         # every kernel, in an extra pass outside the timed region (same steps, events around every launch)
         extra = min(args.steps, 100)
         layer.d.set_profiling(True)
+        wallx0 = time.time()
         for _ in range(extra):
             layer.forward(T, logits, x, fused=args.fused)
         torch.cuda.synchronize()
+        wallx1 = time.time()
         for names in STAGE_KERNELS.values():
             for k in names:
                 ms, n = layer.d.kernel_time(k)
@@ -532,6 +564,13 @@ def main():
             kernel_ms[DOMINANT_KERNEL] = dominant        # the figure from the timed region itself
     layer.d.set_profiling(False)
     layer.d.check_device_status()
+    no_clocks = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    clocks, clocks_extra = dict(no_clocks), dict(no_clocks)
+    if sampler:
+        sampler.stop()
+        clocks = sampler.window(wall0, wall1)
+        if wallx0 is not None:
+            clocks_extra = sampler.window(wallx0, wallx1)
     ms_total = ranks.max_over_ranks(ms_total)
     ms_per_step = ms_total / args.steps
     value = world * T * args.steps / (ms_total * 1e-3)
@@ -593,13 +632,21 @@ def main():
     # with shared experts the kernel is launched twice per step (routed + shared); flops per launch averaged
     gemm1_flop_per_launch = (work["gemm1_flop"] + work["shared_flop"] * 2 / 3) / max(dom_per_step, 1)
     achieved = gemm1_flop_per_launch / (dom_ms * 1e-3) / 1e12 if dom_ms else None
-    peak = peaks["bf16_tflops_sustained"]
+    # the denominator follows the clock regime of the timed region itself (median SM clock sampled inside it; the
+    # dominant kernel is ~63 % of that region, so the region's median is the clock it ran at)
+    peak, regime = tensor_peak_for_clock(peaks, clocks.get("sm_mhz"))
     roofline = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": (achieved / peak) if achieved else None,
                 "traffic": NCU_TRAFFIC_BYTES.get(args.config),
-                "peak_source": f"{peaks['source']} cuBLAS bf16, sustained (kernel timed inside the step)",
+                "regime": regime, "sm_mhz_median": clocks.get("sm_mhz"), "clock_samples": clocks.get("samples", 0),
+                "peak_source": f"{peaks['source']} cuBLAS bf16: burst {peaks['bf16_tflops']} at {peaks['sm_max_mhz']:.0f} MHz, "
+                               f"sustained {peaks['bf16_tflops_sustained']} at {peaks['sustained_sm_mhz']:.0f} MHz; "
+                               "chosen by the median SM clock of the timed region",
                 "flop_per_launch": gemm1_flop_per_launch, "ms_per_launch": dom_ms,
-                "frac_of_burst_peak": (achieved / peaks["bf16_tflops"]) if achieved else None}
+                "mcycles_per_launch": (dom_ms * clocks["sm_mhz"] * 1e-3) if dom_ms and clocks.get("sm_mhz") else None,
+                "frac_of_burst_peak": (achieved / peaks["bf16_tflops"]) if achieved else None,
+                "frac_of_sustained_peak": (achieved / peaks["bf16_tflops_sustained"]) if achieved else None,
+                "frac_of_nominal_2250": (achieved / 2250.0) if achieved else None}
 
     def stage_ms(stage):
         return sum(kernel_ms[k][0] * kernel_ms[k][1] for k in STAGE_KERNELS[stage] if k in kernel_ms)
@@ -612,7 +659,8 @@ def main():
         if ms <= 0:
             continue
         rate = work[key] / (ms * 1e-3) / (1e9 if unit == "GB/s" else 1e12)
-        pk = peaks["hbm_gbs"] if unit == "GB/s" else peaks["bf16_tflops_sustained"]
+        # stage times come from the extra pass (events around every launch): its own clock window picks the ceiling
+        pk = peaks["hbm_gbs"] if unit == "GB/s" else tensor_peak_for_clock(peaks, clocks_extra.get("sm_mhz"))[0]
         stages[stage] = {"ms": round(ms, 4), "rate": round(rate, 2), "unit": unit, "frac_of_measured_peak": round(rate / pk, 4)}
     kernels = {k: {"ms_per_launch": round(v[0], 4), "launches_per_step": v[1]} for k, v in kernel_ms.items()}
 
@@ -637,7 +685,7 @@ def main():
                    "l2": "inputs larger than L2: every step streams the expert weights "
                          f"({3 * s.E * s.F * s.H * 2 / 1e9:.2f} GB) and activations through HBM",
                    "parallelism": "single GPU, logical ranks" if world == 1 else f"{world} independent replicas"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "cuda_graph": bool(args.graph), "roofline": roofline,
+        "clocks": clocks, "clocks_stage_pass": clocks_extra, "e2e": e2e, "gpu_launches": int(launches), "cuda_graph": bool(args.graph), "roofline": roofline,
         "cpu_baseline": cpu_baseline, "stages": stages, "kernels": kernels,
         "ffn_tflops": round(work["ffn_flop"] / (stage_ms("expert_ffn") * 1e-3) / 1e12, 1) if stage_ms("expert_ffn") else None,
     }

@@ -268,9 +268,13 @@ int director_layer_forward_host(director_ctx* ctx, int32_t T, const float* logit
  * on an internal copy stream, the kernels on `stream` and the device->host copies on a second internal
  * copy stream, chained by events, and returns at once with a ticket; wait blocks until that batch's
  * results are in its host buffers.  Inputs, y and the histograms are double-buffered on the device, so
- * the copies of batch i+1 and of batch i-1 run while the kernels of batch i do.  At most two batches
- * may be in flight: wait for ticket i-1 (at the latest) before submitting batch i+1.  The host buffers
- * of a batch (pinned, for real overlap) must stay valid and untouched until its wait returns.
+ * the copies of batch i+1 and of batch i-1 run while the kernels of batch i do.  Two batches can be in
+ * flight: wait for ticket i-1 (at the latest) before submitting batch i+1.  A submit issued while two
+ * batches are still undelivered does not fail: it blocks on the host until the older of them has reached
+ * its host buffers (so it degrades to a synchronous call), and a later wait for that ticket returns at
+ * once.  wait never returns DIRECTOR_OK before the batch's y and histograms are in host memory.  The host
+ * buffers of a batch (pinned, for real overlap) must stay valid and untouched until its wait returns or
+ * until two later submits have returned.
  * Arguments as for director_layer_forward_host; ticket: host, receives the batch's sequence number. */
 int director_layer_submit_host(director_ctx* ctx, int32_t T, const float* logits, const void* x,
                                const void* w_gate, const void* w_up, const void* w_down,
@@ -282,6 +286,16 @@ int director_layer_wait_host(director_ctx* ctx, int64_t ticket);
 /* Synchronises `stream`, returns the sticky device status word (DIRECTOR_OK if clean) and
  * clears it. */
 int director_last_status(director_ctx* ctx, void* stream);
+
+/* Self-test of the failure-detection path (not part of the layer).  Every wait inside the GEMM pipelines
+ * is bounded: when a wait runs out, the waiting role raises its CTA's abort flag, every role leaves its
+ * loop, and the kernel records DIRECTOR_ERR_TIMEOUT in the sticky status word instead of hanging the
+ * GPU.  This call launches a one-warp kernel that waits, with that same helper, on an mbarrier nobody
+ * arrives at, for at most limit_ns (1 us .. 100 ms) - so the wait expires by construction, harmlessly.
+ * Afterwards director_last_status returns DIRECTOR_ERR_TIMEOUT once, then DIRECTOR_OK, and the context
+ * is usable as before.  waited_ns: dev uint64 [1] or NULL, receives the nanoseconds the wait lasted.
+ * Returns DIRECTOR_ERR_INVALID_ARG for a limit outside the range. */
+int director_selftest_bounded_wait(director_ctx* ctx, uint64_t limit_ns, uint64_t* waited_ns, void* stream);
 
 /* Tile scheme of the expert-FFN GEMMs (results are bit-identical across schemes):
  *   2 (default) weight-stationary CTA pairs: 256 weight rows x up to 256 tokens per tile, the token count

@@ -27,6 +27,7 @@ EXPORTED = (
     "director_expert_ffn_gather", "director_set_replica_policy", "director_dispatch_src",
     "director_dedup_dispatch_tokens", "director_route_dispatch_cost", "director_layer_forward",
     "director_reserve_placements", "director_select_placement", "director_set_profiling_filter",
+    "director_selftest_bounded_wait",
 )
 
 REPLICA_ROUND_ROBIN, REPLICA_LOCAL_FIRST = 0, 1
@@ -81,6 +82,7 @@ def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.director_route_dispatch_cost.argtypes = [vp, c_int32] + [vp] * 14
     lib.director_dispatch_src.argtypes = [vp, c_int32] + [vp] * 9
     lib.director_dedup_dispatch_tokens.argtypes = [vp, c_int32, vp, vp, vp, vp]
+    lib.director_selftest_bounded_wait.argtypes = [vp, c_uint64, vp, vp]
     lib.director_kernel_time.argtypes = [vp, c_char_p, POINTER(c_int64)]
     lib.director_kernel_time.restype = c_double
     lib.director_status_string.argtypes = [c_int]
@@ -240,6 +242,11 @@ class Director:
 
     def check_device_status(self):
         _check(self.last_status(), "device status")
+
+    def selftest_bounded_wait(self, limit_ns: int, waited_ns=None):
+        """Launches the kernel whose bounded wait expires by construction (see director_selftest_bounded_wait)."""
+        _check(self.lib.director_selftest_bounded_wait(self._ctx, int(limit_ns), _ptr(waited_ns), _stream()),
+               "director_selftest_bounded_wait")
 
     def set_ffn_variant(self, variant: int):
         _check(self.lib.director_set_ffn_variant(self._ctx, variant), "director_set_ffn_variant")

@@ -468,6 +468,14 @@ int director_layer_submit_host(director_ctx* ctx, int32_t T, const float* logits
     int64_t* c_tok = c_load + s.R;
     uint64_t* c_bytes = reinterpret_cast<uint64_t*>(c_tok + (size_t)s.R * s.R);
 
+    // This slot's previous batch (two submissions ago) must have reached the host before its buffers are reused.  A
+    // caller that keeps at most two batches in flight has already waited for it; one that has not is held here, on the
+    // host, until that batch's copies have landed - so a ticket never reads as complete before its data is.
+    const int64_t prev = ctx->submitted - 2;
+    if (prev >= 0 && ctx->waited[slot] < prev) {
+        if (cudaEventSynchronize(ctx->ev_d2h_done[slot]) != cudaSuccess) return DIRECTOR_ERR_CUDA;
+        ctx->waited[slot] = prev;
+    }
     // inputs: wait until the kernels of the batch that used this slot two submissions ago are done with it
     if (cudaStreamWaitEvent(ctx->h2d_stream, ctx->ev_compute_done[slot], 0) != cudaSuccess ||
         cudaMemcpyAsync(d_logits, logits, sizeof(float) * (size_t)T * s.E, cudaMemcpyHostToDevice, ctx->h2d_stream) != cudaSuccess ||
@@ -509,8 +517,12 @@ int director_layer_submit_host(director_ctx* ctx, int32_t T, const float* logits
 int director_layer_wait_host(director_ctx* ctx, int64_t ticket) {
     REQUIRE_CTX(ctx);
     if (ticket < 0 || ticket >= ctx->submitted) return DIRECTOR_ERR_INVALID_ARG;
-    if (ticket + 2 < ctx->submitted) return DIRECTOR_OK;   // its slot was reused, which waited for it
-    return cuda_status(cudaEventSynchronize(ctx->ev_d2h_done[ticket & 1]));
+    const int slot = (int)(ticket & 1);
+    if (ctx->waited[slot] >= ticket) return DIRECTOR_OK;   // already delivered (waited for, or its slot was reused since)
+    if (cudaEventSynchronize(ctx->ev_d2h_done[slot]) != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    // the event now belongs to the newest batch of this slot, so every ticket of the slot up to that one is in host memory
+    ctx->waited[slot] = ((ctx->submitted - 1) & 1) == slot ? ctx->submitted - 1 : ctx->submitted - 2;
+    return DIRECTOR_OK;
 }
 
 int director_layer_forward(director_ctx* ctx, int32_t T, const float* logits, const void* x, const void* w_gate,

@@ -79,6 +79,7 @@ struct director_ctx {
     cudaEvent_t ev_h2d_done[2] = {nullptr, nullptr}, ev_compute_done[2] = {nullptr, nullptr},
                 ev_d2h_done[2] = {nullptr, nullptr};
     int64_t submitted = 0;
+    int64_t waited[2] = {-1, -1};      // per buffer slot: newest ticket known to have reached host memory
     int32_t* e_topk_idx = nullptr;
     float* e_topk_w = nullptr;
     void* e_xp = nullptr;

@@ -427,8 +427,7 @@ int launch_route(director_ctx* ctx, int T, const float* logits, int32_t* topk_id
     const int groups = (E + 7) / 8;
     int lpt = 1;
     while (lpt < 8 && 2 * lpt <= groups && ((long long)T * lpt < 131072 || groups > 4 * lpt)) lpt *= 2;
-    if (T >= (1 << 19)) lpt = 1;
-    if (const char* ov = getenv("XLPT")) lpt = atoi(ov);   // far above the launch-latency regime a lane per token executes the fewest instructions
+    if (T >= (1 << 19)) lpt = 1;   // far above the launch-latency regime a lane per token executes the fewest instructions
     const long long threads = (long long)T * lpt;
     const dim3 grid((unsigned)((threads + kRouteThreads - 1) / kRouteThreads)), block(kRouteThreads);
     LaunchScope scope(ctx, st, "route_topk_kernel");

@@ -50,18 +50,23 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait.  Returns false if the wait expired or another role of this CTA already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded wait.  Returns false if the wait expired (limit_ns of the global timer) or another role of this CTA
+// already gave up; the caller then stops issuing work, and the kernel reports DIRECTOR_ERR_TIMEOUT.
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                unsigned long long limit_ns) {
     if (mbar_try(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     uint32_t n = 0;
     while (!mbar_try(bar, parity)) {
         if ((++n & 63u) == 0u) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
+            if (global_ns() - t0 > limit_ns) { *abort_flag = 1; return false; }
         }
     }
     return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    return mbar_wait_limit(bar, parity, abort_flag, WAIT_LIMIT_NS);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {

@@ -48,3 +48,17 @@ def test_cuda_arm_refuses_to_run_without_a_device():
     r = _run(["--config", "c1_tiny", "--steps", "1", "--warmup", "0"])
     assert r.returncode != 0
     assert "CUDA" in (r.stderr + r.stdout)
+
+
+def test_roofline_denominator_follows_the_sampled_clock():
+    """The tensor ceiling bench.py divides by is the one measured in the clock regime of the timed region."""
+    sys.path.insert(0, ROOT)
+    import bench
+    peaks = {"bf16_tflops": 1600.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 2000.0, "sustained_sm_mhz": 1300.0}
+    assert bench.tensor_peak_for_clock(peaks, 2000.0) == (1600.0, "burst")
+    assert bench.tensor_peak_for_clock(peaks, 1905.0) == (1600.0, "burst")           # within 5 % of the maximum
+    assert bench.tensor_peak_for_clock(peaks, 1300.0) == (1400.0, "sustained")
+    assert bench.tensor_peak_for_clock(peaks, 1200.0) == (1400.0, "sustained")
+    pk, regime = bench.tensor_peak_for_clock(peaks, 1650.0)                           # half way between the two clocks
+    assert regime == "between" and abs(pk - 1500.0) < 1e-9
+    assert bench.tensor_peak_for_clock(peaks, None)[0] == 1600.0                      # no samples: the stricter ceiling

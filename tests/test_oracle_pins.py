@@ -403,6 +403,38 @@ def test_cost_one_rank_is_all_local_and_source_partition():
     assert np.bincount(orc.source_ranks(10, 4)).tolist() == [3, 2, 3, 2]
 
 
+def test_cost_summary_reductions_against_hand_written_numbers():
+    """Eq. 2's straggler load and Eq. 4's send volumes on a 3-rank example worked by hand.  Row sums,
+    column sums, diagonal, maximum and total all differ, so `sum` for `max`, rows for columns, or a
+    diagonal left in would each fail."""
+    #   tokens sent j -> k            off-diagonal of row j     column sums (= lambda_k, Eq. 1)
+    D_tokens = np.array([[5, 2, 1],   # 2 + 1 = 3               5 + 0 + 3 = 8
+                         [0, 7, 4],   # 0 + 4 = 4               2 + 7 + 3 = 12
+                         [3, 3, 0]],  # 3 + 3 = 6               1 + 4 + 0 = 5
+                        dtype=np.int64)
+    d = 8                             # bytes per token: H = 4 hidden values of 2 bytes
+    cost = dict(rank_load=D_tokens.sum(axis=0), dispatch_tokens=D_tokens,
+                dispatch_bytes=(D_tokens * d).astype(np.uint64))
+    s = orc.cost_summary(cost)
+    assert s["max_rank_load"] == 12                       # Eq. 2: the straggler executes 12 assignments
+    assert s["send_bytes"].tolist() == [24, 32, 48]       # Eq. 4: sum over k != j of D[j,k], in bytes
+    assert s["max_send_bytes"] == 48                      # the straggler sender (rank 2), not the total
+    assert s["cross_rank_bytes"] == 104                   # 24 + 32 + 48; the diagonal (5, 7, 0) is local
+    # the same quantities through placement_cost on an assignment list that realises this D exactly:
+    # K = 1, single-copy placement expert k -> rank k, so D[j,k] = tokens of rank j that chose expert k
+    src, idx = [], []
+    for j in range(3):
+        for k in range(3):
+            src += [j] * int(D_tokens[j, k])
+            idx += [k] * int(D_tokens[j, k])
+    c = orc.placement_cost(np.array(idx, dtype=np.int32)[:, None], np.eye(3, dtype=np.uint8), 1, 4,
+                           np.array(src, dtype=np.int32))
+    assert np.array_equal(c["dispatch_tokens"], D_tokens) and c["rank_load"].tolist() == [8, 12, 5]
+    s2 = orc.cost_summary(c)
+    assert (s2["max_rank_load"], s2["max_send_bytes"], s2["cross_rank_bytes"]) == (12, 48, 104)
+    assert s2["send_bytes"].tolist() == [24, 32, 48]
+
+
 # ------------------------------------------------------------------- balanced placement input
 
 def test_balanced_placement_is_valid_and_near_brute_force_optimum_on_c1():

@@ -5,12 +5,13 @@ device heap, loops that must never wait on the allocator, processes with a fixed
 cannot create a context, because creating one allocates its workspace.  This entry point keeps its
 scratch in a fixed array inside the library instead.  The test calls it through the C ABI twice in a
 row, on two different batches, and requires bit-identical results to director_dispatch (the existing,
-context-based entry point), and that the device's free memory does not change across the calls.
+context-based entry point) and to the CPU oracle's permutation, and that the device's free memory does not change across the calls.
 
 The file name makes pytest collect it after every other test file."""
 import numpy as np
 import pytest
 
+from oracle import director_oracle as orc
 from paper_2607_08782_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -73,6 +74,12 @@ def test_static_entry_point_matches_director_dispatch_on_two_calls_in_a_row():
         assert torch.equal(inv_row, layer.inv_row[:T]), f"call {call}: inv_row"
         assert torch.equal(dest_rank, layer.dest_rank[:T]), f"call {call}: dest_rank"
         assert int(seg_offsets[-1]) == A
+        # and directly against the CPU oracle's definition of the permutation
+        d_o = orc.dispatch(layer.topk_idx[:T].cpu().numpy(), X, C)
+        assert np.array_equal(seg_offsets.cpu().numpy(), d_o["seg_offsets"]), f"call {call}: seg_offsets vs oracle"
+        assert np.array_equal(row_token.cpu().numpy(), d_o["row_token"]), f"call {call}: row_token vs oracle"
+        assert np.array_equal(inv_row.cpu().numpy(), d_o["inv_row"]), f"call {call}: inv_row vs oracle"
+        assert np.array_equal(dest_rank.cpu().numpy(), d_o["dest_rank"]), f"call {call}: dest_rank vs oracle"
 
 
 def test_static_entry_point_rejects_problems_beyond_its_fixed_scratch():
