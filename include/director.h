@@ -306,6 +306,14 @@ int director_selftest_bounded_wait(director_ctx* ctx, uint64_t limit_ns, uint64_
  * (their addresses differ by 2^40 bytes or more). */
 int director_set_ffn_variant(director_ctx* ctx, int32_t variant);
 
+/* SM clock the expert GEMMs really ran at.  Every CTA of a grouped-GEMM launch reads the SM cycle counter and
+ * the global nanosecond timer when it starts and when it ends; this call synchronises the device and returns
+ * (sum of cycles) / (sum of nanoseconds) over the CTAs of the context's most recent launch, in MHz.
+ * which: 0 = gate|up GEMM, 1 = down GEMM.  busy_us: host, or NULL; receives the longest CTA's time in
+ * microseconds.  A host-side clock sampler has millisecond resolution and lags; this is the clock during
+ * the kernel itself, the one a tensor-pipe roofline has to be read against.  Negative on error. */
+double director_gemm_sm_mhz(director_ctx* ctx, int32_t which, double* busy_us);
+
 /* Number of kernels this context has launched since it was created. */
 int64_t director_launch_count(const director_ctx* ctx);
 

@@ -27,7 +27,7 @@ EXPORTED = (
     "director_expert_ffn_gather", "director_set_replica_policy", "director_dispatch_src",
     "director_dedup_dispatch_tokens", "director_route_dispatch_cost", "director_layer_forward",
     "director_reserve_placements", "director_select_placement", "director_set_profiling_filter",
-    "director_selftest_bounded_wait",
+    "director_selftest_bounded_wait", "director_gemm_sm_mhz",
 )
 
 REPLICA_ROUND_ROBIN, REPLICA_LOCAL_FIRST = 0, 1
@@ -83,12 +83,14 @@ def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.director_dispatch_src.argtypes = [vp, c_int32] + [vp] * 9
     lib.director_dedup_dispatch_tokens.argtypes = [vp, c_int32, vp, vp, vp, vp]
     lib.director_selftest_bounded_wait.argtypes = [vp, c_uint64, vp, vp]
+    lib.director_gemm_sm_mhz.argtypes = [vp, c_int32, POINTER(c_double)]
+    lib.director_gemm_sm_mhz.restype = c_double
     lib.director_kernel_time.argtypes = [vp, c_char_p, POINTER(c_int64)]
     lib.director_kernel_time.restype = c_double
     lib.director_status_string.argtypes = [c_int]
     lib.director_status_string.restype = c_char_p
     for name in EXPORTED:
-        if name not in ("director_launch_count", "director_kernel_time", "director_status_string"):
+        if name not in ("director_launch_count", "director_kernel_time", "director_status_string", "director_gemm_sm_mhz"):
             getattr(lib, name).restype = c_int
     _lib = lib
     return lib
@@ -250,6 +252,15 @@ class Director:
 
     def set_ffn_variant(self, variant: int):
         _check(self.lib.director_set_ffn_variant(self._ctx, variant), "director_set_ffn_variant")
+
+    def gemm_sm_mhz(self, which: int = 0):
+        """(SM MHz, longest CTA's microseconds) of the most recent gate|up (0) or down (1) GEMM launch, measured
+        by the kernel itself (cycle counter against the global timer)."""
+        busy = c_double(0.0)
+        mhz = float(self.lib.director_gemm_sm_mhz(self._ctx, which, ctypes.byref(busy)))
+        if mhz < 0:
+            raise DirectorError(4, "director_gemm_sm_mhz")
+        return mhz, float(busy.value)
 
     def launch_count(self) -> int:
         return int(self.lib.director_launch_count(self._ctx))

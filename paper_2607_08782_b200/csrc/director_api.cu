@@ -3,6 +3,7 @@
 // director_<stage>.cu files.
 #include "director_common.cuh"
 
+#include <algorithm>
 #include <cstring>
 #include <new>
 
@@ -39,7 +40,7 @@ void free_all(director_ctx* c) {
             if (p) cudaFree(p);
     }
     void* ptrs[] = {c->d_tile_counts, c->d_seg_offsets, c->d_ticket, c->d_tile_rep,
-                    c->d_status, c->d_hidden, c->d_hidden_shared, c->d_one_seg, c->d_sched,
+                    c->d_status, c->d_hidden, c->d_hidden_shared, c->d_one_seg, c->d_sched, c->d_gemm_clock,
                     c->d_zero_expert, c->e_logits2[0], c->e_logits2[1], c->e_x2[0], c->e_x2[1], c->e_topk_idx,
                     c->e_topk_w, c->e_xp, c->e_yp, c->e_y2[0], c->e_y2[1], c->e_y_shared, c->e_row_token, c->e_inv_row,
                     c->e_dest_rank, c->e_cost2[0], c->e_cost2[1]};
@@ -124,6 +125,7 @@ int director_create(const director_shape* shape, director_ctx** out) {
               dev_alloc(&c->d_host_mask, s.E) && dev_alloc(&c->d_tile_rep, (size_t)c->n_tiles_max * c->G) &&
               dev_alloc(&c->d_one_seg, 2) && dev_alloc(&c->d_sched, 4) &&
               dev_alloc(&c->d_zero_expert, 1) &&
+              dev_alloc(&c->d_gemm_clock, 4 * (size_t)kGemmClockCtas) &&
               dev_alloc(reinterpret_cast<uint16_t**>(&c->d_hidden), A * s.F) &&
               dev_alloc(reinterpret_cast<uint16_t**>(&c->d_hidden_shared), T * s.S * s.F) &&
               dev_alloc(&c->e_logits2[0], T * s.E) && dev_alloc(&c->e_logits2[1], T * s.E) &&
@@ -146,7 +148,8 @@ int director_create(const director_shape* shape, director_ctx** out) {
     c->bank.push_back({c->d_rep_start, c->d_rep_slot, c->d_slot_expert, c->d_host_mask, 0, false});
     ok = cudaMemset(c->d_ticket, 0, sizeof(unsigned int)) == cudaSuccess &&
          cudaMemset(c->d_status, 0, sizeof(int32_t)) == cudaSuccess &&
-         cudaMemset(c->d_zero_expert, 0, sizeof(int32_t)) == cudaSuccess;
+         cudaMemset(c->d_zero_expert, 0, sizeof(int32_t)) == cudaSuccess &&
+         cudaMemset(c->d_gemm_clock, 0, sizeof(unsigned long long) * 4 * kGemmClockCtas) == cudaSuccess;
 
     cudaDriverEntryPointQueryResult qres;
     if (ok) {
@@ -583,12 +586,32 @@ int director_last_status(director_ctx* ctx, void* stream) {
 
 int director_set_ffn_variant(director_ctx* ctx, int32_t variant) {
     REQUIRE_CTX(ctx);
-    if (variant < 0 || variant > 2) return DIRECTOR_ERR_INVALID_ARG;
-    ctx->ffn_variant = variant;
+    if (variant < 0 || variant > 5) return DIRECTOR_ERR_INVALID_ARG;
+    // 3, 4, 5: scheme 2 with two token tiles per work item in both GEMMs / the gate|up GEMM only / the down GEMM only
+    ctx->ffn_dual = variant == 3 ? 3 : variant == 4 ? 1 : variant == 5 ? 2 : 0;
+    ctx->ffn_variant = variant > 2 ? 2 : variant;
     return DIRECTOR_OK;
 }
 
 int director_pair_clusters(const director_ctx* ctx) { return ctx ? ctx->pair_clusters : -1; }
+
+double director_gemm_sm_mhz(director_ctx* ctx, int32_t which, double* busy_us) {
+    if (ctx == nullptr || which < 0 || which > 1) return -1.0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return -1.0;
+    std::vector<unsigned long long> h(2 * (size_t)kGemmClockCtas);
+    if (cudaMemcpy(h.data(), ctx->d_gemm_clock + (size_t)which * 2 * kGemmClockCtas, h.size() * sizeof(unsigned long long),
+                   cudaMemcpyDeviceToHost) != cudaSuccess)
+        return -1.0;
+    const int ctas = std::min(2 * ctx->pair_clusters, (int)kGemmClockCtas);
+    double cycles = 0.0, ns = 0.0, ns_max = 0.0;
+    for (int i = 0; i < ctas; ++i) {
+        cycles += (double)h[2 * i];
+        ns += (double)h[2 * i + 1];
+        ns_max = std::max(ns_max, (double)h[2 * i + 1]);
+    }
+    if (busy_us) *busy_us = ns_max * 1e-3;
+    return ns > 0.0 ? cycles / ns * 1e3 : 0.0;
+}
 
 int64_t director_launch_count(const director_ctx* ctx) { return ctx ? ctx->launches : -1; }
 

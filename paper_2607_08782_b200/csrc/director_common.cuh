@@ -19,6 +19,7 @@ constexpr int kMaxK = 8;
 constexpr int kMaxR = 64;
 constexpr int kMaxC = 16;
 constexpr int kMaxG = kMaxR * kMaxC;
+constexpr int kGemmClockCtas = 512;   // CTAs per GEMM launch whose {cycles, ns} records fit the clock buffer
 
 struct KernelEvent {
     const char* name;
@@ -68,6 +69,7 @@ struct director_ctx {
     unsigned int* d_sched = nullptr;   // [4] work-item counters of the GEMM launches of one expert_ffn call
     int32_t* d_one_seg = nullptr;      // [2] segment table {0, T} used for the shared experts
     int32_t* d_zero_expert = nullptr;  // [1] = {0}
+    unsigned long long* d_gemm_clock = nullptr;   // [2][kGemmClockCtas][2] {SM cycles, ns} per CTA of the last gate|up / down launch
 
     // buffers of the host-buffer entry points; inputs, y and the histograms exist twice so that the
     // copies of one batch overlap the kernels of its neighbours
@@ -91,6 +93,7 @@ struct director_ctx {
 
     int pair_clusters = 0;              // CTA pairs the device can hold at once (pair variant's grid)
     int ffn_variant = 2;                // tile scheme of the expert-FFN GEMMs, see director_set_ffn_variant
+    int ffn_dual = 0;                   // bit 0 / bit 1: the gate|up / down GEMM takes two token tiles per work item
     void* encode_tiled = nullptr;       // cuTensorMapEncodeTiled, resolved through the runtime
 
     int64_t launches = 0;
