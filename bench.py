@@ -289,7 +289,7 @@ DOMINANT_KERNEL = "grouped_gemm_swiglu_kernel"      # the gate||up grouped GEMM:
 
 STAGE_KERNELS = {
     "route": ["route_topk_kernel", "front_small_kernel"],   # the fused front end (T <= 256) is booked under route
-    "dispatch": ["dispatch_count_scan_kernel", "dispatch_index_kernel", "dispatch_scatter_rows_kernel",
+    "dispatch": ["dispatch_plan_kernel", "dispatch_count_scan_kernel", "dispatch_index_kernel", "dispatch_scatter_rows_kernel",
                  "dispatch_travel_count_scan_kernel", "dispatch_slot_count_scan_kernel", "dispatch_local_index_kernel"],
     "expert_ffn": ["grouped_gemm_swiglu_kernel", "grouped_gemm_down_kernel", "one_segment_kernel"],
     "combine": ["combine_kernel"],
@@ -552,6 +552,7 @@ def main():
     except Exception:
         kernel_clock = None
     kernel_ms = {}
+    stage_ms_measured = {}
     wallx0 = wallx1 = None
     if graph is None:
         ms, n = layer.d.kernel_time(DOMINANT_KERNEL)
@@ -571,6 +572,20 @@ def main():
                     kernel_ms[k] = (ms / n, n // extra)
         if dominant:
             kernel_ms[DOMINANT_KERNEL] = dominant        # the figure from the timed region itself
+        # every stage, in a third pass: ONE pair of events around all launches of a stage, so a stage of several small
+        # kernels pays the bracket once (a pair of events around a microsecond kernel costs as much as the kernel)
+        layer.d.set_profiling(2)
+        for _ in range(extra):
+            layer.forward(T, logits, x, fused=args.fused)
+        torch.cuda.synchronize()
+        wallx1 = time.time()
+        for stage in STAGE_KERNELS:
+            ms, n = layer.d.kernel_time("stage_" + stage)
+            if n:
+                stage_ms_measured[stage] = ms / extra
+        ms, n = layer.d.kernel_time("stage_front_small")
+        if n:
+            stage_ms_measured["front_small"] = ms / extra
     layer.d.set_profiling(False)
     layer.d.check_device_status()
     no_clocks = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
@@ -665,6 +680,10 @@ def main():
                 "frac_of_nominal_2250": (achieved / 2250.0) if achieved else None}
 
     def stage_ms(stage):
+        """Time of a stage per step: its own bracket (one pair of events around all its launches) when that pass ran,
+        else the sum of its individually bracketed kernels."""
+        if stage in stage_ms_measured and stage != "expert_ffn":   # the GEMMs are long: their kernel brackets are exact
+            return stage_ms_measured[stage]
         return sum(kernel_ms[k][0] * kernel_ms[k][1] for k in STAGE_KERNELS[stage] if k in kernel_ms)
 
     stages = {}
@@ -677,7 +696,13 @@ def main():
         rate = work[key] / (ms * 1e-3) / (1e9 if unit == "GB/s" else 1e12)
         # stage times come from the extra pass (events around every launch): its own clock window picks the ceiling
         pk = peaks["hbm_gbs"] if unit == "GB/s" else tensor_peak_for_clock(peaks, clocks_extra.get("sm_mhz"))[0]
-        stages[stage] = {"ms": round(ms, 4), "rate": round(rate, 2), "unit": unit, "frac_of_measured_peak": round(rate / pk, 4)}
+        stages[stage] = {"ms": round(ms, 4), "rate": round(rate, 2), "unit": unit, "frac_of_measured_peak": round(rate / pk, 4),
+                         "timing": "one event pair around the stage" if stage in stage_ms_measured and stage != "expert_ffn" else "sum of per-kernel event pairs",
+                         "ms_sum_of_kernel_brackets": round(sum(kernel_ms[k][0] * kernel_ms[k][1] for k in STAGE_KERNELS[stage]
+                                                                 if k in kernel_ms), 4)}
+    if "front_small" in stage_ms_measured:
+        stages["front_small"] = {"ms": round(stage_ms_measured["front_small"], 4), "unit": "ms",
+                                 "what": "gate + dispatch indices + placement cost of a decode batch in one launch"}
     kernels = {k: {"ms_per_launch": round(v[0], 4), "launches_per_step": v[1]} for k, v in kernel_ms.items()}
 
     # ---- CPU baseline: the oracle on a bounded sample, on this machine's host cores ----

@@ -317,10 +317,13 @@ double director_gemm_sm_mhz(director_ctx* ctx, int32_t which, double* busy_us);
 /* Number of kernels this context has launched since it was created. */
 int64_t director_launch_count(const director_ctx* ctx);
 
-/* Per-kernel device timing.  While enabled, every launch is bracketed by CUDA events on its
- * stream.  director_kernel_time synchronises the device, then returns the summed duration in
- * milliseconds and the number of launches of the kernels whose name contains `name_substr`
- * since profiling was last enabled; returns a negative value on error. */
+/* Device timing.  enabled = 1: every kernel launch is bracketed by CUDA events on its stream.  enabled = 2:
+ * every STAGE (route, dispatch, expert FFN, combine, placement cost; all kernels and memsets of the stage) is
+ * bracketed by one pair of events, recorded under the names "stage_route", "stage_dispatch", "stage_expert_ffn",
+ * "stage_combine", "stage_placement_cost" ("stage_front_small" for the one-launch front end of decode batches) -
+ * the stage's time on an otherwise idle stream with the event pair paid once.  enabled = 0: off.
+ * director_kernel_time synchronises the device, then returns the summed duration in milliseconds and the
+ * number of brackets whose name contains `name_substr` since profiling was last enabled; negative on error. */
 int director_set_profiling(director_ctx* ctx, int32_t enabled);
 /* Restricts the timing to kernels whose name contains `name_substr` (NULL or "" = all kernels): two event records
  * per launch are cheap but not free, and a measurement that wants one kernel's duration inside an otherwise

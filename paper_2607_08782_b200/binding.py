@@ -265,11 +265,12 @@ class Director:
     def launch_count(self) -> int:
         return int(self.lib.director_launch_count(self._ctx))
 
-    def set_profiling(self, enabled: bool, only: str | None = None):
-        """Per-kernel device timing on/off; `only`: time just the kernels whose name contains this string."""
+    def set_profiling(self, enabled, only: str | None = None):
+        """Device timing: True / 1 = events around every kernel, 2 = one pair of events around every stage, False /
+        0 = off; `only`: time just the kernels whose name contains this string (per-kernel mode)."""
         _check(self.lib.director_set_profiling_filter(self._ctx, only.encode() if only else None),
                "director_set_profiling_filter")
-        _check(self.lib.director_set_profiling(self._ctx, 1 if enabled else 0), "director_set_profiling")
+        _check(self.lib.director_set_profiling(self._ctx, int(enabled)), "director_set_profiling")
 
     def kernel_time(self, name_substr: str):
         """(total milliseconds, launches) of kernels whose name contains name_substr since profiling was enabled."""

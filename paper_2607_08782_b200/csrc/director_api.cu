@@ -121,7 +121,7 @@ int director_create(const director_shape* shape, director_ctx** out) {
 
     bool ok = dev_alloc(&c->d_rep_start, s.E + 1) && dev_alloc(&c->d_rep_slot, (size_t)s.E * s.R) &&
               dev_alloc(&c->d_slot_expert, c->G) && dev_alloc(&c->d_tile_counts, (size_t)c->n_tiles_max * s.E) &&
-              dev_alloc(&c->d_seg_offsets, c->G + 1) && dev_alloc(&c->d_ticket, 1) && dev_alloc(&c->d_status, 1) &&
+              dev_alloc(&c->d_seg_offsets, c->G + 1) && dev_alloc(&c->d_ticket, 4) && dev_alloc(&c->d_status, 1) &&
               dev_alloc(&c->d_host_mask, s.E) && dev_alloc(&c->d_tile_rep, (size_t)c->n_tiles_max * c->G) &&
               dev_alloc(&c->d_one_seg, 2) && dev_alloc(&c->d_sched, 4) &&
               dev_alloc(&c->d_zero_expert, 1) &&
@@ -146,7 +146,7 @@ int director_create(const director_shape* shape, director_ctx** out) {
         return DIRECTOR_ERR_WORKSPACE;
     }
     c->bank.push_back({c->d_rep_start, c->d_rep_slot, c->d_slot_expert, c->d_host_mask, 0, false});
-    ok = cudaMemset(c->d_ticket, 0, sizeof(unsigned int)) == cudaSuccess &&
+    ok = cudaMemset(c->d_ticket, 0, 4 * sizeof(unsigned int)) == cudaSuccess &&
          cudaMemset(c->d_status, 0, sizeof(int32_t)) == cudaSuccess &&
          cudaMemset(c->d_zero_expert, 0, sizeof(int32_t)) == cudaSuccess &&
          cudaMemset(c->d_gemm_clock, 0, sizeof(unsigned long long) * 4 * kGemmClockCtas) == cudaSuccess;
@@ -157,7 +157,7 @@ int director_create(const director_shape* shape, director_ctx** out) {
                                               &qres) == cudaSuccess &&
              qres == cudaDriverEntryPointSuccess && c->encode_tiled != nullptr;
     }
-    if (ok) ok = ffn_init(c) == DIRECTOR_OK && dispatch_local_init(c) == DIRECTOR_OK;
+    if (ok) ok = ffn_init(c) == DIRECTOR_OK && dispatch_local_init(c) == DIRECTOR_OK && dispatch_init(c) == DIRECTOR_OK;
     if (ok) {
         ok = cudaStreamCreateWithFlags(&c->h2d_stream, cudaStreamNonBlocking) == cudaSuccess &&
              cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking) == cudaSuccess;
@@ -620,7 +620,7 @@ int director_set_profiling(director_ctx* ctx, int32_t enabled) {
     if (cudaDeviceSynchronize() != cudaSuccess) return DIRECTOR_ERR_CUDA;
     for (auto& ev : ctx->events) ctx->free_events.push_back(ev);
     ctx->events.clear();
-    ctx->profiling = enabled != 0;
+    ctx->profiling = enabled == 2 ? 2 : (enabled != 0 ? 1 : 0);
     return DIRECTOR_OK;
 }
 

@@ -101,6 +101,7 @@ combine_kernel(const uint4* __restrict__ yp, const int32_t* __restrict__ inv_row
 
 int launch_combine(director_ctx* ctx, int T, const void* yp, const int32_t* inv_row, const float* topk_w,
                    const void* y_shared, void* y, cudaStream_t st) {
+    StageScope stage(ctx, st, "stage_combine");
     const director_shape& s = ctx->shape;
     const int row_vec = s.H * 2 / 16;
     const int slices = (row_vec + kCombineSliceVec - 1) / kCombineSliceVec;

@@ -60,7 +60,8 @@ struct director_ctx {
     int32_t* d_tile_counts = nullptr;   // [n_tiles_max, E] per-tile expert counts -> exclusive prefix
     int32_t* d_tile_rep = nullptr;      // [n_tiles_max, G] per-tile replica counts (locality-first dispatch)
     int32_t* d_seg_offsets = nullptr;   // [G+1] internal copy (placement-cost path, host forward)
-    unsigned int* d_ticket = nullptr;   // last-CTA-done counter, self-resetting
+    unsigned int* d_ticket = nullptr;   // [4]: [0] last-CTA-done counter, [1..2] grid barrier of the one-launch index kernel; self-resetting
+    int plan_max_tiles = 0;             // most 256-token tiles that kernel's cooperative launch can hold
     int32_t* d_status = nullptr;        // sticky device status word
 
     // expert FFN workspace
@@ -97,7 +98,8 @@ struct director_ctx {
     void* encode_tiled = nullptr;       // cuTensorMapEncodeTiled, resolved through the runtime
 
     int64_t launches = 0;
-    bool profiling = false;
+    int profiling = 0;                  // 0 off, 1 events around every kernel, 2 events around every stage
+    bool stage_open = false;            // a stage bracket is recording (stages do not nest)
     std::string profile_filter;         // when not empty, only kernels whose name contains it are timed
     std::vector<director::KernelEvent> events;
     std::vector<director::KernelEvent> free_events;
@@ -113,7 +115,7 @@ struct LaunchScope {
     bool timed = false;
     LaunchScope(director_ctx* c, cudaStream_t s, const char* name) : ctx(c), stream(s) {
         ctx->launches++;
-        if (ctx->profiling && (ctx->profile_filter.empty() || strstr(name, ctx->profile_filter.c_str()) != nullptr)) {
+        if (ctx->profiling == 1 && (ctx->profile_filter.empty() || strstr(name, ctx->profile_filter.c_str()) != nullptr)) {
             if (!ctx->free_events.empty()) {
                 ev = ctx->free_events.back();
                 ctx->free_events.pop_back();
@@ -133,6 +135,38 @@ struct LaunchScope {
     }
 };
 
+// Brackets all launches (kernels and memsets) of one stage of the layer with ONE pair of events when stage profiling
+// is on: the stage's time on an otherwise idle stream, launch gaps between its kernels included, the cost of the event
+// pair paid once per stage instead of once per kernel.
+struct StageScope {
+    director_ctx* ctx;
+    cudaStream_t stream;
+    KernelEvent ev{};
+    bool timed = false;
+    StageScope(director_ctx* c, cudaStream_t s, const char* name) : ctx(c), stream(s) {
+        if (ctx->profiling != 2 || ctx->stage_open) return;
+        if (!ctx->free_events.empty()) {
+            ev = ctx->free_events.back();
+            ctx->free_events.pop_back();
+            timed = true;
+        } else {
+            timed = cudaEventCreate(&ev.start) == cudaSuccess && cudaEventCreate(&ev.stop) == cudaSuccess;
+        }
+        ev.name = name;
+        if (timed) {
+            ctx->stage_open = true;
+            cudaEventRecord(ev.start, stream);
+        }
+    }
+    ~StageScope() {
+        if (timed) {
+            cudaEventRecord(ev.stop, stream);
+            ctx->events.push_back(ev);
+            ctx->stage_open = false;
+        }
+    }
+};
+
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? DIRECTOR_OK : DIRECTOR_ERR_CUDA; }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -148,6 +182,7 @@ int launch_dispatch(director_ctx*, int T, const void* x, const int32_t* topk_idx
                     int32_t* row_token, int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, cudaStream_t);
 int launch_scatter_rows(director_ctx*, int T, const void* x, const int32_t* inv_row, void* xp, cudaStream_t);
 int dispatch_local_init(director_ctx*);
+int dispatch_init(director_ctx*);
 int launch_dispatch_local_first(director_ctx*, int T, const void* x, const int32_t* topk_idx, const int32_t* src_rank,
                                 void* xp, int32_t* row_token, int32_t* inv_row, int32_t* dest_rank,
                                 int32_t* seg_offsets, cudaStream_t);

@@ -6,6 +6,14 @@
 // placement-cost histograms (Section VI-A: workload matrix W, Eq. 1 load, Eq. 3 dispatch volume).
 //
 // Kernels
+//   dispatch_plan_kernel  the whole index computation in ONE cooperative launch (batches whose 256-token
+//                      tiles are all resident at once, i.e. up to ~300 K tokens): per-tile expert counts
+//                      from lane bitmasks, a grid-wide barrier, then EVERY CTA sums the count columns it
+//                      needs (tiles before its own -> its prefix, all tiles -> the totals), splits the totals
+//                      over the replicas, scans the slot lengths and writes its own tokens' inv_row /
+//                      dest_rank / row_token - the bitmasks never leave shared memory and no CTA waits for
+//                      a single scanning CTA.  Larger batches and the allocation-free entry point use the
+//                      two kernels below.
 //   count_scan_kernel  per 256-token tile: per-expert counts from lane bitmasks; the last CTA to
 //                      finish (atomic ticket, no spinning) turns them into exclusive per-tile
 //                      prefixes, splits every expert's total over its replicas and scans the
@@ -70,15 +78,19 @@ count_scan_kernel(const int32_t* __restrict__ topk_idx, int T, int E, int K, int
     for (int e = threadIdx.x; e < E; e += blockDim.x) {
         const int run = scan_column(tile_counts, n_tiles, E, e);
         const int r0 = rep_start[e], r_e = rep_start[e + 1] - r0;
-        for (int q = 0; q < r_e; ++q)               // replica q gets ceil((N_e - q) / r_e) rows
-            slot_len[rep_slot[r0 + q]] = (run > q) ? (run - q + r_e - 1) / r_e : 0;
+        if (r_e < 1 && run > 0) director_set_status(status, DIRECTOR_ERR_BAD_INDEX);   // a routed-to expert without a host
+        for (int q = 0; q < r_e; ++q) {             // replica q gets ceil((N_e - q) / r_e) rows
+            const int slot = rep_slot[r0 + q];
+            if ((unsigned)slot < (unsigned)G) slot_len[slot] = (run > q) ? (run - q + r_e - 1) / r_e : 0;
+            else director_set_status(status, DIRECTOR_ERR_BAD_INDEX);
+        }
     }
     __syncthreads();
     scan_slots(slot_len, G, warp_sum, seg_offsets_a, seg_offsets_b, ticket);
 }
 
 __global__ void __launch_bounds__(kTokenTile)
-index_kernel(const int32_t* __restrict__ topk_idx, int T, int E, int K, int C_max,
+index_kernel(const int32_t* __restrict__ topk_idx, int T, int E, int K, int C_max, int G,
              const int32_t* __restrict__ rep_start, const int32_t* __restrict__ rep_slot,
              const int32_t* __restrict__ tile_prefix, const int32_t* __restrict__ seg_offsets,
              int32_t* __restrict__ row_token, int32_t* __restrict__ inv_row, int32_t* __restrict__ dest_rank,
@@ -97,15 +109,189 @@ index_kernel(const int32_t* __restrict__ topk_idx, int T, int E, int K, int C_ma
         if ((unsigned)e < (unsigned)E) {
             const int n = __ldg(tile_prefix + (size_t)tile * E + e) + tile_rank(mask, warp_prefix, e, w, lane);
             const int r0 = __ldg(rep_start + e), r_e = __ldg(rep_start + e + 1) - r0;
-            const int q = n % r_e, p = n / r_e;
-            const int slot = __ldg(rep_slot + r0 + q);
-            row = __ldg(seg_offsets + slot) + p;
-            dest = slot / C_max;
-            row_token[row] = t;
+            // the context's tables are validated when the placement is set; caller-built tables (the allocation-free
+            // entry point) are not, so an expert without a host or a slot outside the table is skipped and flagged
+            const int slot = r_e >= 1 ? __ldg(rep_slot + r0 + n % r_e) : -1;
+            if ((unsigned)slot < (unsigned)G) {
+                row = __ldg(seg_offsets + slot) + n / r_e;
+                dest = slot / C_max;
+                row_token[row] = t;
+            } else {
+                director_set_status(status, DIRECTOR_ERR_BAD_INDEX);
+            }
         }
         inv_row[(size_t)t * K + s] = row;
         dest_rank[(size_t)t * K + s] = dest;
     }
+}
+
+// Grid-wide barrier of a cooperative launch (all CTAs resident).  bar[0] counts arrivals, bar[1] departures; the last
+// CTA to leave zeroes both for the next launch.  The wait is bounded: on expiry the CTA reports false.
+__device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned long long plan_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ bool grid_barrier(unsigned int* bar, unsigned int n_ctas, int* s_flag) {
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        atomicAdd(bar, 1u);
+        int ok = 1;
+        if (ld_acquire_gpu(bar) < n_ctas) {
+            const unsigned long long t0 = plan_timer_ns();
+            unsigned int spins = 0;
+            while (ld_acquire_gpu(bar) < n_ctas) {
+                __nanosleep(32);
+                if ((++spins & 255u) == 0u && plan_timer_ns() - t0 > 2000000000ull) { ok = 0; break; }
+            }
+        }
+        *s_flag = ok;
+    }
+    __syncthreads();
+    return *s_flag != 0;
+}
+__device__ __forceinline__ void grid_barrier_leave(unsigned int* bar, unsigned int n_ctas) {
+    if (threadIdx.x == 0 && atomicAdd(bar + 1, 1u) == n_ctas - 1u) {
+        bar[0] = 0u;                // everybody has passed the wait: ready for the next launch on this stream
+        bar[1] = 0u;
+    }
+}
+
+__global__ void __launch_bounds__(kTokenTile)
+dispatch_plan_kernel(const int32_t* __restrict__ topk_idx, int T, int E, int K, int C_max, int G, int n_tiles,
+                     const int32_t* __restrict__ rep_start, const int32_t* __restrict__ rep_slot,
+                     int32_t* __restrict__ tile_counts, int32_t* __restrict__ seg_offsets_a,
+                     int32_t* __restrict__ seg_offsets_b, int32_t* __restrict__ row_token, int32_t* __restrict__ inv_row,
+                     int32_t* __restrict__ dest_rank, unsigned int* __restrict__ bar, int32_t* __restrict__ status) {
+    __shared__ uint32_t mask[kMaxE][kTileWarps];
+    __shared__ uint16_t warp_prefix[kMaxE][kTileWarps];
+    __shared__ int32_t s_pre[kMaxE], s_tot[kMaxE];
+    __shared__ int32_t s_seg[kMaxG + 1];          // slot lengths, then their exclusive prefix
+    __shared__ int32_t warp_sum[kTileWarps];
+    __shared__ int s_flag;
+
+    const int tile = blockIdx.x;
+    build_masks(mask, topk_idx, tile, T, E, K, status);
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
+        int c = 0;
+#pragma unroll
+        for (int w = 0; w < kTileWarps; ++w) c += __popc(mask[e][w]);
+        tile_counts[(size_t)tile * E + e] = c;
+        s_pre[e] = 0;
+        s_tot[e] = 0;
+    }
+    for (int g = threadIdx.x; g <= G; g += blockDim.x) s_seg[g] = 0;
+    build_warp_prefix(mask, warp_prefix, E);
+    if (!grid_barrier(bar, (unsigned)n_tiles, &s_flag)) {
+        if (threadIdx.x == 0) director_set_status(status, DIRECTOR_ERR_TIMEOUT);
+        return;
+    }
+    // every CTA of this grid is running: a programmatically dependent kernel (the row copies) may be scheduled into
+    // the free SMs now; it still waits for this grid to finish before it reads the indices
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    // ---- every CTA: column sums over the tiles (tiles before mine -> my prefix; all tiles -> the totals) ----
+    // 256 threads = `parts` groups of E_pad threads; group p sums tiles p, p + parts, ... of its expert's column;
+    // the partial sums meet in shared memory (integer adds: the order does not matter).
+    int e_pad = 1;
+    while (e_pad < E) e_pad <<= 1;
+    const int parts = kTokenTile / e_pad;                       // E <= 256 = blockDim
+    const int e_mine = threadIdx.x & (e_pad - 1), part = threadIdx.x / e_pad;
+    if (e_mine < E) {
+        int pre = 0, tot = 0;
+        for (int i0 = part; i0 < n_tiles; i0 += 8 * parts) {    // eight independent loads in flight per thread
+            int c[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int i = i0 + k * parts;
+                c[k] = i < n_tiles ? __ldcg(tile_counts + (size_t)i * E + e_mine) : 0;
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                tot += c[k];
+                if (i0 + k * parts < tile) pre += c[k];
+            }
+        }
+        if (parts > 1) {
+            if (pre) atomicAdd(&s_pre[e_mine], pre);
+            if (tot) atomicAdd(&s_tot[e_mine], tot);
+        } else {
+            s_pre[e_mine] = pre;
+            s_tot[e_mine] = tot;
+        }
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
+        const int run = s_tot[e];
+        const int r0 = __ldg(rep_start + e), r_e = __ldg(rep_start + e + 1) - r0;
+        if (r_e < 1 && run > 0 && tile == 0) director_set_status(status, DIRECTOR_ERR_BAD_INDEX);
+        for (int q = 0; q < r_e; ++q) {             // replica q gets ceil((N_e - q) / r_e) rows
+            const int slot = __ldg(rep_slot + r0 + q);
+            if ((unsigned)slot < (unsigned)G) s_seg[slot] = (run > q) ? (run - q + r_e - 1) / r_e : 0;
+        }
+    }
+    __syncthreads();
+    {   // exclusive scan of the slot lengths, in place; entry G receives the total
+        const int per = (G + blockDim.x - 1) / blockDim.x;
+        const int lo = min((int)threadIdx.x * per, G), hi = min(lo + per, G);
+        int local = 0;
+        for (int g = lo; g < hi; ++g) local += s_seg[g];
+        const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+        int incl = local;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) warp_sum[w] = incl;
+        __syncthreads();
+        int base = incl - local;
+        for (int i = 0; i < w; ++i) base += warp_sum[i];
+        for (int g = lo; g < hi; ++g) {
+            const int len = s_seg[g];
+            s_seg[g] = base;
+            base += len;
+        }
+        if (threadIdx.x == blockDim.x - 1) s_seg[G] = base;
+        __syncthreads();
+    }
+    if (tile == 0) {
+        for (int g = threadIdx.x; g <= G; g += blockDim.x) {
+            seg_offsets_a[g] = s_seg[g];
+            if (seg_offsets_b) seg_offsets_b[g] = s_seg[g];
+        }
+    }
+
+    // ---- my tile's assignments ----
+    const int t = tile * kTokenTile + threadIdx.x;
+    if (t < T) {
+        const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        for (int s = 0; s < K; ++s) {
+            const int e = __ldg(topk_idx + (size_t)t * K + s);
+            int row = -1, dest = -1;
+            if ((unsigned)e < (unsigned)E) {
+                const int n = s_pre[e] + tile_rank(mask, warp_prefix, e, w, lane);
+                const int r0 = __ldg(rep_start + e), r_e = __ldg(rep_start + e + 1) - r0;
+                const int slot = r_e >= 1 ? __ldg(rep_slot + r0 + n % r_e) : -1;
+                if ((unsigned)slot < (unsigned)G) {
+                    row = s_seg[slot] + n / r_e;
+                    dest = slot / C_max;
+                    row_token[row] = t;
+                } else {
+                    director_set_status(status, DIRECTOR_ERR_BAD_INDEX);
+                }
+            }
+            inv_row[(size_t)t * K + s] = row;
+            dest_rank[(size_t)t * K + s] = dest;
+        }
+    }
+    grid_barrier_leave(bar, (unsigned)n_tiles);
 }
 
 // One warp copies a 2 KB slice (4 x 16 bytes per lane) of row t of x to its K destination rows.
@@ -123,10 +309,15 @@ scatter_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ inv
     const int v0 = (int)(item % slices_per_row) * (32 * kSliceVec) + lane;
     const uint4* src = x + (size_t)t * row_vec;
     uint4 v[kSliceVec];
+    // x is an input of the whole dispatch: its slice is fetched before the wait below, while the index kernel
+    // that this launch programmatically depends on may still be finishing
 #pragma unroll
     for (int i = 0; i < kSliceVec; ++i)
         if (v0 + 32 * i < row_vec) v[i] = __ldcs(src + v0 + 32 * i);
-    int my_row = (lane < K) ? __ldg(inv_row + (size_t)t * K + lane) : -1;
+    // launched with programmatic stream serialization: returns once the preceding kernel of the stream has
+    // completed and its writes (inv_row) are visible; a no-op under an ordinary launch
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    int my_row = (lane < K) ? __ldcg(inv_row + (size_t)t * K + lane) : -1;
     for (int s = 0; s < K; ++s) {
         const int row = __shfl_sync(0xFFFFFFFFu, my_row, s);
         if (row < 0) continue;
@@ -393,30 +584,73 @@ int launch_count_scan(director_ctx* ctx, const char* name, int T, const int32_t*
 
 }  // namespace
 
+// Largest number of 256-token tiles the one-launch index kernel can take: all its CTAs must be resident at once.
+int dispatch_init(director_ctx* ctx) {
+    int per_sm = 0, coop = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dispatch_plan_kernel, kTokenTile, 0) != cudaSuccess ||
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, ctx->device) != cudaSuccess)
+        return DIRECTOR_ERR_CUDA;
+    ctx->plan_max_tiles = coop ? per_sm * ctx->sm_count : 0;
+    return DIRECTOR_OK;
+}
+
 int launch_scatter_rows(director_ctx* ctx, int T, const void* x, const int32_t* inv_row, void* xp, cudaStream_t st) {
+    StageScope stage(ctx, st, "stage_dispatch");
     const director_shape& s = ctx->shape;
     const int row_vec = s.H * 2 / 16;
     const int slices = (s.H * 2 + kSliceBytes - 1) / kSliceBytes;
     const long long items = (long long)T * slices;
     const unsigned grid = (unsigned)((items + kScatterWarps - 1) / kScatterWarps);
     LaunchScope scope(ctx, st, "dispatch_scatter_rows_kernel");
-    scatter_rows_kernel<<<grid, kScatterWarps * 32, 0, st>>>(static_cast<const uint4*>(x), inv_row,
-                                                             static_cast<uint4*>(xp), T, s.K, row_vec, slices);
-    return cuda_status(cudaGetLastError());
+    // programmatic dependent launch: the copy kernel's CTAs may be set up, and read their slices of x, while the
+    // kernel before it in the stream (the index kernel) drains; they wait for it before touching inv_row
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kScatterWarps * 32);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cuda_status(cudaLaunchKernelEx(&cfg, scatter_rows_kernel, static_cast<const uint4*>(x), inv_row,
+                                          static_cast<uint4*>(xp), T, (int)s.K, row_vec, slices));
 }
 
 int launch_dispatch(director_ctx* ctx, int T, const void* x, const int32_t* topk_idx, const int32_t* src_rank, void* xp,
                     int32_t* row_token, int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, cudaStream_t st) {
+    StageScope stage(ctx, st, "stage_dispatch");
     if (ctx->replica_policy == DIRECTOR_REPLICA_LOCAL_FIRST)
         return launch_dispatch_local_first(ctx, T, x, topk_idx, src_rank, xp, row_token, inv_row, dest_rank,
                                            seg_offsets, st);
     const director_shape& s = ctx->shape;
     const int n_tiles = (T + kTokenTile - 1) / kTokenTile;
-    int rc = launch_count_scan(ctx, "dispatch_count_scan_kernel", T, topk_idx, seg_offsets, ctx->d_seg_offsets, st);
+    int rc;
+    if (n_tiles <= ctx->plan_max_tiles) {
+        // one cooperative launch: counts, grid barrier, per-CTA scans, indices
+        int E = s.E, K = s.K, C_max = s.C_max, G = ctx->G, nt = n_tiles, Tv = T;
+        const int32_t* rs = ctx->d_rep_start;
+        const int32_t* rl = ctx->d_rep_slot;
+        int32_t* tc = ctx->d_tile_counts;
+        int32_t* seg_b = ctx->d_seg_offsets;
+        unsigned int* bar = ctx->d_ticket + 1;
+        int32_t* status = ctx->d_status;
+        void* args[] = {&topk_idx, &Tv, &E, &K, &C_max, &G, &nt, &rs, &rl, &tc, &seg_offsets, &seg_b,
+                        &row_token, &inv_row, &dest_rank, &bar, &status};
+        {
+            LaunchScope scope(ctx, st, "dispatch_plan_kernel");
+            rc = cuda_status(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(dispatch_plan_kernel), dim3(n_tiles),
+                                                         dim3(kTokenTile), args, 0, st));
+        }
+        if (rc != DIRECTOR_OK) return rc;
+        if (xp != nullptr) rc = launch_scatter_rows(ctx, T, x, inv_row, xp, st);
+        return rc;
+    }
+    rc = launch_count_scan(ctx, "dispatch_count_scan_kernel", T, topk_idx, seg_offsets, ctx->d_seg_offsets, st);
     if (rc != DIRECTOR_OK) return rc;
     {
         LaunchScope scope(ctx, st, "dispatch_index_kernel");
-        index_kernel<<<n_tiles, kTokenTile, 0, st>>>(topk_idx, T, s.E, s.K, s.C_max, ctx->d_rep_start, ctx->d_rep_slot,
+        index_kernel<<<n_tiles, kTokenTile, 0, st>>>(topk_idx, T, s.E, s.K, s.C_max, ctx->G, ctx->d_rep_start, ctx->d_rep_slot,
                                                      ctx->d_tile_counts, seg_offsets, row_token, inv_row, dest_rank,
                                                      ctx->d_status);
         rc = cuda_status(cudaGetLastError());
@@ -450,6 +684,7 @@ int launch_cost_batch(director_ctx* ctx, const int64_t* workload, int n, const u
 
 int launch_cost(director_ctx* ctx, int T, const int32_t* topk_idx, const int32_t* src_rank, int64_t* workload,
                 int64_t* rank_load, int64_t* dispatch_tokens, uint64_t* dispatch_bytes, cudaStream_t st) {
+    StageScope stage(ctx, st, "stage_placement_cost");
     const director_shape& s = ctx->shape;
     const int n_tiles = (T + kTokenTile - 1) / kTokenTile;
     const bool local_first = ctx->replica_policy == DIRECTOR_REPLICA_LOCAL_FIRST;
@@ -554,7 +789,7 @@ extern "C" int director_dispatch_index_static(int32_t T, int32_t K, int32_t E, i
     count_scan_kernel<<<n_tiles, kTokenTile, 0, st>>>(topk_idx, T, E, K, G, n_tiles, rep_start, rep_slot, tile_counts,
                                                       seg_offsets, nullptr, ticket, status);
     if (cudaGetLastError() != cudaSuccess) return DIRECTOR_ERR_CUDA;
-    index_kernel<<<n_tiles, kTokenTile, 0, st>>>(topk_idx, T, E, K, C_max, rep_start, rep_slot, tile_counts, seg_offsets,
+    index_kernel<<<n_tiles, kTokenTile, 0, st>>>(topk_idx, T, E, K, C_max, G, rep_start, rep_slot, tile_counts, seg_offsets,
                                                  row_token, inv_row, dest_rank, status);
     return cuda_status(cudaGetLastError());
 }

@@ -277,12 +277,13 @@ int launch_travel_scan(director_ctx* ctx, const char* name, int T, const int32_t
 }  // namespace
 
 int dispatch_local_init(director_ctx* ctx) {
-    // worst case (E = 256, G = 1024 replicas) needs 56 KB of dynamic shared memory
-    const int E = ctx->shape.E, G = ctx->G;
+    // The attribute belongs to the kernel, not to the context: opt in once for the largest supported shape
+    // (E = 256, G = 1024 replicas: 56 KB), so that a context of a smaller shape never lowers another one's limit.
+    (void)ctx;
     if (cudaFuncSetAttribute(slot_count_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)slot_count_smem_bytes(E, G, G)) != cudaSuccess ||
+                             (int)slot_count_smem_bytes(kMaxE, kMaxG, kMaxG)) != cudaSuccess ||
         cudaFuncSetAttribute(local_index_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)local_index_smem_bytes(G)) != cudaSuccess)
+                             (int)local_index_smem_bytes(kMaxG)) != cudaSuccess)
         return DIRECTOR_ERR_CUDA;
     return DIRECTOR_OK;
 }

@@ -317,6 +317,7 @@ int ffn_init(director_ctx* ctx) {
 int launch_expert_ffn(director_ctx* ctx, int T, const void* xp, const int32_t* row_token, const int32_t* seg_offsets,
                       const void* w_gate, const void* w_up, const void* w_down, void* yp, const void* x,
                       const void* ws_gate, const void* ws_up, const void* ws_down, void* y_shared, cudaStream_t st) {
+    StageScope stage(ctx, st, "stage_expert_ffn");
     const director_shape& s = ctx->shape;
     // work-item counters of the (up to four) GEMM launches below
     if (cudaMemsetAsync(ctx->d_sched, 0, 4 * sizeof(unsigned int), st) != cudaSuccess) return DIRECTOR_ERR_CUDA;

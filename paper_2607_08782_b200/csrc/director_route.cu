@@ -404,6 +404,7 @@ bool front_small_applies(const director_ctx* ctx, int T) {
 int launch_front_small(director_ctx* ctx, int T, const float* logits, int32_t* topk_idx, float* topk_w,
                        int32_t* row_token, int32_t* inv_row, int32_t* dest_rank, int32_t* seg_offsets, int64_t* workload,
                        int64_t* rank_load, int64_t* dispatch_tokens, uint64_t* dispatch_bytes, cudaStream_t st) {
+    StageScope stage(ctx, st, "stage_front_small");
     const director_shape& s = ctx->shape;
     LaunchScope scope(ctx, st, "front_small_kernel");
 #define FRONT_LAUNCH(VEC, K8)                                                                                          \
@@ -421,6 +422,7 @@ int launch_front_small(director_ctx* ctx, int T, const float* logits, int32_t* t
 }
 
 int launch_route(director_ctx* ctx, int T, const float* logits, int32_t* topk_idx, float* topk_w, cudaStream_t st) {
+    StageScope stage(ctx, st, "stage_route");
     const int E = ctx->shape.E, K = ctx->shape.K;
     // lanes per token: splitting a token over more lanes adds merge work, so use the fewest lanes (at most one per
     // group of eight experts, at most 8) that give the GPU about 128 K threads and each lane at most four groups

@@ -383,12 +383,13 @@ def test_routing_and_indices_at_half_a_million_tokens():
     assert np.array_equal(row_token.cpu().numpy(), d_o["row_token"])
 
 
-def test_cuda_graph_replay_reproduces_the_direct_pass():
+@pytest.mark.parametrize("T", [200, 1000])      # the single-CTA front end, and the cooperative index kernel
+def test_cuda_graph_replay_reproduces_the_direct_pass(T):
     """Every entry point is capturable: a graph of the whole layer replays to the same bits, also after the
     inputs in the captured buffers have changed."""
     import torch
     from paper_2607_08782_b200.layer import tensor_to_bf16_bits
-    shape, logits, x, weights = _custom(95, 200, 256, 16, 4, 256, 1, 4, 5, 1.2)
+    shape, logits, x, weights = _custom(95, T, 256, 16, 4, 256, 1, 4, 5, 1.2)
     X = _random_placement(95, 16, 4, 5, 3)
     case = GpuCase(shape, logits, x, weights)
     L, T = case.layer, shape.T
@@ -476,7 +477,7 @@ def test_fused_front_end_matches_the_separate_stages_and_the_oracle(seed, T, H, 
                             o["seg"], o["W"], o["load"], o["dt"], o["db"])
     torch.cuda.synchronize()
     assert L.d.last_status() == 0
-    assert L.d.launch_count() - n0 == (2 if T <= 256 else 6)
+    assert L.d.launch_count() - n0 == (2 if T <= 256 else 5)     # route, one-launch indices, row copies, two cost kernels
     from paper_2607_08782_b200.layer import tensor_to_bf16_bits
     assert np.array_equal(o["idx"].cpu().numpy(), g.topk_idx)
     assert np.array_equal(o["w"].cpu().numpy(), g.topk_w)                # same arithmetic: same bits
