@@ -291,7 +291,8 @@ STAGE_KERNELS = {
     "route": ["route_topk_kernel", "front_small_kernel"],   # the fused front end (T <= 256) is booked under route
     "dispatch": ["dispatch_plan_kernel", "dispatch_count_scan_kernel", "dispatch_index_kernel", "dispatch_scatter_rows_kernel",
                  "dispatch_travel_count_scan_kernel", "dispatch_slot_count_scan_kernel", "dispatch_local_index_kernel"],
-    "expert_ffn": ["grouped_gemm_swiglu_kernel", "grouped_gemm_down_kernel", "one_segment_kernel"],
+    "expert_ffn": ["grouped_gemm_swiglu_kernel", "grouped_gemm_down_kernel", "one_segment_kernel",
+                   "small_ffn_swiglu_kernel", "small_ffn_down_kernel"],
     "combine": ["combine_kernel"],
     "placement_cost": ["cost_workload_hist_kernel", "cost_from_workload_kernel", "cost_count_scan_kernel", "cost_kernel",
                        "cost_travel_count_scan_kernel", "cost_local_kernel"],
@@ -450,7 +451,7 @@ def main():
     ap.add_argument("--config", default="c2_mixtral", choices=sorted(WORKLOAD_TEXT))
     ap.add_argument("--tokens", type=int, default=None, help="batch size override (c5_qwen3 sweep: 1, 64, 1024, 32768)")
     ap.add_argument("--placement", default="auto", choices=["auto", "primary"])
-    ap.add_argument("--ffn-variant", type=int, default=None, choices=[0, 1, 2, 3, 4, 5],
+    ap.add_argument("--ffn-variant", type=int, default=None, choices=[0, 1, 2, 3, 4, 5, 6],
                     help="expert-FFN tile scheme: 0 = one CTA per 128x256 tile, 1 = CTA pairs (256x256); default: library's")
     ap.add_argument("--replica-policy", default="round_robin", choices=["round_robin", "local_first"],
                     help="which replica of a replicated expert an assignment uses (the default is the headline setting)")

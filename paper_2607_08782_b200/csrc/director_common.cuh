@@ -19,6 +19,7 @@ constexpr int kMaxK = 8;
 constexpr int kMaxR = 64;
 constexpr int kMaxC = 16;
 constexpr int kMaxG = kMaxR * kMaxC;
+constexpr int kSmallFfnTokens = 4;      // batches of at most this many tokens take the weight-streaming FFN kernels
 constexpr int kGemmClockCtas = 512;   // CTAs per GEMM launch whose {cycles, ns} records fit the clock buffer
 
 struct KernelEvent {
@@ -94,6 +95,7 @@ struct director_ctx {
 
     int pair_clusters = 0;              // CTA pairs the device can hold at once (pair variant's grid)
     int ffn_variant = 2;                // tile scheme of the expert-FFN GEMMs, see director_set_ffn_variant
+    bool ffn_small = true;              // decode-sized batches (T <= kSmallFfnTokens) use the weight-streaming kernels
     int ffn_dual = 0;                   // bit 0 / bit 1: the gate|up / down GEMM takes two token tiles per work item
     void* encode_tiled = nullptr;       // cuTensorMapEncodeTiled, resolved through the runtime
 

@@ -23,6 +23,8 @@
 #include "director_common.cuh"
 #include "director_umma.cuh"
 
+#include <algorithm>
+
 namespace director {
 
 int ffn_swap_init(director_ctx* ctx);   // director_ffn_swap.cu
@@ -30,6 +32,10 @@ int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int
                   const int32_t* seg_offsets, const int32_t* slot_expert, int G, const void* w_gate, const void* w_up,
                   const void* w_down, uint64_t n_experts, int Fw, void* hidden, void* out, unsigned int* counters,
                   const DenseFfn* dense, cudaStream_t st);
+int ffn_small_init(director_ctx* ctx);  // director_ffn_small.cu
+int ffn_pass_small(director_ctx* ctx, const void* in, const int32_t* seg_offsets, const int32_t* slot_expert, int G,
+                   const void* w_gate, const void* w_up, const void* w_down, int Fw, void* hidden, void* out, int rows_max,
+                   int max_segments, cudaStream_t st);
 int ffn_pair_init(director_ctx* ctx);   // director_ffn_pair.cu
 int launch_gemm_pair(director_ctx* ctx, int mode, const char* name, const CUtensorMap& a, const CUtensorMap& b0,
                      const CUtensorMap& b1, const umma::GroupedGemmParams& p, cudaStream_t st);
@@ -305,7 +311,8 @@ __global__ void one_segment_kernel(int32_t* seg, int T) {
 }  // namespace
 
 int ffn_init(director_ctx* ctx) {
-    if (ffn_pair_init(ctx) != DIRECTOR_OK || ffn_swap_init(ctx) != DIRECTOR_OK) return DIRECTOR_ERR_CUDA;
+    if (ffn_pair_init(ctx) != DIRECTOR_OK || ffn_swap_init(ctx) != DIRECTOR_OK || ffn_small_init(ctx) != DIRECTOR_OK)
+        return DIRECTOR_ERR_CUDA;
     if (cudaFuncSetAttribute(grouped_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
         cudaFuncSetAttribute(grouped_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
         return DIRECTOR_ERR_CUDA;
@@ -319,10 +326,23 @@ int launch_expert_ffn(director_ctx* ctx, int T, const void* xp, const int32_t* r
                       const void* ws_gate, const void* ws_up, const void* ws_down, void* y_shared, cudaStream_t st) {
     StageScope stage(ctx, st, "stage_expert_ffn");
     const director_shape& s = ctx->shape;
-    // work-item counters of the (up to four) GEMM launches below
-    if (cudaMemsetAsync(ctx->d_sched, 0, 4 * sizeof(unsigned int), st) != cudaSuccess) return DIRECTOR_ERR_CUDA;
     const uint64_t A = (uint64_t)T * s.K;
     const bool shared = s.S > 0 && x != nullptr && y_shared != nullptr;
+    if (ctx->ffn_variant == 2 && ctx->ffn_small && row_token == nullptr && T <= kSmallFfnTokens) {
+        // decode-sized batch: every segment has at most T rows; stream the touched weights once, feature by feature
+        int rc = ffn_pass_small(ctx, xp, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up, w_down, s.F, ctx->d_hidden,
+                                yp, T, (int)std::min<uint64_t>((uint64_t)ctx->G, A), st);
+        if (rc != DIRECTOR_OK || !shared) return rc;
+        {
+            LaunchScope scope(ctx, st, "one_segment_kernel");
+            one_segment_kernel<<<1, 1, 0, st>>>(ctx->d_one_seg, T);
+            if ((rc = cuda_status(cudaGetLastError())) != DIRECTOR_OK) return rc;
+        }
+        return ffn_pass_small(ctx, x, ctx->d_one_seg, ctx->d_zero_expert, 1, ws_gate, ws_up, ws_down, s.S * s.F,
+                              ctx->d_hidden_shared, y_shared, T, 1, st);
+    }
+    // work-item counters of the (up to four) GEMM launches below
+    if (cudaMemsetAsync(ctx->d_sched, 0, 4 * sizeof(unsigned int), st) != cudaSuccess) return DIRECTOR_ERR_CUDA;
     if (shared && row_token == nullptr && ctx->ffn_variant == 2) {
         // routed and shared experts in the same two launches: the shared experts' work items follow the routed ones
         const DenseFfn dense{x, (uint64_t)T, ws_gate, ws_up, ws_down, s.S * s.F, ctx->d_hidden_shared, y_shared};

@@ -309,7 +309,7 @@ def test_host_buffer_entry_points_match_the_device_path():
         assert np.array_equal(b["load"].numpy(), b["load_ref"])
 
 
-@pytest.mark.parametrize("variant", [0, 1, 2, 3, 4, 5])
+@pytest.mark.parametrize("variant", [0, 1, 2, 3, 4, 5, 6])
 def test_every_ffn_tile_scheme_matches_the_oracle_and_the_others(variant):
     """The three tile schemes of the expert-FFN GEMMs (single CTA, CTA pair, weight-stationary CTA pair)
     accumulate every output in the same order, so they must agree bit for bit, and each must match the oracle."""
@@ -632,3 +632,34 @@ def test_a_bounded_wait_that_runs_out_sets_the_timeout_status_and_leaves_the_con
     for bad in (0, 999, 10 ** 9):          # limits outside 1 us .. 100 ms are refused before any launch
         with pytest.raises(DirectorError):
             d.selftest_bounded_wait(bad)
+
+
+@pytest.mark.parametrize("seed,T,H,E,K,F,S,R,C,extra", [
+    (111, 1, 2048, 128, 8, 768, 0, 16, 9, 16),     # one token of the Qwen3-shaped layer
+    (112, 4, 512, 16, 4, 1408, 2, 4, 5, 4),        # the largest streamed batch, F not a multiple of 256, shared experts
+    (113, 3, 256, 6, 3, 128, 1, 3, 4, 6),          # every expert replicated: segments of one or two rows
+    (114, 3, 4608, 8, 2, 4224, 0, 8, 2, 2),        # contraction longer than one staged chunk in both kernels
+])
+def test_decode_batches_stream_the_weights_and_match_the_oracle_and_the_tensor_core_path(seed, T, H, E, K, F, S, R, C, extra):
+    """Batches of at most 4 tokens take the weight-streaming FFN kernels: whole-tensor parity with the oracle, the
+    tensor-core kernels on the same input agree within the same tolerance, results are bitwise reproducible."""
+    shape, logits, x, weights = _custom(seed, T, H, E, K, F, S, R, C)
+    X = _random_placement(seed, E, R, C, extra)
+    case = GpuCase(shape, logits, x, weights)
+    n0 = case.layer.d.launch_count()
+    g = case.run(X)
+    idx, w, w64, d, c = _oracle_front(shape, logits, x, X, C)
+    _check_outputs(shape, g, x, weights, idx, w, w64, d, c, np.arange(T), f"decode{seed}")
+    g2 = case.run(X)
+    assert np.array_equal(g.yp, g2.yp) and np.array_equal(g.y, g2.y)
+    case.layer.d.set_profiling(True)
+    case.run(X)
+    assert case.layer.d.kernel_time("small_ffn")[1] == (4 if S > 0 else 2)        # the streaming kernels ran ...
+    assert case.layer.d.kernel_time("grouped_gemm")[1] == 0                       # ... and no tensor-core kernel
+    case.layer.d.set_profiling(False)
+    case.layer.d.set_ffn_variant(6)                                               # tensor cores for every batch size
+    gt = case.run(X)
+    case.layer.d.set_ffn_variant(2)
+    a, b = orc.bf16_to_f64(g.y), orc.bf16_to_f64(gt.y)
+    assert rel_l2(a, b) <= REL_L2_TOL and max_abs(a, b) <= MAX_ABS_TOL
+    assert np.array_equal(g.inv_row, gt.inv_row)
