@@ -120,7 +120,7 @@ int director_create(const director_shape* shape, director_ctx** out) {
     const size_t cost_words = (size_t)s.R * s.E + s.R + 2 * (size_t)s.R * s.R;
 
     bool ok = dev_alloc(&c->d_rep_start, s.E + 1) && dev_alloc(&c->d_rep_slot, (size_t)s.E * s.R) &&
-              dev_alloc(&c->d_slot_expert, c->G) && dev_alloc(&c->d_tile_counts, (size_t)c->n_tiles_max * s.E) &&
+              dev_alloc(&c->d_slot_expert, 2 * (size_t)c->G) && dev_alloc(&c->d_tile_counts, (size_t)c->n_tiles_max * s.E) &&
               dev_alloc(&c->d_seg_offsets, c->G + 1) && dev_alloc(&c->d_ticket, 4) && dev_alloc(&c->d_status, 1) &&
               dev_alloc(&c->d_host_mask, s.E) && dev_alloc(&c->d_tile_rep, (size_t)c->n_tiles_max * c->G) &&
               dev_alloc(&c->d_one_seg, 2) && dev_alloc(&c->d_sched, 4) &&
@@ -190,7 +190,8 @@ int director_set_placement(director_ctx* ctx, const uint8_t* X, void* stream) {
     if (X == nullptr) return DIRECTOR_ERR_INVALID_ARG;
     const director_shape& s = ctx->shape;
     const int E = s.E, R = s.R, C = s.C_max;
-    std::vector<int32_t> rep_start(E + 1, 0), rep_slot, slot_expert((size_t)R * C, -1), slot_of((size_t)E * R, -1);
+    // slot_expert [G] is followed by slot_order [G]: the slots sorted by (expert, slot), unused slots last
+    std::vector<int32_t> rep_start(E + 1, 0), rep_slot, slot_expert(2 * (size_t)R * C, -1), slot_of((size_t)E * R, -1);
     // hosted(j): experts on rank j in ascending id -> slots j*C + 0,1,...   (capacity: sum_i x_ij <= C_max)
     for (int j = 0; j < R; ++j) {
         int p = 0;
@@ -213,6 +214,13 @@ int director_set_placement(director_ctx* ctx, const uint8_t* X, void* stream) {
         if ((int32_t)rep_slot.size() == rep_start[e]) return DIRECTOR_ERR_PLACEMENT;
     }
     rep_start[E] = (int32_t)rep_slot.size();
+    {
+        const size_t Gs = (size_t)R * C;
+        size_t n = 0;
+        for (int32_t v : rep_slot) slot_expert[Gs + n++] = v;          // replicas are listed by (expert, rank): that order
+        for (size_t g = 0; g < Gs; ++g)
+            if (slot_expert[g] < 0) slot_expert[Gs + n++] = (int32_t)g;   // the unused slots close the list
+    }
     std::vector<unsigned long long> host_mask(E, 0ull);
     for (int e = 0; e < E; ++e)
         for (int j = 0; j < R; ++j)
@@ -239,7 +247,7 @@ int director_reserve_placements(director_ctx* ctx, int32_t n) {
     while ((int)ctx->bank.size() < n) {
         director_ctx::PlacementTables t{nullptr, nullptr, nullptr, nullptr, 0, false};
         const bool ok = dev_alloc(&t.rep_start, s.E + 1) && dev_alloc(&t.rep_slot, (size_t)s.E * s.R) &&
-                        dev_alloc(&t.slot_expert, ctx->G) && dev_alloc(&t.host_mask, s.E);
+                        dev_alloc(&t.slot_expert, 2 * (size_t)ctx->G) && dev_alloc(&t.host_mask, s.E);
         if (!ok) {
             cudaGetLastError();
             void* tables[] = {t.rep_start, t.rep_slot, t.slot_expert, t.host_mask};

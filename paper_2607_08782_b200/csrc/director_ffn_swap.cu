@@ -38,14 +38,20 @@ constexpr int S_HEADER_BYTES = 384;                            // barriers, sche
 constexpr int S_MAX_SMEM = 232448;                             // opt-in shared memory per CTA on sm_100
 // Shared memory of a launch: alignment slack, the operand ring, the header, and the segment tables of its G slots
 // (seg_offsets and token-tile prefix as int32, expert ids as int16).
-constexpr int swap_smem_bytes(int stages, int G, bool dual = false) {
-    return 1024 + stages * stage_bytes(dual) + S_HEADER_BYTES + (G + 1) * 10 + 6;
+// (segment starts, work-item prefix as int32, expert ids as int16; segment ends as int32 when the segments are
+// walked in expert order rather than slot order).
+constexpr int swap_smem_bytes(int stages, int G, bool dual = false, bool ordered = false) {
+    return 1024 + stages * stage_bytes(dual) + S_HEADER_BYTES + (G + 1) * (ordered ? 14 : 10) + 6;
 }
 // The operand stream is latency-bound (a stage comes back ~2.5 us after it is released), so the ring is as deep as
 // shared memory allows: seven stages when the segment tables are small enough, else six.
-inline int swap_stages(int G) { return swap_smem_bytes(7, G) <= S_MAX_SMEM ? 7 : 6; }
+inline int swap_stages(int G, bool ordered = false) { return swap_smem_bytes(7, G, false, ordered) <= S_MAX_SMEM ? 7 : 6; }
+// Walking the segments in expert order costs four more bytes of shared memory per segment; it is done when that
+// does not cost the ring its seventh stage.
+inline bool swap_can_order(int G) { return swap_stages(G, true) == swap_stages(G, false); }
 constexpr int DUAL_STAGES = 4;                                 // 4 x 48 KB: fits with the largest segment table
-static_assert(swap_smem_bytes(DUAL_STAGES, kMaxG, true) <= S_MAX_SMEM, "dual ring does not fit");
+static_assert(swap_smem_bytes(DUAL_STAGES, kMaxG, true, true) <= S_MAX_SMEM, "dual ring does not fit");
+static_assert(swap_smem_bytes(6, kMaxG, false, true) <= S_MAX_SMEM, "six stages do not fit with the largest segment table");
 constexpr int TOKEN_TILE = 256;                                // tokens per full tile (N of the pair's MMA)
 constexpr int TOKEN_STEP = 32;                                 // granularity of N
 // Epilogue warps per TMEM lane quadrant.  The SwiGLU epilogue of GEMM-1 is long (shuffle, exp, reciprocal,
@@ -109,6 +115,10 @@ constexpr int SCHED_AHEAD = 1;      // items the scheduler may claim beyond the 
 struct SwapParams {
     const int32_t* seg_offsets;
     const int32_t* slot_expert;
+    // Optional: the order in which the segments are walked, [G] slot ids sorted by (expert, slot), unused slots last.
+    // Replica segments of one expert then follow each other in the work-item order, so the second replica finds the
+    // expert's weights still in L2 instead of streaming them from HBM again.  nullptr: slot order.
+    const int32_t* slot_order;
     int G;
     int w_blocks;              // weight-row blocks per expert (128 f per pair in GEMM-1, 256 h in GEMM-2)
     int k_steps;
@@ -147,7 +157,8 @@ __device__ __forceinline__ int sub_valid(const SwapTile& t, int j) { return min(
 __device__ __forceinline__ int round_n(int valid) { return (valid + TOKEN_STEP - 1) / TOKEN_STEP * TOKEN_STEP; }
 
 struct SwapWalker {
-    const int32_t* seg_off;
+    const int32_t* seg_off;     // first row of the i-th segment of the walk
+    const int32_t* seg_end;     // one past its last row
     const int32_t* tt_start;    // prefix of work items (per weight block) per segment
     const int16_t* expert;
     int w_blocks, w_rows_per_expert, rows_per_block, total, item_rows, g = 0;
@@ -160,7 +171,7 @@ struct SwapWalker {
         t.wb = local / nt;
         const int tt = local - t.wb * nt;
         t.row0 = seg_off[g] + tt * item_rows;
-        t.valid = min(item_rows, seg_off[g + 1] - t.row0);
+        t.valid = min(item_rows, seg_end[g] - t.row0);
         t.w_row = expert[g] * w_rows_per_expert + t.wb * rows_per_block;
         return true;
     }
@@ -200,6 +211,10 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     int32_t* s_seg = reinterpret_cast<int32_t*>(gen + S_HEADER_BYTES);
     int32_t* s_tt = s_seg + (G + 1);
     int16_t* s_exp = reinterpret_cast<int16_t*>(s_tt + (G + 1));
+    // in slot order a segment ends where the next one starts; in expert order the ends are a table of their own
+    const bool ordered = p.slot_order != nullptr;
+    int32_t* s_hi = reinterpret_cast<int32_t*>(gen + S_HEADER_BYTES + (((G + 1) * 10 + 3) & ~3));   // 4-byte aligned, behind s_exp
+    const int32_t* s_end = ordered ? s_hi : s_seg + 1;
 
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
@@ -217,8 +232,17 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     if (threadIdx.x == 0) { clk0 = clock64(); ns0 = global_ns(); }
 
     constexpr int n_threads = 96 + 128 * EPI_GROUPS;               // producer, MMA and scheduler warps + epilogue warps
-    for (int g = threadIdx.x; g <= G; g += n_threads) s_seg[g] = __ldg(p.seg_offsets + g);
-    for (int g = threadIdx.x; g < G; g += n_threads) s_exp[g] = (int16_t)__ldg(p.slot_expert + g);
+    if (ordered) {
+        for (int i = threadIdx.x; i < G; i += n_threads) {
+            const int g = __ldg(p.slot_order + i);
+            s_seg[i] = __ldg(p.seg_offsets + g);
+            s_hi[i] = __ldg(p.seg_offsets + g + 1);
+            s_exp[i] = (int16_t)__ldg(p.slot_expert + g);
+        }
+    } else {
+        for (int g = threadIdx.x; g <= G; g += n_threads) s_seg[g] = __ldg(p.seg_offsets + g);
+        for (int g = threadIdx.x; g < G; g += n_threads) s_exp[g] = (int16_t)__ldg(p.slot_expert + g);
+    }
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         *prod_taken = 0;
@@ -231,7 +255,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     __syncthreads();
     {
         auto tiles_of = [&](int g) {
-            const int len = s_seg[g + 1] - s_seg[g];
+            const int len = s_end[g] - s_seg[g];
             return (s_exp[g] >= 0 && len > 0) ? (len + ITEM_ROWS - 1) / ITEM_ROWS : 0;
         };
         const int per = (G + n_threads - 1) / n_threads;
@@ -263,7 +287,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     const uint32_t tmem_base = *tmem_slot;
 
     constexpr int ROWS_PER_BLOCK = (MODE == 0) ? 128 : 256;   // weight rows (f or h) per pair block
-    SwapWalker walker{s_seg, s_tt, s_exp, p.w_blocks, p.w_rows_per_expert, ROWS_PER_BLOCK, s_tt[G] * p.w_blocks, ITEM_ROWS};
+    SwapWalker walker{s_seg, s_end, s_tt, s_exp, p.w_blocks, p.w_rows_per_expert, ROWS_PER_BLOCK, s_tt[G] * p.w_blocks, ITEM_ROWS};
     SwapTile t;
 
     // Work items (segment, weight block, token tile) are handed out dynamically, in their natural order, from a
@@ -598,7 +622,7 @@ int launch_swap_n(director_ctx* ctx, const char* name, const CUtensorMap& w, con
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * ctx->pair_clusters));
     cfg.blockDim = dim3(96 + 128 * EPI_GROUPS);
-    cfg.dynamicSmemBytes = (size_t)swap_smem_bytes(STAGES, p.G, DUAL);
+    cfg.dynamicSmemBytes = (size_t)swap_smem_bytes(STAGES, p.G, DUAL, p.slot_order != nullptr);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -618,20 +642,20 @@ int launch_swap(director_ctx* ctx, const char* name, const CUtensorMap& w, const
     if constexpr (!GATHER) {
         if (dual) return launch_swap_n<MODE, EPI_GROUPS, false, DUAL_STAGES, true>(ctx, name, w, x, w2, x2, p, st);
     }
-    return swap_stages(p.G) == 7 ? launch_swap_n<MODE, EPI_GROUPS, GATHER, 7, false>(ctx, name, w, x, w2, x2, p, st)
+    return swap_stages(p.G, p.slot_order != nullptr) == 7 ? launch_swap_n<MODE, EPI_GROUPS, GATHER, 7, false>(ctx, name, w, x, w2, x2, p, st)
                                  : launch_swap_n<MODE, EPI_GROUPS, GATHER, 6, false>(ctx, name, w, x, w2, x2, p, st);
 }
 
 template <int MODE, int EPI_GROUPS, bool GATHER>
 bool swap_opt_in() {
     bool ok = cudaFuncSetAttribute(grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, 6, false>,
-                                   cudaFuncAttributeMaxDynamicSharedMemorySize, swap_smem_bytes(6, kMaxG)) == cudaSuccess &&
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, swap_smem_bytes(6, kMaxG, false, true)) == cudaSuccess &&
               cudaFuncSetAttribute(grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, 7, false>,
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, S_MAX_SMEM) == cudaSuccess;
     if constexpr (!GATHER)
         ok = ok && cudaFuncSetAttribute(grouped_gemm_swap_kernel<MODE, EPI_GROUPS, false, DUAL_STAGES, true>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        swap_smem_bytes(DUAL_STAGES, kMaxG, true)) == cudaSuccess;
+                                        swap_smem_bytes(DUAL_STAGES, kMaxG, true, true)) == cudaSuccess;
     return ok;
 }
 
@@ -682,14 +706,16 @@ int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int
         if (!map_interleaved(ctx, &d_gu, id.first, id.delta, dense->Fw, H)) return DIRECTOR_ERR_UNSUPPORTED;
     }
     const int d_rows = dense ? (int)dense->rows : 0, d_Fw = dense ? dense->Fw : 0;
-    SwapParams p1{seg_offsets, slot_expert, G, Fw / 128, H / BLOCK_K, Fw, Fw, ia.gate_first ? 1 : 0, hidden, ctx->d_status,
+    // the context's own slot table comes with its expert order (stored behind it); any other table is walked as is
+    const int32_t* order = (slot_expert == ctx->d_slot_expert && G == ctx->G && swap_can_order(G)) ? slot_expert + G : nullptr;
+    SwapParams p1{seg_offsets, slot_expert, order, G, Fw / 128, H / BLOCK_K, Fw, Fw, ia.gate_first ? 1 : 0, hidden, ctx->d_status,
                   counters, gather_rows, d_rows, d_Fw / 128, H / BLOCK_K, d_Fw, id.gate_first ? 1 : 0,
                   dense ? dense->hidden : nullptr, ctx->d_gemm_clock};
     const bool dual1 = (ctx->ffn_dual & 1) != 0, dual2 = (ctx->ffn_dual & 2) != 0;
     int rc = gather_rows ? launch_swap<0, EPI_GROUPS_GEMM1, true>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, d_gu, d_in, p1, false, st)
                          : launch_swap<0, EPI_GROUPS_GEMM1, false>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, d_gu, d_in, p1, dual1, st);
     if (rc != DIRECTOR_OK) return rc;
-    SwapParams p2{seg_offsets, slot_expert, G, H / 256, Fw / BLOCK_K, H, H, 1, out, ctx->d_status, counters + 1, nullptr,
+    SwapParams p2{seg_offsets, slot_expert, order, G, H / 256, Fw / BLOCK_K, H, H, 1, out, ctx->d_status, counters + 1, nullptr,
                   d_rows, H / 256, d_Fw / BLOCK_K, H, 1, dense ? dense->out : nullptr,
                   ctx->d_gemm_clock ? ctx->d_gemm_clock + 2 * kGemmClockCtas : nullptr};
     return launch_swap<1, EPI_GROUPS_GEMM2, false>(ctx, "grouped_gemm_down_kernel", m_d, m_h, d_d, d_h, p2, dual2, st);
