@@ -37,8 +37,8 @@ UNIT = "tokens/s"
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from the
 # committed ncu summary of that kernel on that workload (None until a capture for the workload exists).
 NCU_TRAFFIC_BYTES = {
-    # gate||up GEMM, full-size workload: 2 420 504 576 B read + 229 234 176 B written
-    "c2_mixtral": 2649738752,
+    # gate||up GEMM, full-size workload: 1 953 554 688 B read + 229 207 808 B written
+    "c2_mixtral": 2182762496,
 }
 
 
@@ -163,7 +163,7 @@ def build_layer(args, device):
     from paper_2607_08782_b200 import placement, synth
     from paper_2607_08782_b200.layer import MoELayer, bf16_bits_to_tensor
 
-    wl = synth.make_workload(args.config, args.tokens)
+    wl = synth.make_workload(args.config, args.tokens, E=args.experts)
     s, w = wl.shape, wl.weights
     wg, wu, wd = (bf16_bits_to_tensor(a, device) for a in (w.w_gate, w.w_up, w.w_down))
     sg = su = sd = None
@@ -450,6 +450,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c2_mixtral", choices=sorted(WORKLOAD_TEXT))
     ap.add_argument("--tokens", type=int, default=None, help="batch size override (c5_qwen3 sweep: 1, 64, 1024, 32768)")
+    ap.add_argument("--experts", type=int, default=None,
+                    help="cut the workload down to this many routed experts (same tile shapes, smaller device footprint: "
+                         "for profiler captures; not the headline workload)")
     ap.add_argument("--placement", default="auto", choices=["auto", "primary"])
     ap.add_argument("--ffn-variant", type=int, default=None, choices=[0, 1, 2, 3, 4, 5, 6],
                     help="expert-FFN tile scheme: 0 = one CTA per 128x256 tile, 1 = CTA pairs (256x256); default: library's")
@@ -722,7 +725,8 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": WORKLOAD_TEXT[args.config], "tokens": T, "placement": pname,
+        "config": {"workload": WORKLOAD_TEXT[args.config] + (f" [cut down to {s.E} experts]" if args.experts else ""),
+                   "tokens": T, "placement": pname,
                    "replica_policy": args.replica_policy,
                    "l2": "inputs larger than L2: every step streams the expert weights "
                          f"({3 * s.E * s.F * s.H * 2 / 1e9:.2f} GB) and activations through HBM",

@@ -72,6 +72,36 @@ def build_synth(force: bool = False) -> Path:
     return SYNTH_LIB
 
 
+def ptxas_summary() -> str:
+    """Compiles every CUDA source with ``-Xptxas -v`` (objects are thrown away) and returns one line per kernel:
+    source file, kernel, registers per thread, static shared memory, stack frame and spill bytes."""
+    import re
+    import tempfile
+    rows = ["file | kernel | registers | static smem B | stack B | spill stores B | spill loads B", "---|---|---|---|---|---|---"]
+    for src in director_sources():
+        with tempfile.NamedTemporaryFile(suffix=".o") as obj:
+            cmd = [_nvcc(), "-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
+                   "--expt-relaxed-constexpr", f"-I{INCLUDE}", f"-I{CSRC}", "-Xptxas", "-v", "-c", "-o", obj.name, str(src)]
+            res = subprocess.run(cmd, capture_output=True, text=True)
+        if res.returncode != 0:
+            raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+        lines = (res.stdout + res.stderr).splitlines()
+        for i, ln in enumerate(lines):
+            m = re.search(r"Compiling entry function '([^']+)'", ln)
+            if not m:
+                continue
+            name = subprocess.run(["c++filt", m.group(1)], capture_output=True, text=True).stdout.strip()
+            name = name.replace("(anonymous namespace)::", "").replace("director::", "").replace("void ", "")
+            name = re.sub(r"\(.*", "", name)
+            blob = " ".join(lines[i + 1:i + 4])
+            regs = re.search(r"Used (\d+) registers", blob)
+            smem = re.search(r"(\d+) bytes smem", blob)
+            spill = re.search(r"(\d+) bytes stack frame, (\d+) bytes spill stores, (\d+) bytes spill loads", blob)
+            rows.append(" | ".join([src.name, name, regs.group(1) if regs else "?", smem.group(1) if smem else "0",
+                                    *(spill.groups() if spill else ("?", "?", "?"))]))
+    return "\n".join(rows)
+
+
 def build_all(force: bool = False, verbose: bool = False) -> None:
     build_synth(force)
     build_director(force, verbose)
@@ -79,5 +109,8 @@ def build_all(force: bool = False, verbose: bool = False) -> None:
 
 if __name__ == "__main__":
     import sys
-    build_all(force="--force" in sys.argv, verbose="-v" in sys.argv)
-    print(DIRECTOR_LIB, SYNTH_LIB)
+    if "--ptxas-summary" in sys.argv:
+        print(ptxas_summary())
+    else:
+        build_all(force="--force" in sys.argv, verbose="-v" in sys.argv)
+        print(DIRECTOR_LIB, SYNTH_LIB)

@@ -156,20 +156,33 @@ struct SwapTile {
 __device__ __forceinline__ int sub_valid(const SwapTile& t, int j) { return min(max(t.valid - j * TOKEN_TILE, 0), TOKEN_TILE); }
 __device__ __forceinline__ int round_n(int valid) { return (valid + TOKEN_STEP - 1) / TOKEN_STEP * TOKEN_STEP; }
 
+// Work items in their hand-out order.  Consecutive segments of the walk that hold the same expert (the replicas of
+// an expert, adjacent when the segments are walked in expert order) form a group, and the items of a group are
+// ordered weight block first: for every weight block, the token tiles of all the group's segments.  The clusters
+// that run together therefore work on one weight block of one expert, whichever replica the tokens belong to, and
+// every weight tile is fetched from HBM once per step, not once per replica.
 struct SwapWalker {
     const int32_t* seg_off;     // first row of the i-th segment of the walk
     const int32_t* seg_end;     // one past its last row
     const int32_t* tt_start;    // prefix of work items (per weight block) per segment
     const int16_t* expert;
-    int w_blocks, w_rows_per_expert, rows_per_block, total, item_rows, g = 0;
+    int w_blocks, w_rows_per_expert, rows_per_block, total, item_rows, G;
+    int gs = 0, ge = 0;         // current group: segments [gs, ge) of the walk
     __device__ bool get(int w, SwapTile& t) {
         if (w >= total) return false;
-        while (w >= tt_start[g + 1] * w_blocks) ++g;
-        const int nt = tt_start[g + 1] - tt_start[g];
-        const int local = w - tt_start[g] * w_blocks;
+        while (w >= tt_start[ge] * w_blocks) {              // w only grows: groups are entered in order
+            gs = ge;
+            ge = gs + 1;
+            while (ge < G && expert[ge] == expert[gs]) ++ge;
+        }
+        const int nt = tt_start[ge] - tt_start[gs];         // token tiles of the group
+        const int local = w - tt_start[gs] * w_blocks;
         t.prob = 0;
         t.wb = local / nt;
-        const int tt = local - t.wb * nt;
+        const int tig = local - t.wb * nt;                  // tile inside the group
+        int g = gs;
+        while (tt_start[g + 1] - tt_start[gs] <= tig) ++g;  // its segment
+        const int tt = tig - (tt_start[g] - tt_start[gs]);
         t.row0 = seg_off[g] + tt * item_rows;
         t.valid = min(item_rows, seg_end[g] - t.row0);
         t.w_row = expert[g] * w_rows_per_expert + t.wb * rows_per_block;
@@ -177,10 +190,6 @@ struct SwapWalker {
     }
 };
 
-// MODE 0: gate/up + SwiGLU (A from the 3-D interleaving map).  MODE 1: down projection (A from a 2-D map).
-// GATHER (GEMM-1 only): the token rows are not read from a permuted copy but gathered straight from the layer
-// input x through row_token - tm_x then describes x with a one-row box and the whole producer warp issues the
-// loads, four rows per lane - so the dispatch step needs no row copies at all.
 // DUAL: a work item covers two consecutive token tiles of its segment (the last item of a segment may have one, or a
 // short second one).  Both tiles multiply the SAME weight tile, which is loaded once per k-step and feeds two MMAs
 // into the two accumulator buffers: 48 KB of operands per CTA and k-step for 2 x 256 tokens instead of 2 x 32 KB.
@@ -287,7 +296,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     const uint32_t tmem_base = *tmem_slot;
 
     constexpr int ROWS_PER_BLOCK = (MODE == 0) ? 128 : 256;   // weight rows (f or h) per pair block
-    SwapWalker walker{s_seg, s_end, s_tt, s_exp, p.w_blocks, p.w_rows_per_expert, ROWS_PER_BLOCK, s_tt[G] * p.w_blocks, ITEM_ROWS};
+    SwapWalker walker{s_seg, s_end, s_tt, s_exp, p.w_blocks, p.w_rows_per_expert, ROWS_PER_BLOCK, s_tt[G] * p.w_blocks, ITEM_ROWS, G};
     SwapTile t;
 
     // Work items (segment, weight block, token tile) are handed out dynamically, in their natural order, from a

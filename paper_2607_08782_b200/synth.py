@@ -128,12 +128,18 @@ SHAPES = {
 C5_SWEEP = (1, 64, 1024, 32768)
 
 
-def shape_for(name: str, T: int | None = None) -> Shape:
+def shape_for(name: str, T: int | None = None, E: int | None = None) -> Shape:
+    """The named workload's shape; T overrides the batch size (config 5's sweep), E the number of routed experts
+    (a cut-down copy of a workload with the same tile shapes and a smaller device footprint, for profiler captures)."""
     s = SHAPES[name]
-    if T is None or T == s.T:
+    if (T is None or T == s.T) and (E is None or E == s.E):
         return s
+    T = s.T if T is None else T
+    E = s.E if E is None else E
+    if not (s.K <= E <= s.E):
+        raise ValueError(f"{name}: experts must be in [{s.K}, {s.E}]")
     seed = s.seed + (C5_SWEEP.index(T) if (name == "c5_qwen3" and T in C5_SWEEP) else 0)
-    return Shape(s.name, T, s.H, s.E, s.K, s.F, s.S, s.R, s.C_max, s.zipf_s, seed,
+    return Shape(s.name, T, s.H, E, s.K, s.F, s.S, s.R, s.C_max, s.zipf_s, seed,
                  s.segment_tokens, s.zipf_s_range)
 
 
@@ -215,7 +221,7 @@ def primary_ranks(shape: Shape) -> np.ndarray:
     if shape.name == "c3_dsv2lite":
         return e // 8
     if shape.name == "c4_qwen15":
-        return (e * 8) // 60
+        return (e * 8) // max(E, 60)
     if shape.name == "c5_qwen3":
         return e % R
     raise KeyError(shape.name)
@@ -237,8 +243,8 @@ class Workload:
     X_primary: np.ndarray = field(default=None)
 
 
-def make_workload(name: str, T: int | None = None, with_weights: bool = True) -> Workload:
-    shape = shape_for(name, T)
+def make_workload(name: str, T: int | None = None, with_weights: bool = True, E: int | None = None) -> Workload:
+    shape = shape_for(name, T, E)
     return Workload(
         shape=shape,
         logits=make_logits(shape),
