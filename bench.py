@@ -552,7 +552,9 @@ def main():
         (mhz1, us1), (mhz2, us2) = layer.d.gemm_sm_mhz(0), layer.d.gemm_sm_mhz(1)
         kernel_clock = {"gate_up_sm_mhz": round(mhz1, 1), "gate_up_us": round(us1, 1), "down_sm_mhz": round(mhz2, 1),
                         "down_us": round(us2, 1),
-                        "how": "cycle counter / global timer inside the last launch of the timed region (tile scheme 2)"}
+                        "how": "cycle counter / global timer inside the last launch of the timed region (tile scheme 2)",
+                        "gate_up": {k: round(v, 4) for k, v in layer.d.gemm_counters(0).items()},
+                        "down": {k: round(v, 4) for k, v in layer.d.gemm_counters(1).items()}}
     except Exception:
         kernel_clock = None
     kernel_ms = {}

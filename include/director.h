@@ -314,6 +314,19 @@ int director_set_ffn_variant(director_ctx* ctx, int32_t variant);
  * the kernel itself, the one a tensor-pipe roofline has to be read against.  Negative on error. */
 double director_gemm_sm_mhz(director_ctx* ctx, int32_t which, double* busy_us);
 
+/* What the expert GEMM kernels (default tile scheme) measured about themselves in their most recent launch, summed
+ * over the CTAs; which: 0 = gate|up GEMM, 1 = down GEMM; out: host int64 [DIRECTOR_GEMM_COUNTERS].  Synchronises
+ * the device.  All times are SM cycles of the reading thread unless noted:
+ *   [0] cycles and [1] nanoseconds every CTA spent in the kernel (cycles / ns = SM clock);
+ *   the MMA-issuing thread of every CTA pair: [2] cycles waiting for a free accumulator buffer (the epilogue of
+ *   an earlier tile had not finished), [3] cycles from an item's first operand wait to the issue of its last MMA,
+ *   [4] k-steps issued, [5] work items (so [3] / [4] = cycles per k-step as the issuing thread sees them);
+ *   one epilogue warp of every CTA: [6] cycles waiting for a complete accumulator, [7] cycles draining
+ *   accumulators (tensor memory -> registers -> bf16 -> global), [8] token tiles drained;
+ *   [9] reserved;  [10] the longest CTA's nanoseconds;  [11] number of CTAs summed. */
+#define DIRECTOR_GEMM_COUNTERS 12
+int director_gemm_counters(director_ctx* ctx, int32_t which, int64_t* out);
+
 /* Number of kernels this context has launched since it was created. */
 int64_t director_launch_count(const director_ctx* ctx);
 

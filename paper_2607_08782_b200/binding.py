@@ -27,7 +27,7 @@ EXPORTED = (
     "director_expert_ffn_gather", "director_set_replica_policy", "director_dispatch_src",
     "director_dedup_dispatch_tokens", "director_route_dispatch_cost", "director_layer_forward",
     "director_reserve_placements", "director_select_placement", "director_set_profiling_filter",
-    "director_selftest_bounded_wait", "director_gemm_sm_mhz",
+    "director_selftest_bounded_wait", "director_gemm_sm_mhz", "director_gemm_counters",
 )
 
 REPLICA_ROUND_ROBIN, REPLICA_LOCAL_FIRST = 0, 1
@@ -85,6 +85,7 @@ def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.director_selftest_bounded_wait.argtypes = [vp, c_uint64, vp, vp]
     lib.director_gemm_sm_mhz.argtypes = [vp, c_int32, POINTER(c_double)]
     lib.director_gemm_sm_mhz.restype = c_double
+    lib.director_gemm_counters.argtypes = [vp, c_int32, POINTER(c_int64)]
     lib.director_kernel_time.argtypes = [vp, c_char_p, POINTER(c_int64)]
     lib.director_kernel_time.restype = c_double
     lib.director_status_string.argtypes = [c_int]
@@ -261,6 +262,25 @@ class Director:
         if mhz < 0:
             raise DirectorError(4, "director_gemm_sm_mhz")
         return mhz, float(busy.value)
+
+    def gemm_counters(self, which: int = 0) -> dict:
+        """What the most recent gate|up (0) or down (1) GEMM launch measured about itself (see
+        director_gemm_counters), as derived figures."""
+        raw = (c_int64 * 12)()
+        _check(self.lib.director_gemm_counters(self._ctx, which, raw), "director_gemm_counters")
+        c = [int(v) for v in raw]
+        pairs = max(c[11] // 2, 1)
+        return {
+            "sm_mhz": c[0] / c[1] * 1e3 if c[1] else 0.0,
+            "cycles_per_cta": c[0] / max(c[11], 1),
+            "k_steps_per_pair": c[4] / pairs, "items_per_pair": c[5] / pairs,
+            "cycles_per_k_step": c[3] / c[4] if c[4] else 0.0,
+            "issuer_wait_for_accumulator_frac": c[2] / (c[0] / 2) if c[0] else 0.0,
+            "issuer_k_loop_frac": c[3] / (c[0] / 2) if c[0] else 0.0,
+            "epilogue_drain_cycles_per_tile": c[7] / c[8] if c[8] else 0.0,
+            "epilogue_wait_cycles_per_tile": c[6] / c[8] if c[8] else 0.0,
+            "longest_cta_us": c[10] * 1e-3,
+        }
 
     def launch_count(self) -> int:
         return int(self.lib.director_launch_count(self._ctx))

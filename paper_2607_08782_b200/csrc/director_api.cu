@@ -125,7 +125,7 @@ int director_create(const director_shape* shape, director_ctx** out) {
               dev_alloc(&c->d_host_mask, s.E) && dev_alloc(&c->d_tile_rep, (size_t)c->n_tiles_max * c->G) &&
               dev_alloc(&c->d_one_seg, 2) && dev_alloc(&c->d_sched, 4) &&
               dev_alloc(&c->d_zero_expert, 1) &&
-              dev_alloc(&c->d_gemm_clock, 4 * (size_t)kGemmClockCtas) &&
+              dev_alloc(&c->d_gemm_clock, 2 * (size_t)kGemmClockWords * kGemmClockCtas) &&
               dev_alloc(reinterpret_cast<uint16_t**>(&c->d_hidden), A * s.F) &&
               dev_alloc(reinterpret_cast<uint16_t**>(&c->d_hidden_shared), T * s.S * s.F) &&
               dev_alloc(&c->e_logits2[0], T * s.E) && dev_alloc(&c->e_logits2[1], T * s.E) &&
@@ -149,7 +149,7 @@ int director_create(const director_shape* shape, director_ctx** out) {
     ok = cudaMemset(c->d_ticket, 0, 4 * sizeof(unsigned int)) == cudaSuccess &&
          cudaMemset(c->d_status, 0, sizeof(int32_t)) == cudaSuccess &&
          cudaMemset(c->d_zero_expert, 0, sizeof(int32_t)) == cudaSuccess &&
-         cudaMemset(c->d_gemm_clock, 0, sizeof(unsigned long long) * 4 * kGemmClockCtas) == cudaSuccess;
+         cudaMemset(c->d_gemm_clock, 0, sizeof(unsigned long long) * 2 * kGemmClockWords * kGemmClockCtas) == cudaSuccess;
 
     cudaDriverEntryPointQueryResult qres;
     if (ok) {
@@ -605,22 +605,29 @@ int director_set_ffn_variant(director_ctx* ctx, int32_t variant) {
 
 int director_pair_clusters(const director_ctx* ctx) { return ctx ? ctx->pair_clusters : -1; }
 
-double director_gemm_sm_mhz(director_ctx* ctx, int32_t which, double* busy_us) {
-    if (ctx == nullptr || which < 0 || which > 1) return -1.0;
-    if (cudaDeviceSynchronize() != cudaSuccess) return -1.0;
-    std::vector<unsigned long long> h(2 * (size_t)kGemmClockCtas);
-    if (cudaMemcpy(h.data(), ctx->d_gemm_clock + (size_t)which * 2 * kGemmClockCtas, h.size() * sizeof(unsigned long long),
-                   cudaMemcpyDeviceToHost) != cudaSuccess)
-        return -1.0;
+int director_gemm_counters(director_ctx* ctx, int32_t which, int64_t* out) {
+    if (ctx == nullptr || which < 0 || which > 1 || out == nullptr) return DIRECTOR_ERR_INVALID_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return DIRECTOR_ERR_CUDA;
+    std::vector<unsigned long long> h((size_t)kGemmClockWords * kGemmClockCtas);
+    if (cudaMemcpy(h.data(), ctx->d_gemm_clock + (size_t)which * kGemmClockWords * kGemmClockCtas,
+                   h.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return DIRECTOR_ERR_CUDA;
     const int ctas = std::min(2 * ctx->pair_clusters, (int)kGemmClockCtas);
-    double cycles = 0.0, ns = 0.0, ns_max = 0.0;
+    for (int k = 0; k < DIRECTOR_GEMM_COUNTERS; ++k) out[k] = 0;
     for (int i = 0; i < ctas; ++i) {
-        cycles += (double)h[2 * i];
-        ns += (double)h[2 * i + 1];
-        ns_max = std::max(ns_max, (double)h[2 * i + 1]);
+        const unsigned long long* r = h.data() + (size_t)i * kGemmClockWords;
+        for (int k = 0; k < kGemmClockWords; ++k) out[k] += (int64_t)r[k];
+        out[kGemmClockWords] = std::max<int64_t>(out[kGemmClockWords], (int64_t)r[1]);   // longest CTA, ns
     }
-    if (busy_us) *busy_us = ns_max * 1e-3;
-    return ns > 0.0 ? cycles / ns * 1e3 : 0.0;
+    out[kGemmClockWords + 1] = ctas;
+    return DIRECTOR_OK;
+}
+
+double director_gemm_sm_mhz(director_ctx* ctx, int32_t which, double* busy_us) {
+    int64_t c[DIRECTOR_GEMM_COUNTERS];
+    if (director_gemm_counters(ctx, which, c) != DIRECTOR_OK) return -1.0;
+    if (busy_us) *busy_us = (double)c[kGemmClockWords] * 1e-3;
+    return c[1] > 0 ? (double)c[0] / (double)c[1] * 1e3 : 0.0;
 }
 
 int64_t director_launch_count(const director_ctx* ctx) { return ctx ? ctx->launches : -1; }

@@ -20,7 +20,8 @@ constexpr int kMaxR = 64;
 constexpr int kMaxC = 16;
 constexpr int kMaxG = kMaxR * kMaxC;
 constexpr int kSmallFfnTokens = 4;      // batches of at most this many tokens take the weight-streaming FFN kernels
-constexpr int kGemmClockCtas = 512;   // CTAs per GEMM launch whose {cycles, ns} records fit the clock buffer
+constexpr int kGemmClockCtas = 512;   // CTAs per GEMM launch whose records fit the clock buffer
+constexpr int kGemmClockWords = 10;   // 64-bit words per CTA record, see director_gemm_counters
 
 struct KernelEvent {
     const char* name;
@@ -71,7 +72,7 @@ struct director_ctx {
     unsigned int* d_sched = nullptr;   // [4] work-item counters of the GEMM launches of one expert_ffn call
     int32_t* d_one_seg = nullptr;      // [2] segment table {0, T} used for the shared experts
     int32_t* d_zero_expert = nullptr;  // [1] = {0}
-    unsigned long long* d_gemm_clock = nullptr;   // [2][kGemmClockCtas][2] {SM cycles, ns} per CTA of the last gate|up / down launch
+    unsigned long long* d_gemm_clock = nullptr;   // [2][kGemmClockCtas][kGemmClockWords] per-CTA records of the last gate|up / down launch
 
     // buffers of the host-buffer entry points; inputs, y and the histograms exist twice so that the
     // copies of one batch overlap the kernels of its neighbours

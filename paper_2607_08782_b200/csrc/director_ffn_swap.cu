@@ -138,9 +138,10 @@ struct SwapParams {
     int dense_out_pitch;
     int dense_gate_first;
     void* dense_out;
-    // Optional: every CTA writes {SM cycles, nanoseconds} it spent in the kernel to clock_out[2 * blockIdx.x .. +1]
-    // (clock64 and the global timer read by one thread at both ends): cycles / ns is the SM clock the kernel really
-    // ran at, which a host-side sampler with millisecond resolution cannot see.
+    // Optional: every CTA writes a record of kGemmClockWords 64-bit words about itself (see director_gemm_counters):
+    // SM cycles and nanoseconds spent in the kernel (clock64 and the global timer read by one thread at both ends:
+    // cycles / ns is the SM clock the kernel really ran at, which a host-side sampler with millisecond resolution
+    // cannot see), and where the MMA-issuing thread and one epilogue warp spent their cycles.
     unsigned long long* clock_out;
 };
 
@@ -167,9 +168,26 @@ struct SwapWalker {
     const int32_t* tt_start;    // prefix of work items (per weight block) per segment
     const int16_t* expert;
     int w_blocks, w_rows_per_expert, rows_per_block, total, item_rows, G;
+    bool grouped;               // false: every segment is its own group (the walk is in slot order)
     int gs = 0, ge = 0;         // current group: segments [gs, ge) of the walk
     __device__ bool get(int w, SwapTile& t) {
         if (w >= total) return false;
+        if (!grouped) {
+            // one segment per group: the short form of the code below (the decode of an item is on the scheduler
+            // thread's critical path when items are short, as in the down projection of a decode-sized batch)
+            int g = gs;
+            while (w >= tt_start[g + 1] * w_blocks) ++g;
+            gs = g;
+            const int nt = tt_start[g + 1] - tt_start[g];
+            const int local = w - tt_start[g] * w_blocks;
+            t.prob = 0;
+            t.wb = local / nt;
+            const int tt = local - t.wb * nt;
+            t.row0 = seg_off[g] + tt * item_rows;
+            t.valid = min(item_rows, seg_end[g] - t.row0);
+            t.w_row = expert[g] * w_rows_per_expert + t.wb * rows_per_block;
+            return true;
+        }
         while (w >= tt_start[ge] * w_blocks) {              // w only grows: groups are entered in order
             gs = ge;
             ge = gs + 1;
@@ -238,6 +256,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     const bool leader = rank == 0;
     long long clk0 = 0;
     unsigned long long ns0 = 0;
+    long long stat_a = 0, stat_b = 0, stat_c = 0, stat_d = 0;      // per-role cycle counters, see SwapParams::clock_out
     if (threadIdx.x == 0) { clk0 = clock64(); ns0 = global_ns(); }
 
     constexpr int n_threads = 96 + 128 * EPI_GROUPS;               // producer, MMA and scheduler warps + epilogue warps
@@ -296,7 +315,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     const uint32_t tmem_base = *tmem_slot;
 
     constexpr int ROWS_PER_BLOCK = (MODE == 0) ? 128 : 256;   // weight rows (f or h) per pair block
-    SwapWalker walker{s_seg, s_end, s_tt, s_exp, p.w_blocks, p.w_rows_per_expert, ROWS_PER_BLOCK, s_tt[G] * p.w_blocks, ITEM_ROWS, G};
+    SwapWalker walker{s_seg, s_end, s_tt, s_exp, p.w_blocks, p.w_rows_per_expert, ROWS_PER_BLOCK, s_tt[G] * p.w_blocks, ITEM_ROWS, G, ordered};
     SwapTile t;
 
     // Work items (segment, weight block, token tile) are handed out dynamically, in their natural order, from a
@@ -429,6 +448,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 const int n_sub = (DUAL && t.valid > TOKEN_TILE) ? 2 : 1;
                 uint32_t d_tmem[2], idesc[2];
                 int acc[2];
+                const long long c_item = clock64();
                 for (int j = 0; j < n_sub && ok; ++j) {
                     acc[j] = (int)((tile_no + j) & 1u);
                     ok = mbar_wait(tempty_bar(acc[j]), ((((tile_no + j) >> 1) & 1u) ^ 1u), abort_flag);
@@ -439,6 +459,10 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 tile_no += (uint32_t)n_sub;
                 tc_fence_after();
                 const int k_steps = t.prob ? p.dense_k_steps : p.k_steps;
+                const long long c_loop = clock64();
+                stat_a += c_loop - c_item;                  // waited for the accumulator buffer(s)
+                stat_c += k_steps;
+                stat_d += 1;
                 for (int kb = 0; kb < k_steps; ++kb) {
                     if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag))) break;
                     tc_fence_after();
@@ -465,6 +489,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                     umma_commit_both(empty_bar(stage));
                     if (++stage == S_STAGES) { stage = 0; phase ^= 1u; }
                 }
+                stat_b += clock64() - c_loop;               // operand waits and MMA issue of the item's k loop
             }
         }
     } else if (warp == 2) {
@@ -526,7 +551,10 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
             for (int sub = 0; sub < n_sub && ok; ++sub, ++tile_no) {
                 const int acc = (int)(tile_no & 1u);
                 const int row0 = t.row0 + sub * TOKEN_TILE, valid = sub_valid(t, sub), n = round_n(valid);
+                const long long c_wait = clock64();
                 if (!(ok = mbar_wait(tfull_bar(acc), (tile_no >> 1) & 1u, abort_flag))) break;
+                const long long c_drain = clock64();
+                stat_a += c_drain - c_wait;
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * TOKEN_TILE);
                 if constexpr (MODE == 0) {
@@ -577,6 +605,8 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+                stat_b += clock64() - c_drain;
+                stat_c += 1;
             }
         }
     }
@@ -585,9 +615,23 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     __syncthreads();
     cluster_sync_all();
     if (threadIdx.x == 0 && *abort_flag) director_set_status(p.status, DIRECTOR_ERR_TIMEOUT);
-    if (threadIdx.x == 0 && p.clock_out != nullptr && blockIdx.x < (unsigned)kGemmClockCtas) {
-        p.clock_out[2 * blockIdx.x] = (unsigned long long)(clock64() - clk0);
-        p.clock_out[2 * blockIdx.x + 1] = global_ns() - ns0;
+    unsigned long long* const rec = (p.clock_out != nullptr && blockIdx.x < (unsigned)kGemmClockCtas)
+                                        ? p.clock_out + (size_t)blockIdx.x * kGemmClockWords : nullptr;
+    if (threadIdx.x == 0 && rec != nullptr) {
+        rec[0] = (unsigned long long)(clock64() - clk0);
+        rec[1] = global_ns() - ns0;
+        rec[9] = 0ull;
+    }
+    if (threadIdx.x == 32 && rec != nullptr) {              // the MMA-issuing thread (idle in the peer CTA: zeros)
+        rec[2] = (unsigned long long)stat_a;
+        rec[3] = (unsigned long long)stat_b;
+        rec[4] = (unsigned long long)stat_c;
+        rec[5] = (unsigned long long)stat_d;
+    }
+    if (threadIdx.x == 96 && rec != nullptr) {              // lane 0 of the first epilogue warp
+        rec[6] = (unsigned long long)stat_a;
+        rec[7] = (unsigned long long)stat_b;
+        rec[8] = (unsigned long long)stat_c;
     }
     if (warp == 1) {
         tc_fence_after();
@@ -726,7 +770,7 @@ int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int
     if (rc != DIRECTOR_OK) return rc;
     SwapParams p2{seg_offsets, slot_expert, order, G, H / 256, Fw / BLOCK_K, H, H, 1, out, ctx->d_status, counters + 1, nullptr,
                   d_rows, H / 256, d_Fw / BLOCK_K, H, 1, dense ? dense->out : nullptr,
-                  ctx->d_gemm_clock ? ctx->d_gemm_clock + 2 * kGemmClockCtas : nullptr};
+                  ctx->d_gemm_clock ? ctx->d_gemm_clock + (size_t)kGemmClockWords * kGemmClockCtas : nullptr};
     return launch_swap<1, EPI_GROUPS_GEMM2, false>(ctx, "grouped_gemm_down_kernel", m_d, m_h, d_d, d_h, p2, dual2, st);
 }
 
