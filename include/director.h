@@ -154,7 +154,12 @@ int director_dedup_dispatch_tokens(director_ctx* ctx, int32_t T, const int32_t* 
  * Shared experts (only if the context has S > 0 and x != NULL): the S always-on FFNs applied
  * to every token's own row, summed: x: dev bf16 [T,H]; ws_gate, ws_up: dev bf16 [S*F,H] (the S
  * experts stacked); ws_down: dev bf16 [H,S*F] (the S experts side by side);
- * y_shared: dev bf16 [T,H]. */
+ * y_shared: dev bf16 [T,H].
+ * Batches of more than 4 tokens run as two grouped GEMMs on the tensor cores (tcgen05, accumulators in tensor
+ * memory, operands by TMA).  A batch of at most 4 tokens is a stream of the touched experts' weights through a few
+ * dot products, bound by HBM bandwidth: it runs as two weight-streaming kernels (one warp per pair of output
+ * features, fp32 accumulation in a fixed order), which use every SM whatever the number of segments.  Both paths
+ * round Hg to bf16 between the projections; their results agree within the layer's tolerance, not bit for bit. */
 int director_expert_ffn(director_ctx* ctx, int32_t T, const void* xp, const int32_t* seg_offsets,
                         const void* w_gate, const void* w_up, const void* w_down, void* yp,
                         const void* x, const void* ws_gate, const void* ws_up, const void* ws_down,
@@ -223,7 +228,8 @@ int director_placement_cost_batch(director_ctx* ctx, const int64_t* workload, in
  * Inputs, all dev: topk_idx int32 [T,K]; the placement as replica tables: rep_start int32 [E+1]
  * (exclusive prefix of replica counts, rep_start[0] = 0) and rep_slot int32 [rep_start[E]], the slot
  * g = rank*C_max + p of each replica, an expert's replicas in ascending rank order (slot numbering as
- * in the header comment; the caller builds the tables, they are not validated).
+ * in the header comment; the caller builds the tables: an expert that is routed to but has no replica, or a
+ * slot outside [0, R*C_max), is skipped and reported as DIRECTOR_ERR_BAD_INDEX, the assignment's row is -1).
  * Outputs, all dev: row_token int32 [T*K], inv_row int32 [T,K], dest_rank int32 [T,K], seg_offsets
  * int32 [R*C_max+1], exactly as director_dispatch writes them.  device_status: dev int32 [1] that the
  * caller has zeroed, receives DIRECTOR_ERR_BAD_INDEX if an expert id outside [0,E) was skipped; may be
@@ -297,11 +303,17 @@ int director_last_status(director_ctx* ctx, void* stream);
  * Returns DIRECTOR_ERR_INVALID_ARG for a limit outside the range. */
 int director_selftest_bounded_wait(director_ctx* ctx, uint64_t limit_ns, uint64_t* waited_ns, void* stream);
 
-/* Tile scheme of the expert-FFN GEMMs (results are bit-identical across schemes):
+/* Tile scheme of the expert-FFN GEMMs (results are bit-identical across the tensor-core schemes):
  *   2 (default) weight-stationary CTA pairs: 256 weight rows x up to 256 tokens per tile, the token count
  *               of a tile is a runtime operand in steps of 32, so ragged segment tails cost almost nothing;
+ *               batches of at most 4 tokens take the weight-streaming kernels instead (see director_expert_ffn);
  *   1           token-stationary CTA pairs: 256 tokens x 256 weight rows per tile;
- *   0           token-stationary single CTAs: 128 tokens x 256 weight rows per tile.
+ *   0           token-stationary single CTAs: 128 tokens x 256 weight rows per tile;
+ *   3 / 4 / 5   scheme 2 with TWO token tiles per work item (one weight tile feeds two MMAs into the two
+ *               accumulator buffers) in both GEMMs / the gate|up GEMM only / the down GEMM only - measured
+ *               slower than scheme 2 (the accumulator drain is no longer hidden, the operand ring is shallower),
+ *               kept selectable as the record of that experiment;
+ *   6           scheme 2 with the tensor-core kernels for every batch size.
  * Scheme 2 falls back to scheme 0 when w_gate and w_up cannot be described by one strided tensor map
  * (their addresses differ by 2^40 bytes or more). */
 int director_set_ffn_variant(director_ctx* ctx, int32_t variant);

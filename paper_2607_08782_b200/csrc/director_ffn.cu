@@ -33,6 +33,7 @@ int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int
                   const void* w_down, uint64_t n_experts, int Fw, void* hidden, void* out, unsigned int* counters,
                   const DenseFfn* dense, cudaStream_t st);
 int ffn_small_init(director_ctx* ctx);  // director_ffn_small.cu
+bool ffn_small_applies(const director_ctx* ctx, int T, int Fw);
 int ffn_pass_small(director_ctx* ctx, const void* in, const int32_t* seg_offsets, const int32_t* slot_expert, int G,
                    const void* w_gate, const void* w_up, const void* w_down, int Fw, void* hidden, void* out, int rows_max,
                    int max_segments, cudaStream_t st);
@@ -328,7 +329,8 @@ int launch_expert_ffn(director_ctx* ctx, int T, const void* xp, const int32_t* r
     const director_shape& s = ctx->shape;
     const uint64_t A = (uint64_t)T * s.K;
     const bool shared = s.S > 0 && x != nullptr && y_shared != nullptr;
-    if (ctx->ffn_variant == 2 && ctx->ffn_small && row_token == nullptr && T <= kSmallFfnTokens) {
+    if (ctx->ffn_variant == 2 && ctx->ffn_small && row_token == nullptr && ffn_small_applies(ctx, T, s.F) &&
+        (!shared || ffn_small_applies(ctx, T, s.S * s.F))) {
         // decode-sized batch: every segment has at most T rows; stream the touched weights once, feature by feature
         int rc = ffn_pass_small(ctx, xp, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up, w_down, s.F, ctx->d_hidden,
                                 yp, T, (int)std::min<uint64_t>((uint64_t)ctx->G, A), st);

@@ -93,3 +93,47 @@ def test_static_entry_point_rejects_problems_beyond_its_fixed_scratch():
     assert rc == 9 and "fixed scratch" in binding.status_string(rc)
     assert lib.director_dispatch_index_static(0, 2, 128, 16, 9, p, p, p, p, p, p, p, None, None) == 1
     assert lib.director_dispatch_index_static(64, 2, 128, 16, 9, None, p, p, p, p, p, p, None, None) == 1
+
+
+def test_static_entry_point_skips_and_flags_a_routed_expert_without_a_replica():
+    """Caller-built tables are not trusted: an expert that tokens are routed to but that has no replica in the
+    tables is skipped (row -1), DIRECTOR_ERR_BAD_INDEX is raised in the status word, nothing is written out of bounds
+    and every other assignment is placed exactly as the oracle places it on the remaining experts."""
+    import torch
+    from paper_2607_08782_b200 import binding
+    E, K, R, C, T = 6, 2, 3, 2, 500
+    dev = "cuda"
+    rng = np.random.default_rng(5)
+    idx = np.stack([rng.permutation(E)[:K] for _ in range(T)]).astype(np.int32)
+    X = synth.placement_from_ranks(np.arange(E) % R, R)
+    rep_start, rep_slot = _replica_tables(X, C)
+    # drop expert 2's only replica from the tables: rep_start keeps its prefix form, expert 2 gets zero replicas
+    lo, hi = int(rep_start[2]), int(rep_start[3])
+    bad_slot = np.delete(rep_slot, np.arange(lo, hi))
+    bad_start = rep_start.copy()
+    bad_start[3:] -= (hi - lo)
+    d_idx = torch.from_numpy(idx).to(dev)
+    A = T * K
+    guard = 64                                               # canaries around every output
+    bufs = {n: torch.full((size + 2 * guard,), -7, dtype=torch.int32, device=dev)
+            for n, size in (("row_token", A), ("inv_row", A), ("dest_rank", A), ("seg", R * C + 1))}
+    view = {n: b[guard:-guard] for n, b in bufs.items()}
+    status = torch.zeros((1,), dtype=torch.int32, device=dev)
+    binding.dispatch_index_static(T, K, E, R, C, d_idx, torch.from_numpy(bad_start).to(dev),
+                                  torch.from_numpy(bad_slot).to(dev), view["row_token"], view["inv_row"].view(T, K),
+                                  view["dest_rank"].view(T, K), view["seg"], status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 7                           # DIRECTOR_ERR_BAD_INDEX
+    for n, b in bufs.items():                                # nothing outside the arrays was touched
+        assert bool((b[:guard] == -7).all()) and bool((b[-guard:] == -7).all()), n
+    inv = view["inv_row"].view(T, K).cpu().numpy()
+    hit = idx == 2
+    assert (inv[hit] == -1).all() and (inv[~hit] >= 0).all()
+    assert int(view["seg"][-1]) == int((~hit).sum())
+    # the remaining assignments: same rows as the oracle gives when expert 2's choices are routed nowhere, i.e. the
+    # permutation of the other experts' assignments is unchanged by the hole
+    rows = inv[~hit]
+    assert len(np.unique(rows)) == len(rows) and rows.max() == len(rows) - 1
+    rt = view["row_token"].cpu().numpy()[:len(rows)]
+    tok = np.repeat(np.arange(T), K).reshape(T, K)[~hit]
+    assert np.array_equal(rt[rows], tok)
