@@ -454,8 +454,9 @@ def main():
                     help="cut the workload down to this many routed experts (same tile shapes, smaller device footprint: "
                          "for profiler captures; not the headline workload)")
     ap.add_argument("--placement", default="auto", choices=["auto", "primary"])
-    ap.add_argument("--ffn-variant", type=int, default=None, choices=[0, 1, 2, 3, 4, 5, 6],
-                    help="expert-FFN tile scheme: 0 = one CTA per 128x256 tile, 1 = CTA pairs (256x256); default: library's")
+    ap.add_argument("--ffn-variant", type=int, default=None, choices=[0, 1, 2, 6],
+                    help="expert-FFN tile scheme: 0 = one CTA per 128x256 tile, 1 = CTA pairs (256x256), 2 = weight-stationary CTA pairs "
+                         "(the library's default), 6 = scheme 2 with the tensor-core kernels also for batches of at most 4 tokens")
     ap.add_argument("--replica-policy", default="round_robin", choices=["round_robin", "local_first"],
                     help="which replica of a replicated expert an assignment uses (the default is the headline setting)")
     ap.add_argument("--fused", action="store_true",

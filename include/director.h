@@ -309,10 +309,6 @@ int director_selftest_bounded_wait(director_ctx* ctx, uint64_t limit_ns, uint64_
  *               batches of at most 4 tokens take the weight-streaming kernels instead (see director_expert_ffn);
  *   1           token-stationary CTA pairs: 256 tokens x 256 weight rows per tile;
  *   0           token-stationary single CTAs: 128 tokens x 256 weight rows per tile;
- *   3 / 4 / 5   scheme 2 with TWO token tiles per work item (one weight tile feeds two MMAs into the two
- *               accumulator buffers) in both GEMMs / the gate|up GEMM only / the down GEMM only - measured
- *               slower than scheme 2 (the accumulator drain is no longer hidden, the operand ring is shallower),
- *               kept selectable as the record of that experiment;
  *   6           scheme 2 with the tensor-core kernels for every batch size.
  * Scheme 2 falls back to scheme 0 when w_gate and w_up cannot be described by one strided tensor map
  * (their addresses differ by 2^40 bytes or more). */

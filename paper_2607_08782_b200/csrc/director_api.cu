@@ -594,10 +594,8 @@ int director_last_status(director_ctx* ctx, void* stream) {
 
 int director_set_ffn_variant(director_ctx* ctx, int32_t variant) {
     REQUIRE_CTX(ctx);
-    if (variant < 0 || variant > 6) return DIRECTOR_ERR_INVALID_ARG;
-    // 3, 4, 5: scheme 2 with two token tiles per work item in both GEMMs / the gate|up GEMM only / the down GEMM only
+    if (variant < 0 || (variant > 2 && variant != 6)) return DIRECTOR_ERR_INVALID_ARG;
     // 6: scheme 2 with the tensor-core kernels for every batch size (no weight-streaming path for tiny batches)
-    ctx->ffn_dual = variant == 3 ? 3 : variant == 4 ? 1 : variant == 5 ? 2 : 0;
     ctx->ffn_small = variant == 2;
     ctx->ffn_variant = variant > 2 ? 2 : variant;
     return DIRECTOR_OK;

@@ -97,7 +97,7 @@ struct director_ctx {
     int pair_clusters = 0;              // CTA pairs the device can hold at once (pair variant's grid)
     int ffn_variant = 2;                // tile scheme of the expert-FFN GEMMs, see director_set_ffn_variant
     bool ffn_small = true;              // decode-sized batches (T <= kSmallFfnTokens) use the weight-streaming kernels
-    int ffn_dual = 0;                   // bit 0 / bit 1: the gate|up / down GEMM takes two token tiles per work item
+    bool gemm_stats = true;             // the expert GEMMs record their own clock and per-role cycle counters
     void* encode_tiled = nullptr;       // cuTensorMapEncodeTiled, resolved through the runtime
 
     int64_t launches = 0;

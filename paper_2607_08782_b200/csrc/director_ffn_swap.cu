@@ -30,28 +30,23 @@ using namespace umma;
 
 namespace {
 
-// A stage of the operand ring holds, per CTA and k-step, 16 KB of weights and 16 KB of tokens for every token tile
-// of the work item: one tile (32 KB) or, in the DUAL form, two tiles that share the weights (48 KB).
-constexpr int stage_bytes(bool dual) { return A_BYTES + (dual ? 2 : 1) * B_HALF_BYTES; }
-constexpr int S_STAGE_BYTES = stage_bytes(false);
+constexpr int S_STAGE_BYTES = A_BYTES + B_HALF_BYTES;          // 16 KB weights + 16 KB tokens per CTA per k-step
 constexpr int S_HEADER_BYTES = 384;                            // barriers, scheduler ring, TMEM slot, scratch
 constexpr int S_MAX_SMEM = 232448;                             // opt-in shared memory per CTA on sm_100
 // Shared memory of a launch: alignment slack, the operand ring, the header, and the segment tables of its G slots
 // (seg_offsets and token-tile prefix as int32, expert ids as int16).
 // (segment starts, work-item prefix as int32, expert ids as int16; segment ends as int32 when the segments are
 // walked in expert order rather than slot order).
-constexpr int swap_smem_bytes(int stages, int G, bool dual = false, bool ordered = false) {
-    return 1024 + stages * stage_bytes(dual) + S_HEADER_BYTES + (G + 1) * (ordered ? 14 : 10) + 6;
+constexpr int swap_smem_bytes(int stages, int G, bool ordered = false) {
+    return 1024 + stages * S_STAGE_BYTES + S_HEADER_BYTES + (G + 1) * (ordered ? 14 : 10) + 6;
 }
 // The operand stream is latency-bound (a stage comes back ~2.5 us after it is released), so the ring is as deep as
 // shared memory allows: seven stages when the segment tables are small enough, else six.
-inline int swap_stages(int G, bool ordered = false) { return swap_smem_bytes(7, G, false, ordered) <= S_MAX_SMEM ? 7 : 6; }
+inline int swap_stages(int G, bool ordered = false) { return swap_smem_bytes(7, G, ordered) <= S_MAX_SMEM ? 7 : 6; }
 // Walking the segments in expert order costs four more bytes of shared memory per segment; it is done when that
 // does not cost the ring its seventh stage.
 inline bool swap_can_order(int G) { return swap_stages(G, true) == swap_stages(G, false); }
-constexpr int DUAL_STAGES = 4;                                 // 4 x 48 KB: fits with the largest segment table
-static_assert(swap_smem_bytes(DUAL_STAGES, kMaxG, true, true) <= S_MAX_SMEM, "dual ring does not fit");
-static_assert(swap_smem_bytes(6, kMaxG, false, true) <= S_MAX_SMEM, "six stages do not fit with the largest segment table");
+static_assert(swap_smem_bytes(6, kMaxG, true) <= S_MAX_SMEM, "six stages do not fit with the largest segment table");
 constexpr int TOKEN_TILE = 256;                                // tokens per full tile (N of the pair's MMA)
 constexpr int TOKEN_STEP = 32;                                 // granularity of N
 // Epilogue warps per TMEM lane quadrant.  The SwiGLU epilogue of GEMM-1 is long (shuffle, exp, reciprocal,
@@ -116,8 +111,8 @@ struct SwapParams {
     const int32_t* seg_offsets;
     const int32_t* slot_expert;
     // Optional: the order in which the segments are walked, [G] slot ids sorted by (expert, slot), unused slots last.
-    // Replica segments of one expert then follow each other in the work-item order, so the second replica finds the
-    // expert's weights still in L2 instead of streaming them from HBM again.  nullptr: slot order.
+    // Replica segments of one expert then follow each other in the work-item order and share every weight block, so
+    // the second replica finds the expert's weights in L2 instead of streaming them from HBM again.  nullptr: slot order.
     const int32_t* slot_order;
     int G;
     int w_blocks;              // weight-row blocks per expert (128 f per pair in GEMM-1, 256 h in GEMM-2)
@@ -141,21 +136,18 @@ struct SwapParams {
     // Optional: every CTA writes a record of kGemmClockWords 64-bit words about itself (see director_gemm_counters):
     // SM cycles and nanoseconds spent in the kernel (clock64 and the global timer read by one thread at both ends:
     // cycles / ns is the SM clock the kernel really ran at, which a host-side sampler with millisecond resolution
-    // cannot see), and where the MMA-issuing thread and one epilogue warp spent their cycles.
+    // cannot see), and where the MMA-issuing thread and one epilogue warp spent their cycles.  nullptr: nothing is read.
     unsigned long long* clock_out;
 };
 
-// A work item: one weight block against one token tile or (DUAL) against two consecutive token tiles of a segment.
 struct SwapTile {
     int prob;      // 0: grouped problem, 1: dense problem
-    int row0;      // first token row of the item
-    int valid;     // tokens of the item that belong to the segment (1..256, DUAL: 1..512)
+    int row0;      // first token row of the tile
+    int valid;     // tokens of the tile that belong to the segment (1..256)
+    int n;         // valid rounded up to a multiple of 32: N of the MMA
     int w_row;     // first weight row of the pair's block (f index for GEMM-1, W_down row for GEMM-2)
     int wb;
 };
-// Token tile j (0 or 1) of an item: tokens that belong to the segment, and N of its MMAs (rounded up to 32).
-__device__ __forceinline__ int sub_valid(const SwapTile& t, int j) { return min(max(t.valid - j * TOKEN_TILE, 0), TOKEN_TILE); }
-__device__ __forceinline__ int round_n(int valid) { return (valid + TOKEN_STEP - 1) / TOKEN_STEP * TOKEN_STEP; }
 
 // Work items in their hand-out order.  Consecutive segments of the walk that hold the same expert (the replicas of
 // an expert, adjacent when the segments are walked in expert order) form a group, and the items of a group are
@@ -165,68 +157,60 @@ __device__ __forceinline__ int round_n(int valid) { return (valid + TOKEN_STEP -
 struct SwapWalker {
     const int32_t* seg_off;     // first row of the i-th segment of the walk
     const int32_t* seg_end;     // one past its last row
-    const int32_t* tt_start;    // prefix of work items (per weight block) per segment
+    const int32_t* tt_start;    // prefix of token tiles per segment
     const int16_t* expert;
-    int w_blocks, w_rows_per_expert, rows_per_block, total, item_rows, G;
+    int w_blocks, w_rows_per_expert, rows_per_block, total, G;
     bool grouped;               // false: every segment is its own group (the walk is in slot order)
     int gs = 0, ge = 0;         // current group: segments [gs, ge) of the walk
     __device__ bool get(int w, SwapTile& t) {
         if (w >= total) return false;
+        int g, nt, local;
         if (!grouped) {
-            // one segment per group: the short form of the code below (the decode of an item is on the scheduler
-            // thread's critical path when items are short, as in the down projection of a decode-sized batch)
-            int g = gs;
+            // one segment per group: the short form of the search below (decoding an item is on the scheduler
+            // thread's critical path when items are short, as in the down projection of a small batch)
+            g = gs;
             while (w >= tt_start[g + 1] * w_blocks) ++g;
             gs = g;
-            const int nt = tt_start[g + 1] - tt_start[g];
-            const int local = w - tt_start[g] * w_blocks;
-            t.prob = 0;
+            nt = tt_start[g + 1] - tt_start[g];
+            local = w - tt_start[g] * w_blocks;
             t.wb = local / nt;
-            const int tt = local - t.wb * nt;
-            t.row0 = seg_off[g] + tt * item_rows;
-            t.valid = min(item_rows, seg_end[g] - t.row0);
-            t.w_row = expert[g] * w_rows_per_expert + t.wb * rows_per_block;
-            return true;
+            local -= t.wb * nt;
+        } else {
+            while (w >= tt_start[ge] * w_blocks) {          // w only grows: groups are entered in order
+                gs = ge;
+                ge = gs + 1;
+                while (ge < G && expert[ge] == expert[gs]) ++ge;
+            }
+            nt = tt_start[ge] - tt_start[gs];               // token tiles of the group
+            local = w - tt_start[gs] * w_blocks;
+            t.wb = local / nt;
+            local -= t.wb * nt;                             // tile inside the group
+            g = gs;
+            while (tt_start[g + 1] - tt_start[gs] <= local) ++g;   // its segment
+            local -= tt_start[g] - tt_start[gs];
         }
-        while (w >= tt_start[ge] * w_blocks) {              // w only grows: groups are entered in order
-            gs = ge;
-            ge = gs + 1;
-            while (ge < G && expert[ge] == expert[gs]) ++ge;
-        }
-        const int nt = tt_start[ge] - tt_start[gs];         // token tiles of the group
-        const int local = w - tt_start[gs] * w_blocks;
         t.prob = 0;
-        t.wb = local / nt;
-        const int tig = local - t.wb * nt;                  // tile inside the group
-        int g = gs;
-        while (tt_start[g + 1] - tt_start[gs] <= tig) ++g;  // its segment
-        const int tt = tig - (tt_start[g] - tt_start[gs]);
-        t.row0 = seg_off[g] + tt * item_rows;
-        t.valid = min(item_rows, seg_end[g] - t.row0);
+        t.row0 = seg_off[g] + local * TOKEN_TILE;
+        t.valid = min(TOKEN_TILE, seg_end[g] - t.row0);
+        t.n = (t.valid + TOKEN_STEP - 1) / TOKEN_STEP * TOKEN_STEP;
         t.w_row = expert[g] * w_rows_per_expert + t.wb * rows_per_block;
         return true;
     }
 };
 
-// DUAL: a work item covers two consecutive token tiles of its segment (the last item of a segment may have one, or a
-// short second one).  Both tiles multiply the SAME weight tile, which is loaded once per k-step and feeds two MMAs
-// into the two accumulator buffers: 48 KB of operands per CTA and k-step for 2 x 256 tokens instead of 2 x 32 KB.
-// The k-step rate of this kernel is set by the L2 -> shared-memory operand stream, not by the tensor pipe, so the
-// item with the higher arithmetic intensity is the faster one wherever the k loop is long enough to pay for the
-// accumulator drain that is no longer hidden behind the next item (both buffers belong to one item).  Every output
-// element is still accumulated in ascending k, so the results do not change by a bit.
-template <int MODE, int EPI_GROUPS, bool GATHER, int S_STAGES, bool DUAL = false>
+// MODE 0: gate/up + SwiGLU (A from the 3-D interleaving map).  MODE 1: down projection (A from a 2-D map).
+// GATHER (GEMM-1 only): the token rows are not read from a permuted copy but gathered straight from the layer
+// input x through row_token - tm_x then describes x with a one-row box and the whole producer warp issues the
+// loads, four rows per lane - so the dispatch step needs no row copies at all.
+template <int MODE, int EPI_GROUPS, bool GATHER, int S_STAGES>
 __global__ void __launch_bounds__(96 + 128 * EPI_GROUPS, 1)
 grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
                          const __grid_constant__ CUtensorMap tm_w2 /* dense problem */,
                          const __grid_constant__ CUtensorMap tm_x2, const SwapParams p) {
-    static_assert(!(GATHER && DUAL), "the gathering producer loads one token tile per item");
-    constexpr int STAGE_BYTES = stage_bytes(DUAL);
-    constexpr int ITEM_ROWS = DUAL ? 2 * TOKEN_TILE : TOKEN_TILE;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
-    uint8_t* gen = smem_raw + (tiles - raw) + S_STAGES * STAGE_BYTES;
+    uint8_t* gen = smem_raw + (tiles - raw) + S_STAGES * S_STAGE_BYTES;
     uint64_t* bars = reinterpret_cast<uint64_t*>(gen);             // full[8] empty[8] tfull[2] tempty[2]
     // sched_full[4] at +160, sched_empty[4] at +192 (sched_empty: the scheduler CTA's are the ones used)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + 224);
@@ -254,10 +238,11 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     const bool leader = rank == 0;
-    long long clk0 = 0;
-    unsigned long long ns0 = 0;
-    long long stat_a = 0, stat_b = 0, stat_c = 0, stat_d = 0;      // per-role cycle counters, see SwapParams::clock_out
-    if (threadIdx.x == 0) { clk0 = clock64(); ns0 = global_ns(); }
+    // optional self-measurement (see SwapParams::clock_out): nothing is read unless a record is asked for
+    const bool stats = p.clock_out != nullptr;
+    uint32_t stat_a = 0, stat_b = 0, stat_c = 0, stat_d = 0;       // 32-bit cycle sums: enough for two seconds
+    unsigned long long* const t_start = reinterpret_cast<unsigned long long*>(gen + 232);   // {clock64, ns} at the start
+    if (stats && threadIdx.x == 0) { t_start[0] = (unsigned long long)clock64(); t_start[1] = global_ns(); }
 
     constexpr int n_threads = 96 + 128 * EPI_GROUPS;               // producer, MMA and scheduler warps + epilogue warps
     if (ordered) {
@@ -284,7 +269,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     {
         auto tiles_of = [&](int g) {
             const int len = s_end[g] - s_seg[g];
-            return (s_exp[g] >= 0 && len > 0) ? (len + ITEM_ROWS - 1) / ITEM_ROWS : 0;
+            return (s_exp[g] >= 0 && len > 0) ? (len + TOKEN_TILE - 1) / TOKEN_TILE : 0;
         };
         const int per = (G + n_threads - 1) / n_threads;
         const int lo = min((int)threadIdx.x * per, G), hi = min(lo + per, G);
@@ -315,7 +300,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     const uint32_t tmem_base = *tmem_slot;
 
     constexpr int ROWS_PER_BLOCK = (MODE == 0) ? 128 : 256;   // weight rows (f or h) per pair block
-    SwapWalker walker{s_seg, s_end, s_tt, s_exp, p.w_blocks, p.w_rows_per_expert, ROWS_PER_BLOCK, s_tt[G] * p.w_blocks, ITEM_ROWS, G, ordered};
+    SwapWalker walker{s_seg, s_end, s_tt, s_exp, p.w_blocks, p.w_rows_per_expert, ROWS_PER_BLOCK, s_tt[G] * p.w_blocks, G, ordered};
     SwapTile t;
 
     // Work items (segment, weight block, token tile) are handed out dynamically, in their natural order, from a
@@ -327,7 +312,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     // path.  Tail tiles are cheaper than full ones, so fixed assignments leave 6-15 % of imbalance between clusters;
     // and since the items are still taken in order, clusters running at the same time keep working on neighbouring
     // items and share their weight tiles in L2.
-    const int dense_tiles = (p.dense_rows + ITEM_ROWS - 1) / ITEM_ROWS;      // work items per weight block
+    const int dense_tiles = (p.dense_rows + TOKEN_TILE - 1) / TOKEN_TILE;
     const int total_items = walker.total + dense_tiles * p.dense_w_blocks;
     constexpr uint32_t SCHED_RANK = 0;                             // CTA of the pair that owns the ring's barriers
     const bool sched_local = rank == SCHED_RANK;
@@ -342,6 +327,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
             const int4 v = sched_item[q];
             tile.row0 = v.x;
             tile.valid = v.y;
+            tile.n = (v.y + TOKEN_STEP - 1) / TOKEN_STEP * TOKEN_STEP;
             tile.w_row = v.z;
             tile.wb = v.w & 0x3FFFFFFF;
             tile.prob = (v.w >> 30) & 1;
@@ -368,11 +354,12 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
             ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
             t.row0 = __shfl_sync(0xFFFFFFFFu, t.row0, 0);
             t.valid = __shfl_sync(0xFFFFFFFFu, t.valid, 0);
+            t.n = __shfl_sync(0xFFFFFFFFu, t.n, 0);
             t.w_row = __shfl_sync(0xFFFFFFFFu, t.w_row, 0);
             t.wb = __shfl_sync(0xFFFFFFFFu, t.wb, 0);
             t.prob = 0;                                                 // a gathering launch has no dense problem
             if (!ok || t.valid == 0) break;
-            const int half = round_n(t.valid) >> 1;                     // token rows this CTA supplies (multiple of 16)
+            const int half = t.n >> 1;                                  // token rows this CTA supplies (multiple of 16)
             const int x_row = t.row0 + (int)rank * half;
             const int w_row = t.w_row + (int)rank * (ROWS_PER_BLOCK / 2);
             const bool active = 4 * lane < half;
@@ -388,7 +375,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 if (!ok) break;
                 const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
-                const uint32_t a_dst = tiles + stage * STAGE_BYTES;
+                const uint32_t a_dst = tiles + stage * S_STAGE_BYTES;
                 if (lane == 0) {
                     mbar_expect_tx_cluster(leader_full, tx);
                     tma_load_3d_pair(a_dst, &tm_w, leader_full, kb * BLOCK_K, 0, w_row);
@@ -411,11 +398,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 release_item(i);
                 if (sched_local) *prod_taken = i + 1;
                 if (t.valid == 0) break;
-                // this CTA's half of each token tile's rows
-                const int x_row = t.row0 + (int)rank * (round_n(sub_valid(t, 0)) >> 1);
-                const bool second = DUAL && t.valid > TOKEN_TILE;
-                const int x_row1 = t.row0 + TOKEN_TILE + (int)rank * (round_n(sub_valid(t, 1)) >> 1);
-                const uint32_t tx = second ? (uint32_t)STAGE_BYTES : (uint32_t)S_STAGE_BYTES;
+                const int x_row = t.row0 + (int)rank * (t.n >> 1);          // this CTA's half of the tile's tokens
                 const int w_row = t.w_row + (int)rank * (ROWS_PER_BLOCK / 2);
                 const CUtensorMap* mw = t.prob ? &tm_w2 : &tm_w;
                 const CUtensorMap* mx = t.prob ? &tm_x2 : &tm_x;
@@ -423,12 +406,11 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 for (int kb = 0; kb < k_steps; ++kb) {
                     if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag))) break;
                     const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
-                    const uint32_t a_dst = tiles + stage * STAGE_BYTES;
-                    mbar_expect_tx_cluster(leader_full, tx);
+                    const uint32_t a_dst = tiles + stage * S_STAGE_BYTES;
+                    mbar_expect_tx_cluster(leader_full, S_STAGE_BYTES);
                     if (MODE == 0) tma_load_3d_pair(a_dst, mw, leader_full, kb * BLOCK_K, 0, w_row);
                     else tma_load_2d_pair(a_dst, mw, leader_full, kb * BLOCK_K, w_row);
                     tma_load_2d_pair(a_dst + A_BYTES, mx, leader_full, kb * BLOCK_K, x_row);
-                    if (second) tma_load_2d_pair(a_dst + A_BYTES + B_HALF_BYTES, mx, leader_full, kb * BLOCK_K, x_row1);
                     if (++stage == S_STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -438,58 +420,34 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            // The two accumulator buffers are handed out to token tiles in turn; `tile_no` counts the tiles so far
-            // (every role counts them the same way), buffer = tile_no & 1, its phase = (tile_no >> 1) & 1.
-            uint32_t tile_no = 0;
             for (int it = 0; ok; ++it) {
                 if (!(ok = take_item(it, t))) break;
                 release_item(it);
                 if (t.valid == 0) break;
-                const int n_sub = (DUAL && t.valid > TOKEN_TILE) ? 2 : 1;
-                uint32_t d_tmem[2], idesc[2];
-                int acc[2];
-                const long long c_item = clock64();
-                for (int j = 0; j < n_sub && ok; ++j) {
-                    acc[j] = (int)((tile_no + j) & 1u);
-                    ok = mbar_wait(tempty_bar(acc[j]), ((((tile_no + j) >> 1) & 1u) ^ 1u), abort_flag);
-                    d_tmem[j] = tmem_base + (uint32_t)(acc[j] * TOKEN_TILE);
-                    idesc[j] = S_IDESC_BASE | ((uint32_t)(round_n(sub_valid(t, j)) >> 3) << 17);
-                }
-                if (!ok) break;
-                tile_no += (uint32_t)n_sub;
+                const int acc = it & 1;
+                const uint32_t c_item = stats ? (uint32_t)clock() : 0u;
+                if (!(ok = mbar_wait(tempty_bar(acc), (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag))) break;
                 tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TOKEN_TILE);
+                const uint32_t idesc = S_IDESC_BASE | ((uint32_t)(t.n >> 3) << 17);
                 const int k_steps = t.prob ? p.dense_k_steps : p.k_steps;
-                const long long c_loop = clock64();
-                stat_a += c_loop - c_item;                  // waited for the accumulator buffer(s)
-                stat_c += k_steps;
+                const uint32_t c_loop = stats ? (uint32_t)clock() : 0u;
+                stat_a += c_loop - c_item;                  // waited for the accumulator buffer
+                stat_c += (uint32_t)k_steps;
                 stat_d += 1;
                 for (int kb = 0; kb < k_steps; ++kb) {
                     if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag))) break;
                     tc_fence_after();
-                    const uint32_t a_src = tiles + stage * STAGE_BYTES;
-                    const uint64_t a_desc = smem_desc(a_src);
-                    const uint64_t b_desc0 = smem_desc(a_src + A_BYTES);
-                    if (DUAL && n_sub == 2) {
-                        // the two tiles' MMAs alternate: back-to-back MMAs into one accumulator leave the tensor pipe
-                        // idle for ~45 cycles each (the next one waits for the previous one's write-back), MMAs into
-                        // the other accumulator fill that gap
-                        const uint64_t b_desc1 = smem_desc(a_src + A_BYTES + B_HALF_BYTES);
+                    const uint32_t a_src = tiles + stage * S_STAGE_BYTES;
+                    const uint64_t a_desc = smem_desc(a_src), b_desc = smem_desc(a_src + A_BYTES);
 #pragma unroll
-                        for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
-                            umma_pair_n(d_tmem[0], a_desc + 2u * k, b_desc0 + 2u * k, idesc[0], (kb | k) != 0 ? 1u : 0u);
-                            umma_pair_n(d_tmem[1], a_desc + 2u * k, b_desc1 + 2u * k, idesc[1], (kb | k) != 0 ? 1u : 0u);
-                        }
-                        if (kb == k_steps - 1) { umma_commit_both(tfull_bar(acc[0])); umma_commit_both(tfull_bar(acc[1])); }
-                    } else {
-#pragma unroll
-                        for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                            umma_pair_n(d_tmem[0], a_desc + 2u * k, b_desc0 + 2u * k, idesc[0], (kb | k) != 0 ? 1u : 0u);
-                        if (kb == k_steps - 1) umma_commit_both(tfull_bar(acc[0]));
-                    }
+                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                        umma_pair_n(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
                     umma_commit_both(empty_bar(stage));
                     if (++stage == S_STAGES) { stage = 0; phase ^= 1u; }
                 }
-                stat_b += clock64() - c_loop;               // operand waits and MMA issue of the item's k loop
+                if (ok) umma_commit_both(tfull_bar(acc));
+                if (stats) stat_b += (uint32_t)clock() - c_loop;   // operand waits and MMA issue of the item's k loop
             }
         }
     } else if (warp == 2) {
@@ -520,8 +478,8 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                     item = make_int4(t.row0, t.valid, t.w_row, t.wb);
                 } else if (w < total_items) {          // dense problem: (weight block, token tile) over one segment
                     const int local = w - walker.total;
-                    const int wb = local / dense_tiles, row0 = (local - wb * dense_tiles) * ITEM_ROWS;
-                    item = make_int4(row0, min(ITEM_ROWS, p.dense_rows - row0), wb * ROWS_PER_BLOCK, wb | (1 << 30));
+                    const int wb = local / dense_tiles, row0 = (local - wb * dense_tiles) * TOKEN_TILE;
+                    item = make_int4(row0, min(TOKEN_TILE, p.dense_rows - row0), wb * ROWS_PER_BLOCK, wb | (1 << 30));
                 }
                 sched_item[q] = item;
                 st_cluster_v4(map_to_cta(smem_u32(&sched_item[q]), 1u - SCHED_RANK), item);
@@ -539,75 +497,70 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
         uint16_t* const out_b = static_cast<uint16_t*>(p.dense_out);
         const int lane_row = quad * 32 + lane;                     // weight row of this thread inside the CTA's 128
         bool ok = true;
-        uint32_t tile_no = 0;                                      // token tiles so far: picks the accumulator buffer
         for (int it = 0; ok; ++it) {
             if (!(ok = take_item(it, t))) break;
             __syncwarp();
             if (lane == 0) release_item(it);
             if (t.valid == 0) break;
+            const int acc = it & 1;
+            const uint32_t c_wait = stats ? (uint32_t)clock() : 0u;
+            if (!(ok = mbar_wait(tfull_bar(acc), ((uint32_t)it >> 1) & 1u, abort_flag))) break;
+            const uint32_t c_drain = stats ? (uint32_t)clock() : 0u;
+            stat_a += c_drain - c_wait;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * TOKEN_TILE);
             uint16_t* const out = t.prob ? out_b : out_a;
             const int out_pitch = t.prob ? p.dense_out_pitch : p.out_pitch;
-            const int n_sub = (DUAL && t.valid > TOKEN_TILE) ? 2 : 1;
-            for (int sub = 0; sub < n_sub && ok; ++sub, ++tile_no) {
-                const int acc = (int)(tile_no & 1u);
-                const int row0 = t.row0 + sub * TOKEN_TILE, valid = sub_valid(t, sub), n = round_n(valid);
-                const long long c_wait = clock64();
-                if (!(ok = mbar_wait(tfull_bar(acc), (tile_no >> 1) & 1u, abort_flag))) break;
-                const long long c_drain = clock64();
-                stat_a += c_drain - c_wait;
-                tc_fence_after();
-                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * TOKEN_TILE);
-                if constexpr (MODE == 0) {
-                    // even lane: one of (gate, up) for feature f, odd lane: the other; column = token.
-                    // The two lanes of a pair split the tokens: the even lane finishes the even tokens, the odd lane
-                    // the odd ones.  One shuffle per token pair hands each lane the partner value it needs, so all
-                    // 32 lanes stay active and no branch separates the shuffles.
-                    const int f = t.wb * 128 + (int)rank * 64 + (lane_row >> 1);
-                    const bool odd = (lane & 1) != 0;
-                    const bool i_am_gate = (!odd) == ((t.prob ? p.dense_gate_first : p.gate_first) != 0);
-                    uint16_t* ocol = out + (size_t)(row0 + (odd ? 1 : 0)) * out_pitch + f;
-                    const size_t two_rows = 2 * (size_t)out_pitch;
+            if constexpr (MODE == 0) {
+                // even lane: one of (gate, up) for feature f, odd lane: the other; column = token.
+                // The two lanes of a pair split the tokens: the even lane finishes the even tokens, the odd lane
+                // the odd ones.  One shuffle per token pair hands each lane the partner value it needs, so all
+                // 32 lanes stay active and no branch separates the shuffles.
+                const int f = t.wb * 128 + (int)rank * 64 + (lane_row >> 1);
+                const bool odd = (lane & 1) != 0;
+                const bool i_am_gate = (!odd) == ((t.prob ? p.dense_gate_first : p.gate_first) != 0);
+                uint16_t* ocol = out + (size_t)(t.row0 + (odd ? 1 : 0)) * out_pitch + f;
+                const size_t two_rows = 2 * (size_t)out_pitch;
 #pragma unroll 1
-                    for (int c = c_first; c < n; c += CSTEP) {
-                        uint32_t v[32];
-                        tmem_ld32(taddr + c, v);
-                        tmem_ld_wait();
-                        uint16_t* ptr = ocol + (size_t)c * out_pitch;       // my token of pair m is row c + 2m (+1 if odd)
-                        const int rem = valid - c - (odd ? 1 : 0);          // store pair m iff 2m < rem
+                for (int c = c_first; c < t.n; c += CSTEP) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + c, v);
+                    tmem_ld_wait();
+                    uint16_t* ptr = ocol + (size_t)c * out_pitch;       // my token of pair m is row c + 2m (+1 if odd)
+                    const int rem = t.valid - c - (odd ? 1 : 0);        // store pair m iff 2m < rem
 #pragma unroll
-                        for (int m = 0; m < 16; ++m) {
-                            const float mine = __uint_as_float(odd ? v[2 * m + 1] : v[2 * m]);   // my value at my token
-                            const float send = __uint_as_float(odd ? v[2 * m] : v[2 * m + 1]);   // my value at the partner's token
-                            const float other = __shfl_xor_sync(0xFFFFFFFFu, send, 1);           // partner's value at my token
-                            const float g = i_am_gate ? mine : other, u = i_am_gate ? other : mine;
-                            const float h = __fdividef(g * u, 1.0f + __expf(-g));
-                            if (2 * m < rem) *ptr = __bfloat16_as_ushort(__float2bfloat16_rn(h));
-                            ptr += two_rows;
-                        }
-                    }
-                } else {
-                    const int h_col = t.wb * 256 + (int)rank * 128 + lane_row;
-                    uint16_t* ocol = out + (size_t)row0 * out_pitch + h_col;
-#pragma unroll 1
-                    for (int c = c_first; c < n; c += CSTEP) {
-                        uint32_t v[32];
-                        tmem_ld32(taddr + c, v);
-                        tmem_ld_wait();
-                        uint16_t* ptr = ocol + (size_t)c * out_pitch;
-                        const int rem = valid - c;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (j < rem) *ptr = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[j])));
-                            ptr += out_pitch;
-                        }
+                    for (int m = 0; m < 16; ++m) {
+                        const float mine = __uint_as_float(odd ? v[2 * m + 1] : v[2 * m]);   // my value at my token
+                        const float send = __uint_as_float(odd ? v[2 * m] : v[2 * m + 1]);   // my value at the partner's token
+                        const float other = __shfl_xor_sync(0xFFFFFFFFu, send, 1);           // partner's value at my token
+                        const float g = i_am_gate ? mine : other, u = i_am_gate ? other : mine;
+                        const float h = __fdividef(g * u, 1.0f + __expf(-g));
+                        if (2 * m < rem) *ptr = __bfloat16_as_ushort(__float2bfloat16_rn(h));
+                        ptr += two_rows;
                     }
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
-                stat_b += clock64() - c_drain;
-                stat_c += 1;
+            } else {
+                const int h_col = t.wb * 256 + (int)rank * 128 + lane_row;
+                uint16_t* ocol = out + (size_t)t.row0 * out_pitch + h_col;
+#pragma unroll 1
+                for (int c = c_first; c < t.n; c += CSTEP) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + c, v);
+                    tmem_ld_wait();
+                    uint16_t* ptr = ocol + (size_t)c * out_pitch;
+                    const int rem = t.valid - c;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        if (j < rem) *ptr = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[j])));
+                        ptr += out_pitch;
+                    }
+                }
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+            if (stats) stat_b += (uint32_t)clock() - c_drain;
+            stat_c += 1;
         }
     }
 
@@ -615,23 +568,24 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     __syncthreads();
     cluster_sync_all();
     if (threadIdx.x == 0 && *abort_flag) director_set_status(p.status, DIRECTOR_ERR_TIMEOUT);
-    unsigned long long* const rec = (p.clock_out != nullptr && blockIdx.x < (unsigned)kGemmClockCtas)
-                                        ? p.clock_out + (size_t)blockIdx.x * kGemmClockWords : nullptr;
-    if (threadIdx.x == 0 && rec != nullptr) {
-        rec[0] = (unsigned long long)(clock64() - clk0);
-        rec[1] = global_ns() - ns0;
-        rec[9] = 0ull;
-    }
-    if (threadIdx.x == 32 && rec != nullptr) {              // the MMA-issuing thread (idle in the peer CTA: zeros)
-        rec[2] = (unsigned long long)stat_a;
-        rec[3] = (unsigned long long)stat_b;
-        rec[4] = (unsigned long long)stat_c;
-        rec[5] = (unsigned long long)stat_d;
-    }
-    if (threadIdx.x == 96 && rec != nullptr) {              // lane 0 of the first epilogue warp
-        rec[6] = (unsigned long long)stat_a;
-        rec[7] = (unsigned long long)stat_b;
-        rec[8] = (unsigned long long)stat_c;
+    if (stats && blockIdx.x < (unsigned)kGemmClockCtas) {
+        unsigned long long* const rec = p.clock_out + (size_t)blockIdx.x * kGemmClockWords;
+        if (threadIdx.x == 0) {
+            rec[0] = (unsigned long long)clock64() - t_start[0];
+            rec[1] = global_ns() - t_start[1];
+            rec[9] = 0ull;
+        }
+        if (threadIdx.x == 32) {                            // the MMA-issuing thread (idle in the peer CTA: zeros)
+            rec[2] = (unsigned long long)stat_a;
+            rec[3] = (unsigned long long)stat_b;
+            rec[4] = (unsigned long long)stat_c;
+            rec[5] = (unsigned long long)stat_d;
+        }
+        if (threadIdx.x == 96) {                            // lane 0 of the first epilogue warp
+            rec[6] = (unsigned long long)stat_a;
+            rec[7] = (unsigned long long)stat_b;
+            rec[8] = (unsigned long long)stat_c;
+        }
     }
     if (warp == 1) {
         tc_fence_after();
@@ -669,13 +623,13 @@ bool map_interleaved(director_ctx* ctx, CUtensorMap* map, const void* first, uin
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int MODE, int EPI_GROUPS, bool GATHER, int STAGES, bool DUAL>
+template <int MODE, int EPI_GROUPS, bool GATHER, int STAGES>
 int launch_swap_n(director_ctx* ctx, const char* name, const CUtensorMap& w, const CUtensorMap& x, const CUtensorMap& w2,
                   const CUtensorMap& x2, const SwapParams& p, cudaStream_t st) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * ctx->pair_clusters));
     cfg.blockDim = dim3(96 + 128 * EPI_GROUPS);
-    cfg.dynamicSmemBytes = (size_t)swap_smem_bytes(STAGES, p.G, DUAL, p.slot_order != nullptr);
+    cfg.dynamicSmemBytes = (size_t)swap_smem_bytes(STAGES, p.G, p.slot_order != nullptr);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -685,31 +639,23 @@ int launch_swap_n(director_ctx* ctx, const char* name, const CUtensorMap& w, con
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     LaunchScope scope(ctx, st, name);
-    return cuda_status(cudaLaunchKernelEx(&cfg, grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, STAGES, DUAL>, w, x, w2, x2, p));
+    return cuda_status(cudaLaunchKernelEx(&cfg, grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, STAGES>, w, x, w2, x2, p));
 }
 
 // w2 / x2: the dense problem's maps (any valid map when the launch has none)
 template <int MODE, int EPI_GROUPS, bool GATHER>
 int launch_swap(director_ctx* ctx, const char* name, const CUtensorMap& w, const CUtensorMap& x, const CUtensorMap& w2,
-                const CUtensorMap& x2, const SwapParams& p, bool dual, cudaStream_t st) {
-    if constexpr (!GATHER) {
-        if (dual) return launch_swap_n<MODE, EPI_GROUPS, false, DUAL_STAGES, true>(ctx, name, w, x, w2, x2, p, st);
-    }
-    return swap_stages(p.G, p.slot_order != nullptr) == 7 ? launch_swap_n<MODE, EPI_GROUPS, GATHER, 7, false>(ctx, name, w, x, w2, x2, p, st)
-                                 : launch_swap_n<MODE, EPI_GROUPS, GATHER, 6, false>(ctx, name, w, x, w2, x2, p, st);
+                const CUtensorMap& x2, const SwapParams& p, cudaStream_t st) {
+    return swap_stages(p.G, p.slot_order != nullptr) == 7 ? launch_swap_n<MODE, EPI_GROUPS, GATHER, 7>(ctx, name, w, x, w2, x2, p, st)
+                                 : launch_swap_n<MODE, EPI_GROUPS, GATHER, 6>(ctx, name, w, x, w2, x2, p, st);
 }
 
 template <int MODE, int EPI_GROUPS, bool GATHER>
 bool swap_opt_in() {
-    bool ok = cudaFuncSetAttribute(grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, 6, false>,
-                                   cudaFuncAttributeMaxDynamicSharedMemorySize, swap_smem_bytes(6, kMaxG, false, true)) == cudaSuccess &&
-              cudaFuncSetAttribute(grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, 7, false>,
-                                   cudaFuncAttributeMaxDynamicSharedMemorySize, S_MAX_SMEM) == cudaSuccess;
-    if constexpr (!GATHER)
-        ok = ok && cudaFuncSetAttribute(grouped_gemm_swap_kernel<MODE, EPI_GROUPS, false, DUAL_STAGES, true>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        swap_smem_bytes(DUAL_STAGES, kMaxG, true, true)) == cudaSuccess;
-    return ok;
+    return cudaFuncSetAttribute(grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, 6>,
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, swap_smem_bytes(6, kMaxG, true)) == cudaSuccess &&
+           cudaFuncSetAttribute(grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, 7>,
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, S_MAX_SMEM) == cudaSuccess;
 }
 
 }  // namespace
@@ -761,17 +707,17 @@ int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int
     const int d_rows = dense ? (int)dense->rows : 0, d_Fw = dense ? dense->Fw : 0;
     // the context's own slot table comes with its expert order (stored behind it); any other table is walked as is
     const int32_t* order = (slot_expert == ctx->d_slot_expert && G == ctx->G && swap_can_order(G)) ? slot_expert + G : nullptr;
+    unsigned long long* const clk = ctx->gemm_stats ? ctx->d_gemm_clock : nullptr;
     SwapParams p1{seg_offsets, slot_expert, order, G, Fw / 128, H / BLOCK_K, Fw, Fw, ia.gate_first ? 1 : 0, hidden, ctx->d_status,
                   counters, gather_rows, d_rows, d_Fw / 128, H / BLOCK_K, d_Fw, id.gate_first ? 1 : 0,
-                  dense ? dense->hidden : nullptr, ctx->d_gemm_clock};
-    const bool dual1 = (ctx->ffn_dual & 1) != 0, dual2 = (ctx->ffn_dual & 2) != 0;
-    int rc = gather_rows ? launch_swap<0, EPI_GROUPS_GEMM1, true>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, d_gu, d_in, p1, false, st)
-                         : launch_swap<0, EPI_GROUPS_GEMM1, false>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, d_gu, d_in, p1, dual1, st);
+                  dense ? dense->hidden : nullptr, clk};
+    int rc = gather_rows ? launch_swap<0, EPI_GROUPS_GEMM1, true>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, d_gu, d_in, p1, st)
+                         : launch_swap<0, EPI_GROUPS_GEMM1, false>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, d_gu, d_in, p1, st);
     if (rc != DIRECTOR_OK) return rc;
     SwapParams p2{seg_offsets, slot_expert, order, G, H / 256, Fw / BLOCK_K, H, H, 1, out, ctx->d_status, counters + 1, nullptr,
                   d_rows, H / 256, d_Fw / BLOCK_K, H, 1, dense ? dense->out : nullptr,
-                  ctx->d_gemm_clock ? ctx->d_gemm_clock + (size_t)kGemmClockWords * kGemmClockCtas : nullptr};
-    return launch_swap<1, EPI_GROUPS_GEMM2, false>(ctx, "grouped_gemm_down_kernel", m_d, m_h, d_d, d_h, p2, dual2, st);
+                  clk ? clk + (size_t)kGemmClockWords * kGemmClockCtas : nullptr};
+    return launch_swap<1, EPI_GROUPS_GEMM2, false>(ctx, "grouped_gemm_down_kernel", m_d, m_h, d_d, d_h, p2, st);
 }
 
 }  // namespace director

@@ -309,7 +309,7 @@ def test_host_buffer_entry_points_match_the_device_path():
         assert np.array_equal(b["load"].numpy(), b["load_ref"])
 
 
-@pytest.mark.parametrize("variant", [0, 1, 2, 3, 4, 5, 6])
+@pytest.mark.parametrize("variant", [0, 1, 2, 6])
 def test_every_ffn_tile_scheme_matches_the_oracle_and_the_others(variant):
     """The three tile schemes of the expert-FFN GEMMs (single CTA, CTA pair, weight-stationary CTA pair)
     accumulate every output in the same order, so they must agree bit for bit, and each must match the oracle."""
