@@ -564,6 +564,12 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
         }
     }
 
+    // A role that gave up (an expired wait) tells the peer CTA of the pair, whose roles poll their own flag inside
+    // their waits: both CTAs then drain within microseconds and meet at the closing cluster barrier, instead of the
+    // peer running out its own two seconds.  (The peer is still resident: it cannot pass that barrier without us.)
+    if (*abort_flag)
+        asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(map_to_cta(smem_u32(const_cast<const int*>(abort_flag)), 1u - rank)),
+                     "r"(1) : "memory");
     tc_fence_before();
     __syncthreads();
     cluster_sync_all();

@@ -383,7 +383,7 @@ def test_routing_and_indices_at_half_a_million_tokens():
     assert np.array_equal(row_token.cpu().numpy(), d_o["row_token"])
 
 
-@pytest.mark.parametrize("T", [200, 1000])      # the single-CTA front end, and the cooperative index kernel
+@pytest.mark.parametrize("T", [3, 200, 1000])   # weight-streaming FFN; the single-CTA front end; the cooperative index kernel
 def test_cuda_graph_replay_reproduces_the_direct_pass(T):
     """Every entry point is capturable: a graph of the whole layer replays to the same bits, also after the
     inputs in the captured buffers have changed."""
@@ -496,7 +496,7 @@ def test_fused_front_end_matches_the_separate_stages_and_the_oracle(seed, T, H, 
     assert np.array_equal(o["inv_row"].cpu().numpy(), d["inv_row"])
 
 
-@pytest.mark.parametrize("seed,T,S", [(71, 900, 1), (72, 64, 0), (73, 2048, 2)])
+@pytest.mark.parametrize("seed,T,S", [(71, 900, 1), (72, 64, 0), (73, 2048, 2), (74, 2, 1)])
 def test_one_call_layer_matches_the_stage_calls(seed, T, S):
     """director_layer_forward: same bits as route / dispatch / expert_ffn / combine / placement_cost in order."""
     import torch
