@@ -663,3 +663,29 @@ def test_decode_batches_stream_the_weights_and_match_the_oracle_and_the_tensor_c
     a, b = orc.bf16_to_f64(g.y), orc.bf16_to_f64(gt.y)
     assert rel_l2(a, b) <= REL_L2_TOL and max_abs(a, b) <= MAX_ABS_TOL
     assert np.array_equal(g.inv_row, gt.inv_row)
+
+
+def test_gemm_self_counters_count_the_work_the_segment_table_implies():
+    """The expert GEMM kernels count their own k-steps, work items and drained tiles: the totals must equal what the
+    segment table implies (token tiles x weight blocks x k-steps), and the measured SM clock must be a plausible one."""
+    shape, logits, x, weights = _custom(121, 3000, 512, 12, 3, 384, 0, 4, 4, 1.1)
+    X = _random_placement(121, 12, 4, 4, 3)
+    case = GpuCase(shape, logits, x, weights)
+    g = case.run(X)
+    lens = np.diff(g.seg_offsets)
+    tiles = int(np.sum(-(-lens[lens > 0] // 256)))
+    H, F = shape.H, shape.F
+    for which, w_blocks, k_steps in ((0, F // 128, H // 64), (1, H // 256, F // 64)):
+        raw = (__import__("ctypes").c_int64 * 12)()
+        assert case.layer.d.lib.director_gemm_counters(case.layer.d._ctx, which, raw) == 0
+        c = list(raw)
+        assert c[5] == tiles * w_blocks, (which, c[5], tiles * w_blocks)            # work items
+        assert c[4] == tiles * w_blocks * k_steps                                    # k-steps issued
+        assert c[8] == 2 * tiles * w_blocks                                          # tiles drained: one epilogue warp per CTA, two CTAs
+        assert c[0] > 0 and c[1] > 0 and c[3] > 0 and c[7] > 0
+        mhz = c[0] / c[1] * 1e3
+        assert 100.0 < mhz < 2500.0, mhz
+    mhz, busy_us = case.layer.d.gemm_sm_mhz(0)
+    assert 100.0 < mhz < 2500.0 and busy_us > 0
+    d = case.layer.d.gemm_counters(1)
+    assert d["cycles_per_k_step"] > 100 and d["items_per_pair"] > 0
