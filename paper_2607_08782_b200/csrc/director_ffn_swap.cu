@@ -19,6 +19,12 @@
 // The accumulator is [weight rows x tokens]; the epilogue writes it transposed (2-byte stores, one
 // token per instruction, 32-64 contiguous bytes per warp) into the row-major [tokens, features] outputs.
 // Barrier protocol, bounded waits and teardown are those of the plain CTA-pair kernel.
+//
+// Roles: warp 0 of both CTAs loads operands (TMA), warp 1 of the leader CTA issues the MMAs, lane 0 of warp 2 of the
+// leader claims work items, the remaining warps drain accumulators.  The producer and the MMA warp run their loops
+// as WHOLE warps in lock step, with one lead lane polling the barriers and issuing: loop state stays warp-uniform,
+// which keeps the issue cost of a k-step well under the 512 cycles a full tile occupies the tensor pipe, so that a
+// ragged tile (fewer tokens, shorter MMAs) really takes less time than a full one.
 #include "director_common.cuh"
 #include "director_umma.cuh"
 
@@ -57,6 +63,61 @@ constexpr int EPI_GROUPS_GEMM1 = 2;
 constexpr int EPI_GROUPS_GEMM2 = 1;
 
 // kind::f16 descriptor for the pair without the N field: D=f32, A=B=bf16, K-major, M=256.
+// One lane of a converged warp (the same lane every time).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xFFFFFFFF;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
+// Bounded barrier wait for a loop that a whole warp runs in lock step.  The spin, the poll of the CTA's abort flag
+// and the time limit sit inside one block of PTX, so the code around the call has no data-dependent branch: loop
+// counters, shared-memory addresses and matrix descriptors stay warp-uniform, and the instructions that want them in
+// uniform registers (tcgen05.mma, tcgen05.commit, the TMA loads) get them without a move per operand.  With one
+// thread running such a loop inside `if (lane == 0)`, issuing a k-step took ~510 cycles whatever the tile's width - as
+// long as the tensor pipe needs for a FULL tile, so that a ragged tile cost as much as a full one.
+// Only the lane with `polls` != 0 waits (31 more lanes polling the same barrier add nothing but power); the others fall
+// through and meet it at the warp's next converging instruction.  `bad` != 0 skips the wait (an earlier wait of this
+// lane expired: the loop runs out without waiting or issuing); returns the new `bad`.  An expiry raises the CTA's
+// abort flag.
+__device__ __forceinline__ uint32_t mbar_wait_conv(uint32_t bar, uint32_t parity, uint32_t abort_addr, uint32_t bad,
+                                                   uint32_t polls) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        ".reg .u64 t0, t1;\n\t"
+        ".reg .u32 ab, n;\n\t"
+        "setp.ne.u32 q, %0, 0;\n\t"
+        "@q bra DONE;\n\t"
+        "setp.eq.u32 q, %5, 0;\n\t"
+        "@q bra DONE;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "@p bra DONE;\n\t"
+        "mov.u64 t0, %globaltimer;\n\t"
+        "mov.u32 n, 0;\n\t"
+        "SPIN:\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "@p bra DONE;\n\t"
+        "add.u32 n, n, 1;\n\t"
+        "and.b32 ab, n, 63;\n\t"
+        "setp.ne.u32 q, ab, 0;\n\t"
+        "@q bra SPIN;\n\t"                       // flag and clock are looked at once in 64 polls
+        "ld.volatile.shared.u32 ab, [%3];\n\t"
+        "setp.ne.u32 q, ab, 0;\n\t"
+        "@q bra FAIL;\n\t"
+        "mov.u64 t1, %globaltimer;\n\t"
+        "sub.u64 t1, t1, t0;\n\t"
+        "setp.lt.u64 q, t1, %4;\n\t"
+        "@q bra SPIN;\n\t"
+        "FAIL:\n\t"
+        "mov.u32 ab, 1;\n\t"
+        "st.volatile.shared.u32 [%3], ab;\n\t"
+        "mov.u32 %0, 1;\n\t"
+        "DONE:\n\t"
+        "}"
+        : "+r"(bad) : "r"(bar), "r"(parity), "r"(abort_addr), "l"(WAIT_LIMIT_NS), "r"(polls) : "memory");
+    return bad;
+}
+
 constexpr uint32_t S_IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 4) << 24);
 
 __device__ __forceinline__ void umma_pair_n(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
@@ -105,7 +166,7 @@ __device__ __forceinline__ bool mbar_wait_acquire_cluster(uint32_t bar, uint32_t
 }
 
 constexpr int SCHED_SLOTS = 4;      // ring through which the scheduler thread hands work items to the other roles
-constexpr int SCHED_AHEAD = 1;      // items the scheduler may claim beyond the one after the producer's current item
+constexpr int CLAIM_LEAD = 32;     // k-steps of claimed work the scheduler keeps ahead of its CTA's producer
 
 struct SwapParams {
     const int32_t* seg_offsets;
@@ -217,7 +278,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + 228);
     int4* sched_item = reinterpret_cast<int4*>(gen + 304);         // [4] decoded work items {row0, valid, w_row, wb}
     int32_t* warp_sum = reinterpret_cast<int32_t*>(gen + 248);     // [11]
-    volatile int* prod_taken = reinterpret_cast<volatile int*>(gen + 292);   // items the scheduler CTA's producer has taken
+    volatile int* prod_k = reinterpret_cast<volatile int*>(gen + 292);       // k-steps the scheduler CTA's producer has issued so far
     const int G = p.G;
     int32_t* s_seg = reinterpret_cast<int32_t*>(gen + S_HEADER_BYTES);
     int32_t* s_tt = s_seg + (G + 1);
@@ -258,7 +319,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     }
     if (threadIdx.x == 0) {
         *abort_flag = 0;
-        *prod_taken = 0;
+        *prod_k = 0;
         for (int s = 0; s < S_STAGES; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8 * EPI_GROUPS); }
         // a slot is free again once every reader has read it: MMA thread, both producers, all epilogue warps
@@ -339,6 +400,19 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
         if (sched_local) mbar_arrive(sched_empty(q));
         else mbar_arrive_cluster(map_to_cta(sched_empty(q), SCHED_RANK));
     };
+    // the same for a warp that runs its loop in lock step: every lane waits for and reads the slot; the outcome and the
+    // item's fields are made warp-uniform (one lane releases the slot afterwards)
+    auto take_item_warp = [&](int i, SwapTile& tile) -> bool {
+        const bool ok = __all_sync(0xFFFFFFFFu, take_item(i, tile));
+        tile.row0 = __shfl_sync(0xFFFFFFFFu, tile.row0, 0);
+        tile.valid = __shfl_sync(0xFFFFFFFFu, tile.valid, 0);
+        tile.n = __shfl_sync(0xFFFFFFFFu, tile.n, 0);
+        tile.w_row = __shfl_sync(0xFFFFFFFFu, tile.w_row, 0);
+        tile.wb = __shfl_sync(0xFFFFFFFFu, tile.wb, 0);
+        tile.prob = __shfl_sync(0xFFFFFFFFu, tile.prob, 0);
+        return ok;
+    };
+    const uint32_t abort_addr = smem_u32(const_cast<const int*>(abort_flag));
 
     if (warp == 0 && GATHER) {
         // whole warp: lane 0 loads the weight tile, every lane gathers four token rows per k-step
@@ -349,7 +423,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
             if (lane == 0) {
                 ok = take_item(i, t) ? 1 : 0;
                 if (ok) release_item(i);
-                if (ok && sched_local) *prod_taken = i + 1;
+                if (ok && sched_local) *prod_k = (i + 1) * p.k_steps;   // counted when the item is taken
             }
             ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
             t.row0 = __shfl_sync(0xFFFFFFFFu, t.row0, 0);
@@ -389,44 +463,50 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
             }
         }
     } else if (warp == 0) {
-        if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            bool ok = true;
-            for (int i = 0; ok; ++i) {
-                if (!(ok = take_item(i, t))) break;
-                release_item(i);
-                if (sched_local) *prod_taken = i + 1;
-                if (t.valid == 0) break;
-                const int x_row = t.row0 + (int)rank * (t.n >> 1);          // this CTA's half of the tile's tokens
-                const int w_row = t.w_row + (int)rank * (ROWS_PER_BLOCK / 2);
-                const CUtensorMap* mw = t.prob ? &tm_w2 : &tm_w;
-                const CUtensorMap* mx = t.prob ? &tm_x2 : &tm_x;
-                const int k_steps = t.prob ? p.dense_k_steps : p.k_steps;
-                for (int kb = 0; kb < k_steps; ++kb) {
-                    if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag))) break;
-                    const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
-                    const uint32_t a_dst = tiles + stage * S_STAGE_BYTES;
+        // Operand producer, both CTAs: the whole warp walks the items and the ring in lock step (warp-uniform loop
+        // state, see mbar_wait_conv); one elected lane arms the leader's barrier and issues the two loads of a k-step.
+        const uint32_t lead_lane = elect_one() ? 1u : 0u;          // polls the barriers and issues the loads
+        int stage = 0, issued_k = 0;
+        uint32_t phase = 0, bad = 0;
+        for (int i = 0;; ++i) {
+            if (!take_item_warp(i, t)) break;
+            if (lane == 0) release_item(i);
+            if (t.valid == 0) break;
+            const int x_row = t.row0 + (int)rank * (t.n >> 1);          // this CTA's half of the tile's tokens
+            const int w_row = t.w_row + (int)rank * (ROWS_PER_BLOCK / 2);
+            const CUtensorMap* mw = t.prob ? &tm_w2 : &tm_w;
+            const CUtensorMap* mx = t.prob ? &tm_x2 : &tm_x;
+            const int k_steps = t.prob ? p.dense_k_steps : p.k_steps;
+            for (int kb = 0; kb < k_steps; ++kb) {
+                const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
+                const uint32_t a_dst = tiles + stage * S_STAGE_BYTES;
+                bad = mbar_wait_conv(empty_bar(stage), phase ^ 1u, abort_addr, bad, lead_lane);
+                ++issued_k;
+                if (lead_lane && !bad) {
                     mbar_expect_tx_cluster(leader_full, S_STAGE_BYTES);
                     if (MODE == 0) tma_load_3d_pair(a_dst, mw, leader_full, kb * BLOCK_K, 0, w_row);
                     else tma_load_2d_pair(a_dst, mw, leader_full, kb * BLOCK_K, w_row);
                     tma_load_2d_pair(a_dst + A_BYTES, mx, leader_full, kb * BLOCK_K, x_row);
-                    if (++stage == S_STAGES) { stage = 0; phase ^= 1u; }
+                    if (sched_local) *prod_k = issued_k;                 // the scheduler claims work against this count
                 }
+                if (++stage == S_STAGES) { stage = 0; phase ^= 1u; }
             }
+            if (__any_sync(0xFFFFFFFFu, bad != 0u)) break;
         }
     } else if (warp == 1) {
-        if (lane == 0 && leader) {
+        // MMA issuer, leader CTA: the whole warp runs the loops in lock step, one elected lane issues the four
+        // MMAs of a k-step and the commit that frees the stage.
+        if (leader) {
+            const uint32_t lead_lane = elect_one() ? 1u : 0u;      // polls the barriers, issues the MMAs and commits
             int stage = 0;
-            uint32_t phase = 0;
-            bool ok = true;
-            for (int it = 0; ok; ++it) {
-                if (!(ok = take_item(it, t))) break;
-                release_item(it);
+            uint32_t phase = 0, bad = 0;
+            for (int it = 0;; ++it) {
+                if (!take_item_warp(it, t)) break;
+                if (lane == 0) release_item(it);
                 if (t.valid == 0) break;
                 const int acc = it & 1;
                 const uint32_t c_item = stats ? (uint32_t)clock() : 0u;
-                if (!(ok = mbar_wait(tempty_bar(acc), (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag))) break;
+                bad = mbar_wait_conv(tempty_bar(acc), (((uint32_t)it >> 1) & 1u) ^ 1u, abort_addr, bad, lead_lane);
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TOKEN_TILE);
                 const uint32_t idesc = S_IDESC_BASE | ((uint32_t)(t.n >> 3) << 17);
@@ -436,17 +516,20 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 stat_c += (uint32_t)k_steps;
                 stat_d += 1;
                 for (int kb = 0; kb < k_steps; ++kb) {
-                    if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag))) break;
-                    tc_fence_after();
                     const uint32_t a_src = tiles + stage * S_STAGE_BYTES;
                     const uint64_t a_desc = smem_desc(a_src), b_desc = smem_desc(a_src + A_BYTES);
+                    bad = mbar_wait_conv(full_bar(stage), phase, abort_addr, bad, lead_lane);
+                    tc_fence_after();
+                    if (lead_lane && !bad) {
 #pragma unroll
-                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                        umma_pair_n(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                    umma_commit_both(empty_bar(stage));
+                        for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                            umma_pair_n(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        umma_commit_both(empty_bar(stage));
+                    }
                     if (++stage == S_STAGES) { stage = 0; phase ^= 1u; }
                 }
-                if (ok) umma_commit_both(tfull_bar(acc));
+                if (__any_sync(0xFFFFFFFFu, bad != 0u)) break;
+                if (lead_lane) umma_commit_both(tfull_bar(acc));
                 if (stats) stat_b += (uint32_t)clock() - c_loop;   // operand waits and MMA issue of the item's k loop
             }
         }
@@ -455,15 +538,18 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
             // scheduler: claim the next item, wait until every reader is done with the slot's previous item, write
             // the item into both CTAs' rings, signal both.  The item past the end is published once: it ends every
             // role's loop.
+            int pub_k = 0;                                         // k-steps of the items published so far
             for (int i = 0;; ++i) {
-                // stay SCHED_AHEAD items ahead of this CTA's producer, no more: items held back by a cluster that is
-                // not ready for them are imbalance at the end of the kernel
-                if (i > *prod_taken + SCHED_AHEAD) {
+                // Claimed work stays CLAIM_LEAD k-steps ahead of this CTA's producer, no more: the claim itself takes a few
+                // k-steps' time, and an item claimed by a cluster that is not ready for it is imbalance at the end of the
+                // kernel (with few, long items per cluster - eight of 224 k-steps each in a Mixtral-shaped down
+                // projection - one item claimed too early by the cluster that finishes last costs a whole item's time).
+                if (pub_k - *prod_k >= CLAIM_LEAD) {
                     const unsigned long long t0 = global_ns();
                     uint32_t n = 0;
                     bool give_up = false;
-                    while (i > *prod_taken + SCHED_AHEAD) {
-                        __nanosleep(256);            // an item lasts microseconds: poll gently, this SM has an epilogue to run
+                    while (pub_k - *prod_k >= CLAIM_LEAD) {
+                        __nanosleep(256);            // a k-step lasts a third of a microsecond: poll gently, this SM has an epilogue to run
                         if ((++n & 63u) == 0u && (*abort_flag || global_ns() - t0 > WAIT_LIMIT_NS)) { give_up = true; break; }
                     }
                     if (give_up) { *abort_flag = 1; break; }
@@ -476,10 +562,12 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 if (w < walker.total) {
                     walker.get(w, t);
                     item = make_int4(t.row0, t.valid, t.w_row, t.wb);
+                    pub_k += p.k_steps;
                 } else if (w < total_items) {          // dense problem: (weight block, token tile) over one segment
                     const int local = w - walker.total;
                     const int wb = local / dense_tiles, row0 = (local - wb * dense_tiles) * TOKEN_TILE;
                     item = make_int4(row0, min(TOKEN_TILE, p.dense_rows - row0), wb * ROWS_PER_BLOCK, wb | (1 << 30));
+                    pub_k += p.dense_k_steps;
                 }
                 sched_item[q] = item;
                 st_cluster_v4(map_to_cta(smem_u32(&sched_item[q]), 1u - SCHED_RANK), item);
