@@ -31,7 +31,7 @@ int ffn_swap_init(director_ctx* ctx);   // director_ffn_swap.cu
 int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int32_t* gather_rows, uint64_t rows,
                   const int32_t* seg_offsets, const int32_t* slot_expert, int G, const void* w_gate, const void* w_up,
                   const void* w_down, uint64_t n_experts, int Fw, void* hidden, void* out, unsigned int* counters,
-                  const DenseFfn* dense, cudaStream_t st);
+                  const DenseFfn* dense, uint64_t max_seg_rows, cudaStream_t st);
 int ffn_small_init(director_ctx* ctx);  // director_ffn_small.cu
 bool ffn_small_applies(const director_ctx* ctx, int T, int Fw);
 int ffn_pass_small(director_ctx* ctx, const void* in, const int32_t* seg_offsets, const int32_t* slot_expert, int G,
@@ -281,13 +281,14 @@ int launch_gemm(director_ctx* ctx, const char* name, const CUtensorMap& a, const
 }
 
 // One SwiGLU FFN pass over a segment table: in [rows, H] -> hidden [rows, Fw] -> out [rows, H].
+// max_seg_rows: an upper bound on any segment's length (a token goes to an expert at most once, so the batch size).
 int ffn_pass(director_ctx* ctx, const void* in, uint64_t in_rows, const int32_t* gather_rows, uint64_t rows,
              const int32_t* seg_offsets, const int32_t* slot_expert, int G, const void* w_gate, const void* w_up,
              const void* w_down, uint64_t n_experts, int Fw, void* hidden, void* out, unsigned int* counters,
-             cudaStream_t st) {
+             uint64_t max_seg_rows, cudaStream_t st) {
     if (ctx->ffn_variant == 2) {
         const int rc = ffn_pass_swap(ctx, in, in_rows, gather_rows, rows, seg_offsets, slot_expert, G, w_gate, w_up, w_down,
-                                     n_experts, Fw, hidden, out, counters, nullptr, st);
+                                     n_experts, Fw, hidden, out, counters, nullptr, max_seg_rows, st);
         if (rc != DIRECTOR_ERR_UNSUPPORTED) return rc;   // weight arrays not expressible as one map: tile scheme 0
     }
     if (gather_rows != nullptr) return DIRECTOR_ERR_UNSUPPORTED;   // only the weight-stationary scheme gathers
@@ -349,13 +350,13 @@ int launch_expert_ffn(director_ctx* ctx, int T, const void* xp, const int32_t* r
         // routed and shared experts in the same two launches: the shared experts' work items follow the routed ones
         const DenseFfn dense{x, (uint64_t)T, ws_gate, ws_up, ws_down, s.S * s.F, ctx->d_hidden_shared, y_shared};
         const int rc = ffn_pass_swap(ctx, xp, A, nullptr, A, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up, w_down,
-                                     s.E, s.F, ctx->d_hidden, yp, ctx->d_sched, &dense, st);
+                                     s.E, s.F, ctx->d_hidden, yp, ctx->d_sched, &dense, (uint64_t)T, st);
         if (rc != DIRECTOR_ERR_UNSUPPORTED) return rc;    // a weight pair not expressible as one map: separate passes
     }
     int rc = row_token ? ffn_pass(ctx, x, (uint64_t)T, row_token, A, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up,
-                                  w_down, s.E, s.F, ctx->d_hidden, yp, ctx->d_sched, st)
+                                  w_down, s.E, s.F, ctx->d_hidden, yp, ctx->d_sched, (uint64_t)T, st)
                        : ffn_pass(ctx, xp, A, nullptr, A, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up, w_down,
-                                  s.E, s.F, ctx->d_hidden, yp, ctx->d_sched, st);
+                                  s.E, s.F, ctx->d_hidden, yp, ctx->d_sched, (uint64_t)T, st);
     if (rc != DIRECTOR_OK || !shared) return rc;
     {
         LaunchScope scope(ctx, st, "one_segment_kernel");
@@ -364,7 +365,7 @@ int launch_expert_ffn(director_ctx* ctx, int T, const void* xp, const int32_t* r
     }
     // The S shared experts as one FFN of width S*F over all T rows of x (a single segment, "expert" 0).
     return ffn_pass(ctx, x, (uint64_t)T, nullptr, (uint64_t)T, ctx->d_one_seg, ctx->d_zero_expert, 1, ws_gate, ws_up,
-                    ws_down, 1, s.S * s.F, ctx->d_hidden_shared, y_shared, ctx->d_sched + 2, st);
+                    ws_down, 1, s.S * s.F, ctx->d_hidden_shared, y_shared, ctx->d_sched + 2, (uint64_t)T, st);
 }
 
 }  // namespace director

@@ -36,15 +36,23 @@ using namespace umma;
 
 namespace {
 
-constexpr int S_STAGE_BYTES = A_BYTES + B_HALF_BYTES;          // 16 KB weights + 16 KB tokens per CTA per k-step
-constexpr int S_HEADER_BYTES = 384;                            // barriers, scheduler ring, TMEM slot, scratch
+constexpr int S_HEADER_BYTES = 384;                            // barriers, scheduler ring, TMEM slot, scratch (ring of <= 8 stages)
 constexpr int S_MAX_SMEM = 232448;                             // opt-in shared memory per CTA on sm_100
+// Two shapes of the operand ring.  The ordinary one: stages of 16 KB weights + 16 KB tokens (128 token rows per CTA,
+// tiles of up to 256 tokens), six or seven of them.  The small-batch one (more than eight stages): the token box
+// shrinks to 32 rows per CTA (tiles of up to 64 tokens), a stage to 20 KB, and ten stages fit - with a batch of at
+// most 64 tokens no segment is longer than that, the weights are streamed from HBM once, and what the launch needs
+// is weight bytes in flight, not token rows it does not have.
+constexpr int S_SMALL_STAGES = 10;
+constexpr int swap_tok_rows(int stages) { return stages > 8 ? 32 : 128; }          // token rows per CTA in a stage
+constexpr int swap_stage_bytes(int stages) { return A_BYTES + swap_tok_rows(stages) * 128; }
+constexpr int swap_bar_slots(int stages) { return stages > 8 ? 16 : 8; }           // capacity of the full / empty barrier arrays
+constexpr int swap_header_bytes(int stages) { return S_HEADER_BYTES + (swap_bar_slots(stages) - 8) * 16; }
 // Shared memory of a launch: alignment slack, the operand ring, the header, and the segment tables of its G slots
-// (seg_offsets and token-tile prefix as int32, expert ids as int16).
 // (segment starts, work-item prefix as int32, expert ids as int16; segment ends as int32 when the segments are
 // walked in expert order rather than slot order).
 constexpr int swap_smem_bytes(int stages, int G, bool ordered = false) {
-    return 1024 + stages * S_STAGE_BYTES + S_HEADER_BYTES + (G + 1) * (ordered ? 14 : 10) + 6;
+    return 1024 + stages * swap_stage_bytes(stages) + swap_header_bytes(stages) + (G + 1) * (ordered ? 14 : 10) + 6;
 }
 // The operand stream is latency-bound (a stage comes back ~2.5 us after it is released), so the ring is as deep as
 // shared memory allows: seven stages when the segment tables are small enough, else six.
@@ -53,7 +61,8 @@ inline int swap_stages(int G, bool ordered = false) { return swap_smem_bytes(7, 
 // does not cost the ring its seventh stage.
 inline bool swap_can_order(int G) { return swap_stages(G, true) == swap_stages(G, false); }
 static_assert(swap_smem_bytes(6, kMaxG, true) <= S_MAX_SMEM, "six stages do not fit with the largest segment table");
-constexpr int TOKEN_TILE = 256;                                // tokens per full tile (N of the pair's MMA)
+static_assert(swap_smem_bytes(S_SMALL_STAGES, kMaxG, true) <= S_MAX_SMEM, "the small-batch ring does not fit with the largest segment table");
+constexpr int TOKEN_TILE = 256;                                // tokens per full tile (N of the pair's MMA); accumulator buffers are this many TMEM columns apart
 constexpr int TOKEN_STEP = 32;                                 // granularity of N
 // Epilogue warps per TMEM lane quadrant.  The SwiGLU epilogue of GEMM-1 is long (shuffle, exp, reciprocal,
 // convert and a 2-byte store per element) and a lone warp per scheduler cannot hide its own latencies, so it
@@ -221,6 +230,7 @@ struct SwapWalker {
     const int32_t* tt_start;    // prefix of token tiles per segment
     const int16_t* expert;
     int w_blocks, w_rows_per_expert, rows_per_block, total, G;
+    int tile_rows;              // tokens per full tile
     bool grouped;               // false: every segment is its own group (the walk is in slot order)
     int gs = 0, ge = 0;         // current group: segments [gs, ge) of the walk
     __device__ bool get(int w, SwapTile& t) {
@@ -251,8 +261,8 @@ struct SwapWalker {
             local -= tt_start[g] - tt_start[gs];
         }
         t.prob = 0;
-        t.row0 = seg_off[g] + local * TOKEN_TILE;
-        t.valid = min(TOKEN_TILE, seg_end[g] - t.row0);
+        t.row0 = seg_off[g] + local * tile_rows;
+        t.valid = min(tile_rows, seg_end[g] - t.row0);
         t.n = (t.valid + TOKEN_STEP - 1) / TOKEN_STEP * TOKEN_STEP;
         t.w_row = expert[g] * w_rows_per_expert + t.wb * rows_per_block;
         return true;
@@ -271,30 +281,35 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
-    uint8_t* gen = smem_raw + (tiles - raw) + S_STAGES * S_STAGE_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(gen);             // full[8] empty[8] tfull[2] tempty[2]
+    constexpr int STAGE_BYTES = swap_stage_bytes(S_STAGES);        // weights + this CTA's token rows of one k-step
+    constexpr int TILE_ROWS = 2 * swap_tok_rows(S_STAGES);         // tokens per full tile
+    constexpr int BAR_SLOTS = swap_bar_slots(S_STAGES);
+    constexpr int HEADER_BYTES = swap_header_bytes(S_STAGES);
+    constexpr int HX = (BAR_SLOTS - 8) * 16;                       // what the larger barrier arrays shift the rest of the header by
+    uint8_t* gen = smem_raw + (tiles - raw) + S_STAGES * STAGE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(gen);             // full[BAR_SLOTS] empty[BAR_SLOTS] tfull[2] tempty[2]
     // sched_full[4] at +160, sched_empty[4] at +192 (sched_empty: the scheduler CTA's are the ones used)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + 224);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + 228);
-    int4* sched_item = reinterpret_cast<int4*>(gen + 304);         // [4] decoded work items {row0, valid, w_row, wb}
-    int32_t* warp_sum = reinterpret_cast<int32_t*>(gen + 248);     // [11]
-    volatile int* prod_k = reinterpret_cast<volatile int*>(gen + 292);       // k-steps the scheduler CTA's producer has issued so far
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + HX + 224);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + HX + 228);
+    int4* sched_item = reinterpret_cast<int4*>(gen + HX + 304);    // [4] decoded work items {row0, valid, w_row, wb}
+    int32_t* warp_sum = reinterpret_cast<int32_t*>(gen + HX + 248);     // [11]
+    volatile int* prod_k = reinterpret_cast<volatile int*>(gen + HX + 292);  // k-steps the scheduler CTA's producer has issued so far
     const int G = p.G;
-    int32_t* s_seg = reinterpret_cast<int32_t*>(gen + S_HEADER_BYTES);
+    int32_t* s_seg = reinterpret_cast<int32_t*>(gen + HEADER_BYTES);
     int32_t* s_tt = s_seg + (G + 1);
     int16_t* s_exp = reinterpret_cast<int16_t*>(s_tt + (G + 1));
     // in slot order a segment ends where the next one starts; in expert order the ends are a table of their own
     const bool ordered = p.slot_order != nullptr;
-    int32_t* s_hi = reinterpret_cast<int32_t*>(gen + S_HEADER_BYTES + (((G + 1) * 10 + 3) & ~3));   // 4-byte aligned, behind s_exp
+    int32_t* s_hi = reinterpret_cast<int32_t*>(gen + HEADER_BYTES + (((G + 1) * 10 + 3) & ~3));   // 4-byte aligned, behind s_exp
     const int32_t* s_end = ordered ? s_hi : s_seg + 1;
 
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
-    auto empty_bar = [&](int s) { return bar0 + 64u + 8u * s; };
-    auto tfull_bar = [&](int a) { return bar0 + 128u + 8u * a; };
-    auto tempty_bar = [&](int a) { return bar0 + 144u + 8u * a; };
-    auto sched_full = [&](int q) { return bar0 + 160u + 8u * q; };
-    auto sched_empty = [&](int q) { return bar0 + 192u + 8u * q; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * BAR_SLOTS + 8u * s; };
+    auto tfull_bar = [&](int a) { return bar0 + HX + 128u + 8u * a; };
+    auto tempty_bar = [&](int a) { return bar0 + HX + 144u + 8u * a; };
+    auto sched_full = [&](int q) { return bar0 + HX + 160u + 8u * q; };
+    auto sched_empty = [&](int q) { return bar0 + HX + 192u + 8u * q; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
@@ -302,7 +317,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     // optional self-measurement (see SwapParams::clock_out): nothing is read unless a record is asked for
     const bool stats = p.clock_out != nullptr;
     uint32_t stat_a = 0, stat_b = 0, stat_c = 0, stat_d = 0;       // 32-bit cycle sums: enough for two seconds
-    unsigned long long* const t_start = reinterpret_cast<unsigned long long*>(gen + 232);   // {clock64, ns} at the start
+    unsigned long long* const t_start = reinterpret_cast<unsigned long long*>(gen + HX + 232);   // {clock64, ns} at the start
     if (stats && threadIdx.x == 0) { t_start[0] = (unsigned long long)clock64(); t_start[1] = global_ns(); }
 
     constexpr int n_threads = 96 + 128 * EPI_GROUPS;               // producer, MMA and scheduler warps + epilogue warps
@@ -330,7 +345,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     {
         auto tiles_of = [&](int g) {
             const int len = s_end[g] - s_seg[g];
-            return (s_exp[g] >= 0 && len > 0) ? (len + TOKEN_TILE - 1) / TOKEN_TILE : 0;
+            return (s_exp[g] >= 0 && len > 0) ? (len + TILE_ROWS - 1) / TILE_ROWS : 0;
         };
         const int per = (G + n_threads - 1) / n_threads;
         const int lo = min((int)threadIdx.x * per, G), hi = min(lo + per, G);
@@ -361,7 +376,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     const uint32_t tmem_base = *tmem_slot;
 
     constexpr int ROWS_PER_BLOCK = (MODE == 0) ? 128 : 256;   // weight rows (f or h) per pair block
-    SwapWalker walker{s_seg, s_end, s_tt, s_exp, p.w_blocks, p.w_rows_per_expert, ROWS_PER_BLOCK, s_tt[G] * p.w_blocks, G, ordered};
+    SwapWalker walker{s_seg, s_end, s_tt, s_exp, p.w_blocks, p.w_rows_per_expert, ROWS_PER_BLOCK, s_tt[G] * p.w_blocks, G, TILE_ROWS, ordered};
     SwapTile t;
 
     // Work items (segment, weight block, token tile) are handed out dynamically, in their natural order, from a
@@ -373,7 +388,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     // path.  Tail tiles are cheaper than full ones, so fixed assignments leave 6-15 % of imbalance between clusters;
     // and since the items are still taken in order, clusters running at the same time keep working on neighbouring
     // items and share their weight tiles in L2.
-    const int dense_tiles = (p.dense_rows + TOKEN_TILE - 1) / TOKEN_TILE;
+    const int dense_tiles = (p.dense_rows + TILE_ROWS - 1) / TILE_ROWS;
     const int total_items = walker.total + dense_tiles * p.dense_w_blocks;
     constexpr uint32_t SCHED_RANK = 0;                             // CTA of the pair that owns the ring's barriers
     const bool sched_local = rank == SCHED_RANK;
@@ -449,7 +464,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 if (!ok) break;
                 const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
-                const uint32_t a_dst = tiles + stage * S_STAGE_BYTES;
+                const uint32_t a_dst = tiles + stage * STAGE_BYTES;
                 if (lane == 0) {
                     mbar_expect_tx_cluster(leader_full, tx);
                     tma_load_3d_pair(a_dst, &tm_w, leader_full, kb * BLOCK_K, 0, w_row);
@@ -479,11 +494,11 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
             const int k_steps = t.prob ? p.dense_k_steps : p.k_steps;
             for (int kb = 0; kb < k_steps; ++kb) {
                 const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
-                const uint32_t a_dst = tiles + stage * S_STAGE_BYTES;
+                const uint32_t a_dst = tiles + stage * STAGE_BYTES;
                 bad = mbar_wait_conv(empty_bar(stage), phase ^ 1u, abort_addr, bad, lead_lane);
                 ++issued_k;
                 if (lead_lane && !bad) {
-                    mbar_expect_tx_cluster(leader_full, S_STAGE_BYTES);
+                    mbar_expect_tx_cluster(leader_full, STAGE_BYTES);
                     if (MODE == 0) tma_load_3d_pair(a_dst, mw, leader_full, kb * BLOCK_K, 0, w_row);
                     else tma_load_2d_pair(a_dst, mw, leader_full, kb * BLOCK_K, w_row);
                     tma_load_2d_pair(a_dst + A_BYTES, mx, leader_full, kb * BLOCK_K, x_row);
@@ -516,7 +531,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 stat_c += (uint32_t)k_steps;
                 stat_d += 1;
                 for (int kb = 0; kb < k_steps; ++kb) {
-                    const uint32_t a_src = tiles + stage * S_STAGE_BYTES;
+                    const uint32_t a_src = tiles + stage * STAGE_BYTES;
                     const uint64_t a_desc = smem_desc(a_src), b_desc = smem_desc(a_src + A_BYTES);
                     bad = mbar_wait_conv(full_bar(stage), phase, abort_addr, bad, lead_lane);
                     tc_fence_after();
@@ -565,8 +580,8 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                     pub_k += p.k_steps;
                 } else if (w < total_items) {          // dense problem: (weight block, token tile) over one segment
                     const int local = w - walker.total;
-                    const int wb = local / dense_tiles, row0 = (local - wb * dense_tiles) * TOKEN_TILE;
-                    item = make_int4(row0, min(TOKEN_TILE, p.dense_rows - row0), wb * ROWS_PER_BLOCK, wb | (1 << 30));
+                    const int wb = local / dense_tiles, row0 = (local - wb * dense_tiles) * TILE_ROWS;
+                    item = make_int4(row0, min(TILE_ROWS, p.dense_rows - row0), wb * ROWS_PER_BLOCK, wb | (1 << 30));
                     pub_k += p.dense_k_steps;
                 }
                 sched_item[q] = item;
@@ -739,13 +754,22 @@ int launch_swap_n(director_ctx* ctx, const char* name, const CUtensorMap& w, con
 // w2 / x2: the dense problem's maps (any valid map when the launch has none)
 template <int MODE, int EPI_GROUPS, bool GATHER>
 int launch_swap(director_ctx* ctx, const char* name, const CUtensorMap& w, const CUtensorMap& x, const CUtensorMap& w2,
-                const CUtensorMap& x2, const SwapParams& p, cudaStream_t st) {
+                const CUtensorMap& x2, const SwapParams& p, bool small, cudaStream_t st) {
+    if constexpr (!GATHER) {
+        if (small) return launch_swap_n<MODE, EPI_GROUPS, GATHER, S_SMALL_STAGES>(ctx, name, w, x, w2, x2, p, st);
+    }
     return swap_stages(p.G, p.slot_order != nullptr) == 7 ? launch_swap_n<MODE, EPI_GROUPS, GATHER, 7>(ctx, name, w, x, w2, x2, p, st)
                                  : launch_swap_n<MODE, EPI_GROUPS, GATHER, 6>(ctx, name, w, x, w2, x2, p, st);
 }
 
 template <int MODE, int EPI_GROUPS, bool GATHER>
 bool swap_opt_in() {
+    if constexpr (!GATHER) {
+        if (cudaFuncSetAttribute(grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, S_SMALL_STAGES>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 swap_smem_bytes(S_SMALL_STAGES, kMaxG, true)) != cudaSuccess)
+            return false;
+    }
     return cudaFuncSetAttribute(grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, 6>,
                                 cudaFuncAttributeMaxDynamicSharedMemorySize, swap_smem_bytes(6, kMaxG, true)) == cudaSuccess &&
            cudaFuncSetAttribute(grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, 7>,
@@ -766,12 +790,20 @@ int ffn_swap_init(director_ctx*) {
 // is in[gather_rows[i]].
 // dense (optional, not with gather_rows): a second FFN over ONE segment of dense->rows rows of dense->in with a single
 // weight set - the shared experts - whose work items ride in the same two launches.
+// max_seg_rows: an upper bound on the length of any segment of the table (`rows` if nothing better is known); with a
+// bound of at most 64 the launches use the small-batch ring (see S_SMALL_STAGES) - correct for any table, since that
+// ring also tiles the tokens by 64.
 // Returns DIRECTOR_ERR_UNSUPPORTED if a pair of weight arrays cannot be described by one interleaving map.
 int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int32_t* gather_rows, uint64_t rows,
                   const int32_t* seg_offsets, const int32_t* slot_expert, int G, const void* w_gate, const void* w_up,
                   const void* w_down, uint64_t n_experts, int Fw, void* hidden, void* out,
-                  unsigned int* counters /* 2 zeroed work-item counters */, const DenseFfn* dense, cudaStream_t st) {
+                  unsigned int* counters /* 2 zeroed work-item counters */, const DenseFfn* dense, uint64_t max_seg_rows,
+                  cudaStream_t st) {
     const int H = ctx->shape.H;
+    // small-batch ring (tiles of 64 tokens, ten stages): when no segment, routed or dense, can be longer than a tile
+    const bool small = !gather_rows && max_seg_rows <= 2u * swap_tok_rows(S_SMALL_STAGES) &&
+                       (!dense || dense->rows <= 2u * swap_tok_rows(S_SMALL_STAGES));
+    const uint32_t tok_box = small ? swap_tok_rows(S_SMALL_STAGES) : 128;
     struct Interleave { bool ok; bool gate_first; const void* first; uint64_t delta; };
     auto interleave = [](const void* g, const void* u) {
         const uintptr_t pg = reinterpret_cast<uintptr_t>(g), pu = reinterpret_cast<uintptr_t>(u);
@@ -783,7 +815,7 @@ int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int
     if (!ia.ok) return DIRECTOR_ERR_UNSUPPORTED;
     if (dense && gather_rows) return DIRECTOR_ERR_INVALID_ARG;
     CUtensorMap m_in, m_gu, m_h, m_d;
-    if (!map_2d(ctx, &m_in, in, in_rows, H, gather_rows ? 1 : 128) || !map_2d(ctx, &m_h, hidden, rows, Fw) ||
+    if (!map_2d(ctx, &m_in, in, in_rows, H, gather_rows ? 1 : tok_box) || !map_2d(ctx, &m_h, hidden, rows, Fw, tok_box) ||
         !map_2d(ctx, &m_d, w_down, n_experts * H, Fw))
         return DIRECTOR_ERR_CUDA;
     if (!map_interleaved(ctx, &m_gu, ia.first, ia.delta, n_experts * Fw, H)) return DIRECTOR_ERR_UNSUPPORTED;
@@ -793,7 +825,8 @@ int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int
     if (dense) {
         id = interleave(dense->w_gate, dense->w_up);
         if (!id.ok) return DIRECTOR_ERR_UNSUPPORTED;
-        if (!map_2d(ctx, &d_in, dense->in, dense->rows, H) || !map_2d(ctx, &d_h, dense->hidden, dense->rows, dense->Fw) ||
+        if (!map_2d(ctx, &d_in, dense->in, dense->rows, H, tok_box) ||
+            !map_2d(ctx, &d_h, dense->hidden, dense->rows, dense->Fw, tok_box) ||
             !map_2d(ctx, &d_d, dense->w_down, H, dense->Fw))
             return DIRECTOR_ERR_CUDA;
         if (!map_interleaved(ctx, &d_gu, id.first, id.delta, dense->Fw, H)) return DIRECTOR_ERR_UNSUPPORTED;
@@ -805,13 +838,13 @@ int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int
     SwapParams p1{seg_offsets, slot_expert, order, G, Fw / 128, H / BLOCK_K, Fw, Fw, ia.gate_first ? 1 : 0, hidden, ctx->d_status,
                   counters, gather_rows, d_rows, d_Fw / 128, H / BLOCK_K, d_Fw, id.gate_first ? 1 : 0,
                   dense ? dense->hidden : nullptr, clk};
-    int rc = gather_rows ? launch_swap<0, EPI_GROUPS_GEMM1, true>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, d_gu, d_in, p1, st)
-                         : launch_swap<0, EPI_GROUPS_GEMM1, false>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, d_gu, d_in, p1, st);
+    int rc = gather_rows ? launch_swap<0, EPI_GROUPS_GEMM1, true>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, d_gu, d_in, p1, false, st)
+                         : launch_swap<0, EPI_GROUPS_GEMM1, false>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, d_gu, d_in, p1, small, st);
     if (rc != DIRECTOR_OK) return rc;
     SwapParams p2{seg_offsets, slot_expert, order, G, H / 256, Fw / BLOCK_K, H, H, 1, out, ctx->d_status, counters + 1, nullptr,
                   d_rows, H / 256, d_Fw / BLOCK_K, H, 1, dense ? dense->out : nullptr,
                   clk ? clk + (size_t)kGemmClockWords * kGemmClockCtas : nullptr};
-    return launch_swap<1, EPI_GROUPS_GEMM2, false>(ctx, "grouped_gemm_down_kernel", m_d, m_h, d_d, d_h, p2, st);
+    return launch_swap<1, EPI_GROUPS_GEMM2, false>(ctx, "grouped_gemm_down_kernel", m_d, m_h, d_d, d_h, p2, small, st);
 }
 
 }  // namespace director

@@ -689,3 +689,37 @@ def test_gemm_self_counters_count_the_work_the_segment_table_implies():
     assert 100.0 < mhz < 2500.0 and busy_us > 0
     d = case.layer.d.gemm_counters(1)
     assert d["cycles_per_k_step"] > 100 and d["items_per_pair"] > 0
+
+
+@pytest.mark.parametrize("seed,H,E,K,F,S,R,C,extra", [
+    (131, 512, 12, 3, 384, 1, 4, 4, 3),
+    (132, 2048, 128, 8, 768, 0, 16, 9, 16),        # Qwen3-shaped routing: most segments hold a handful of rows
+    (133, 256, 2, 2, 256, 0, 2, 1, 0),             # two experts, top-2: both segments are exactly one 64-token tile
+])
+def test_small_batch_ring_gives_the_same_bits_as_the_ordinary_one(seed, H, E, K, F, S, R, C, extra):
+    """Batches of 5..64 tokens run the expert GEMMs with 64-token tiles and a ten-stage operand ring, larger ones with
+    256-token tiles: a token's output does not depend on which (same k order, one accumulator per output element),
+    so the first 64 tokens of a 65-token batch and the same 64 tokens as a batch of their own agree bit for bit."""
+    shape, logits, x, weights = _custom(seed, 65, H, E, K, F, S, R, C)
+    X = _random_placement(seed, E, R, C, extra)
+    case = GpuCase(shape, logits, x, weights)
+    big = case.run(X)                                       # 65 tokens: the ordinary ring
+    small = case.run(X, T=64)                               # 64 tokens: the small-batch ring
+    assert big.status == 0 and small.status == 0
+    assert np.array_equal(small.y, big.y[:64])
+    if small.y_shared is not None:
+        assert np.array_equal(small.y_shared, big.y_shared[:64])
+    lens = np.diff(small.seg_offsets)
+    raw = (__import__("ctypes").c_int64 * 12)()
+    assert case.layer.d.lib.director_gemm_counters(case.layer.d._ctx, 0, raw) == 0
+    tiles64 = int(np.sum(-(-lens[lens > 0] // 64)))                            # 64-token tiles of the routed segments
+    w_routed, w_dense = F // 128, S * F // 128                                 # the shared experts add one dense tile
+    assert raw[5] == tiles64 * w_routed + (w_dense if S > 0 else 0), (raw[5], tiles64)
+    idx, w, w64, d, c = _oracle_front(shape, logits[:64], x[:64], X, C)
+    s64 = synth.Shape(shape.name, 64, H, E, K, F, S, R, C, shape.zipf_s, shape.seed)
+    _check_outputs(s64, small, x[:64], weights, idx, w, w64, d, c, np.arange(64), f"small_ring{seed}")
+    for T in (5, 33):                                       # ragged small batches against the oracle
+        g = case.run(X, T=T)
+        idx, w, w64, d, c = _oracle_front(shape, logits[:T], x[:T], X, C)
+        sT = synth.Shape(shape.name, T, H, E, K, F, S, R, C, shape.zipf_s, shape.seed)
+        _check_outputs(sT, g, x[:T], weights, idx, w, w64, d, c, np.arange(T), f"small_ring{seed}_T{T}")
