@@ -37,6 +37,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32)
 combine_kernel(const uint4* __restrict__ yp, const int32_t* __restrict__ inv_row, const float* __restrict__ topk_w,
                const uint4* __restrict__ y_shared, uint4* __restrict__ y, int T, int K_rt, int row_vec,
                int slices_per_row) {
+    chain_prologue();
     const int K = K_T > 0 ? K_T : K_rt;
     const int lane = threadIdx.x & 31;
     const long long item = (long long)blockIdx.x * kCombineWarps + (threadIdx.x >> 5);
@@ -109,9 +110,9 @@ int launch_combine(director_ctx* ctx, int T, const void* yp, const int32_t* inv_
     const unsigned grid = (unsigned)((items + kCombineWarps - 1) / kCombineWarps);
     LaunchScope scope(ctx, st, "combine_kernel");
 #define COMBINE_LAUNCH(KT)                                                                                      \
-    combine_kernel<KT><<<grid, kCombineWarps * 32, 0, st>>>(static_cast<const uint4*>(yp), inv_row, topk_w,     \
-                                                            static_cast<const uint4*>(y_shared),                \
-                                                            static_cast<uint4*>(y), T, s.K, row_vec, slices)
+    launch_chained(combine_kernel<KT>, dim3(grid), dim3(kCombineWarps * 32), 0, st, static_cast<const uint4*>(yp),  \
+                   inv_row, topk_w, static_cast<const uint4*>(y_shared), static_cast<uint4*>(y), T, (int)s.K, row_vec,  \
+                   slices)
     switch (s.K) {
         case 1: COMBINE_LAUNCH(1); break;
         case 2: COMBINE_LAUNCH(2); break;

@@ -110,6 +110,39 @@ struct director_ctx {
 
 namespace director {
 
+// Programmatic dependent launch.  A kernel launched through launch_chained() may be scheduled onto free SMs while the
+// kernel before it in the stream is still running; chain_prologue(), the first statement of such a kernel, lets the
+// kernel AFTER it do the same and then blocks until the kernel before it has completed and its writes are visible.
+// Nothing of the kernel runs ahead of its predecessor: what overlaps is the launch itself (a few microseconds, which is
+// a good part of what a decode-sized step consists of).  Launched the ordinary way, both instructions do nothing.
+#ifdef __CUDACC__
+__device__ __forceinline__ void chain_prologue() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+// Not while the stream is being captured into a CUDA graph: a replayed graph has no launch latency to hide, and its
+// programmatic edges made the decode-sized steps 3-8 us slower (measured), so captured launches are ordinary ones.
+inline bool chain_allowed(cudaStream_t st) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    return cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone;
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                  Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = chain_allowed(st) ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // Brackets one kernel launch: counts it and, when profiling is on, records events around it.
 struct LaunchScope {
     director_ctx* ctx;

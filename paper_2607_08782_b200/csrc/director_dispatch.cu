@@ -303,6 +303,7 @@ __global__ void __launch_bounds__(kScatterWarps * 32)
 scatter_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ inv_row, uint4* __restrict__ xp,
                     int T, int K, int row_vec /* uint4 per row */, int slices_per_row) {
     const int lane = threadIdx.x & 31;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");     // the kernel after this one may be scheduled
     const long long item = (long long)blockIdx.x * kScatterWarps + (threadIdx.x >> 5);
     if (item >= (long long)T * slices_per_row) return;
     const int t = (int)(item / slices_per_row);

@@ -137,6 +137,7 @@ small_ffn_kernel(const SmallParams p, const int features_per_cta) {
     extern __shared__ __align__(16) uint16_t s_rows[];     // [n][Kdim] bf16: the segment's rows
     __shared__ int s_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    chain_prologue();
 
     // The blockIdx.y-th non-empty segment (slot with an expert and at least one row), found by warp 0: the table is
     // read 256 slots at a time with all loads of a batch in flight together (one round trip to L2 per batch).
@@ -256,8 +257,8 @@ int launch_small(director_ctx* ctx, const char* name, const SmallParams& p, int 
     per_cta = (per_cta + quantum - 1) / quantum * quantum;
     const dim3 grid((unsigned)((p.N + per_cta - 1) / per_cta), (unsigned)max_segments);
     LaunchScope scope(ctx, st, name);
-    small_ffn_kernel<MODE><<<grid, kSmallWarps * 32, small_smem_bytes(rows_max, p.Kdim), st>>>(p, (int)per_cta);
-    return cuda_status(cudaGetLastError());
+    return cuda_status(launch_chained(small_ffn_kernel<MODE>, grid, dim3(kSmallWarps * 32),
+                                      (size_t)small_smem_bytes(rows_max, p.Kdim), st, p, (int)per_cta));
 }
 
 }  // namespace

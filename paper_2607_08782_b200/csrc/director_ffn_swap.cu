@@ -279,6 +279,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                          const __grid_constant__ CUtensorMap tm_w2 /* dense problem */,
                          const __grid_constant__ CUtensorMap tm_x2, const SwapParams p) {
     extern __shared__ uint8_t smem_raw[];
+    chain_prologue();
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     constexpr int STAGE_BYTES = swap_stage_bytes(S_STAGES);        // weights + this CTA's token rows of one k-step
@@ -740,13 +741,15 @@ int launch_swap_n(director_ctx* ctx, const char* name, const CUtensorMap& w, con
     cfg.blockDim = dim3(96 + 128 * EPI_GROUPS);
     cfg.dynamicSmemBytes = (size_t)swap_smem_bytes(STAGES, p.G, p.slot_order != nullptr);
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;    // see chain_prologue()
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = chain_allowed(st) ? 2 : 1;
     LaunchScope scope(ctx, st, name);
     return cuda_status(cudaLaunchKernelEx(&cfg, grouped_gemm_swap_kernel<MODE, EPI_GROUPS, GATHER, STAGES>, w, x, w2, x2, p));
 }

@@ -301,6 +301,7 @@ front_small_kernel(const float* __restrict__ logits, int T, int E, int K, int R,
     __shared__ int32_t s_rep_start[kMaxE + 1];        // the placement tables, fetched while the gate runs
     __shared__ int16_t s_rep_slot[kMaxG];
     const int tid = threadIdx.x;
+    chain_prologue();
     for (int i = tid; i <= E; i += kFrontThreads) s_rep_start[i] = __ldg(rep_start + i);
     for (int i = tid; i < n_replicas; i += kFrontThreads) s_rep_slot[i] = (int16_t)__ldg(rep_slot + i);
 
@@ -408,8 +409,8 @@ int launch_front_small(director_ctx* ctx, int T, const float* logits, int32_t* t
     const director_shape& s = ctx->shape;
     LaunchScope scope(ctx, st, "front_small_kernel");
 #define FRONT_LAUNCH(VEC, K8)                                                                                          \
-    front_small_kernel<VEC, K8><<<1, kFrontThreads, 0, st>>>(                                                          \
-        logits, T, s.E, s.K, s.R, s.C_max, ctx->G, ctx->n_replicas, ctx->d_rep_start, ctx->d_rep_slot, topk_idx, topk_w, \
+    launch_chained(front_small_kernel<VEC, K8>, dim3(1), dim3(kFrontThreads), 0, st,                                    \
+        logits, T, (int)s.E, (int)s.K, (int)s.R, (int)s.C_max, ctx->G, ctx->n_replicas, ctx->d_rep_start, ctx->d_rep_slot, topk_idx, topk_w, \
         row_token,                                                                                                     \
         inv_row, dest_rank, seg_offsets, ctx->d_seg_offsets, reinterpret_cast<unsigned long long*>(workload),          \
         reinterpret_cast<unsigned long long*>(rank_load), reinterpret_cast<unsigned long long*>(dispatch_tokens),      \
