@@ -174,7 +174,9 @@ int director_expert_ffn(director_ctx* ctx, int32_t T, const void* xp, const int3
  * DIRECTOR_ERR_UNSUPPORTED.
  * Cost: the weight-stationary GEMM reads each token tile once per 256-row weight block, so the gather is repeated
  * 2F/256 times per token row and runs as one-row TMA boxes; it saves memory (no xp), not time - the layer's
- * default path materialises xp once. */
+ * default path materialises xp once.  The exception is a batch small enough for the weight-streaming kernels
+ * (director_batch_streams_weights): those stage a segment's few rows in shared memory once per CTA, from xp or
+ * from x alike, so there the gathering form is the cheaper one (no row copies) and the one-call entry points use it. */
 int director_expert_ffn_gather(director_ctx* ctx, int32_t T, const void* x, const int32_t* row_token,
                                const int32_t* seg_offsets, const void* w_gate, const void* w_up,
                                const void* w_down, void* yp, const void* ws_gate, const void* ws_up,
@@ -313,6 +315,13 @@ int director_selftest_bounded_wait(director_ctx* ctx, uint64_t limit_ns, uint64_
  * Scheme 2 falls back to scheme 0 when w_gate and w_up cannot be described by one strided tensor map
  * (their addresses differ by 2^40 bytes or more). */
 int director_set_ffn_variant(director_ctx* ctx, int32_t variant);
+
+/* 1 if a batch of T tokens takes the weight-streaming FFN kernels under the current tile scheme (T <= 4, scheme 2, and
+ * the rows of a segment fit in shared memory), 0 if it takes the tensor-core kernels, -DIRECTOR_ERR_INVALID_ARG for a
+ * NULL context or T outside [1, T_max].  A caller that drives the stages itself can then skip the row copies: xp = NULL in
+ * director_dispatch / director_route_dispatch_cost, followed by director_expert_ffn_gather.  No paper counterpart
+ * (an implementation detail of Section II-A's expert FFNs at decode-sized batches). */
+int director_batch_streams_weights(director_ctx* ctx, int32_t T);
 
 /* SM clock the expert GEMMs really ran at.  Every CTA of a grouped-GEMM launch reads the SM cycle counter and
  * the global nanosecond timer when it starts and when it ends; this call synchronises the device and returns

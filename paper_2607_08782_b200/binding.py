@@ -23,7 +23,7 @@ EXPORTED = (
     "director_expert_ffn", "director_combine", "director_placement_cost", "director_layer_forward_host",
     "director_last_status", "director_launch_count", "director_set_profiling", "director_kernel_time",
     "director_status_string", "director_dispatch_index_static", "director_layer_submit_host",
-    "director_layer_wait_host", "director_set_ffn_variant", "director_placement_cost_batch",
+    "director_layer_wait_host", "director_set_ffn_variant", "director_batch_streams_weights", "director_placement_cost_batch",
     "director_expert_ffn_gather", "director_set_replica_policy", "director_dispatch_src",
     "director_dedup_dispatch_tokens", "director_route_dispatch_cost", "director_layer_forward",
     "director_reserve_placements", "director_select_placement", "director_set_profiling_filter",
@@ -76,6 +76,7 @@ def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.director_set_profiling.argtypes = [vp, c_int32]
     lib.director_set_profiling_filter.argtypes = [vp, c_char_p]
     lib.director_set_ffn_variant.argtypes = [vp, c_int32]
+    lib.director_batch_streams_weights.argtypes = [vp, c_int32]
     lib.director_set_replica_policy.argtypes = [vp, c_int32]
     lib.director_reserve_placements.argtypes = [vp, c_int32]
     lib.director_select_placement.argtypes = [vp, c_int32]
@@ -253,6 +254,13 @@ class Director:
 
     def set_ffn_variant(self, variant: int):
         _check(self.lib.director_set_ffn_variant(self._ctx, variant), "director_set_ffn_variant")
+
+    def batch_streams_weights(self, T: int) -> bool:
+        """True if a batch of T tokens takes the weight-streaming FFN kernels (which need no permuted copy of x)."""
+        rc = int(self.lib.director_batch_streams_weights(self._ctx, T))
+        if rc < 0:
+            raise DirectorError(-rc, "director_batch_streams_weights")
+        return rc == 1
 
     def gemm_sm_mhz(self, which: int = 0):
         """(SM MHz, longest CTA's microseconds) of the most recent gate|up (0) or down (1) GEMM launch, measured

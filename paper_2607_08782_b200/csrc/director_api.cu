@@ -499,13 +499,15 @@ int director_layer_submit_host(director_ctx* ctx, int32_t T, const float* logits
         return DIRECTOR_ERR_CUDA;
     // the permuted rows are materialised once: the weight-stationary GEMM reads every token tile once per weight
     // block, so gathering inside it (director_expert_ffn_gather) repeats the gather 2F/256 times and measured slower
-    int rc = launch_front(ctx, T, d_logits, d_x, ctx->e_topk_idx, ctx->e_topk_w, ctx->e_xp,
+    // (the weight-streaming kernels of a tiny batch stage their few rows from x themselves: no row copies then)
+    const bool stream_w = ffn_streams_weights(ctx, T);
+    int rc = launch_front(ctx, T, d_logits, d_x, ctx->e_topk_idx, ctx->e_topk_w, stream_w ? nullptr : ctx->e_xp,
                           ctx->e_row_token, ctx->e_inv_row, ctx->e_dest_rank, ctx->d_seg_offsets, c_w, c_load, c_tok,
                           c_bytes, st);
     if (rc == DIRECTOR_OK)
-        rc = launch_expert_ffn(ctx, T, ctx->e_xp, nullptr, ctx->d_seg_offsets, w_gate, w_up,
-                               w_down, ctx->e_yp, shared ? d_x : nullptr, ws_gate, ws_up, ws_down,
-                               shared ? ctx->e_y_shared : nullptr, st);
+        rc = launch_expert_ffn(ctx, T, stream_w ? nullptr : ctx->e_xp, stream_w ? ctx->e_row_token : nullptr,
+                               ctx->d_seg_offsets, w_gate, w_up, w_down, ctx->e_yp, (shared || stream_w) ? d_x : nullptr,
+                               ws_gate, ws_up, ws_down, shared ? ctx->e_y_shared : nullptr, st);
     if (rc == DIRECTOR_OK)
         rc = launch_combine(ctx, T, ctx->e_yp, ctx->e_inv_row, ctx->e_topk_w, shared ? ctx->e_y_shared : nullptr, d_y, st);
     if (rc != DIRECTOR_OK) return rc;
@@ -561,12 +563,15 @@ int director_layer_forward(director_ctx* ctx, int32_t T, const float* logits, co
          reinterpret_cast<uintptr_t>(dispatch_tokens) | reinterpret_cast<uintptr_t>(dispatch_bytes)) & 7u)
         return DIRECTOR_ERR_INVALID_ARG;
     cudaStream_t st = as_stream(stream);
-    int rc = launch_front(ctx, T, logits, x, ctx->e_topk_idx, ctx->e_topk_w, ctx->e_xp, ctx->e_row_token,
-                          ctx->e_inv_row, ctx->e_dest_rank, ctx->d_seg_offsets, workload, rank_load, dispatch_tokens,
-                          dispatch_bytes, st);
+    // the weight-streaming kernels of a tiny batch stage their few rows from x themselves: no row copies then
+    const bool stream_w = ffn_streams_weights(ctx, T);
+    int rc = launch_front(ctx, T, logits, x, ctx->e_topk_idx, ctx->e_topk_w, stream_w ? nullptr : ctx->e_xp,
+                          ctx->e_row_token, ctx->e_inv_row, ctx->e_dest_rank, ctx->d_seg_offsets, workload, rank_load,
+                          dispatch_tokens, dispatch_bytes, st);
     if (rc == DIRECTOR_OK)
-        rc = launch_expert_ffn(ctx, T, ctx->e_xp, nullptr, ctx->d_seg_offsets, w_gate, w_up, w_down, ctx->e_yp,
-                               shared ? x : nullptr, ws_gate, ws_up, ws_down, shared ? ctx->e_y_shared : nullptr, st);
+        rc = launch_expert_ffn(ctx, T, stream_w ? nullptr : ctx->e_xp, stream_w ? ctx->e_row_token : nullptr,
+                               ctx->d_seg_offsets, w_gate, w_up, w_down, ctx->e_yp, (shared || stream_w) ? x : nullptr,
+                               ws_gate, ws_up, ws_down, shared ? ctx->e_y_shared : nullptr, st);
     if (rc == DIRECTOR_OK)
         rc = launch_combine(ctx, T, ctx->e_yp, ctx->e_inv_row, ctx->e_topk_w, shared ? ctx->e_y_shared : nullptr, y, st);
     return rc;
@@ -590,6 +595,11 @@ int director_last_status(director_ctx* ctx, void* stream) {
     if (cudaMemsetAsync(ctx->d_status, 0, sizeof(h), st) != cudaSuccess) return DIRECTOR_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return DIRECTOR_ERR_CUDA;
     return h;
+}
+
+int director_batch_streams_weights(director_ctx* ctx, int32_t T) {
+    if (ctx == nullptr || T < 1 || T > ctx->shape.T_max) return -DIRECTOR_ERR_INVALID_ARG;   // 1 is an answer here
+    return ffn_streams_weights(ctx, T) ? 1 : 0;
 }
 
 int director_set_ffn_variant(director_ctx* ctx, int32_t variant) {

@@ -244,6 +244,7 @@ struct DenseFfn {
 int launch_expert_ffn(director_ctx*, int T, const void* xp, const int32_t* row_token, const int32_t* seg_offsets,
                       const void* w_gate, const void* w_up, const void* w_down, void* yp, const void* x,
                       const void* ws_gate, const void* ws_up, const void* ws_down, void* y_shared, cudaStream_t);
+bool ffn_streams_weights(const director_ctx*, int T);   // batch small enough for the weight-streaming FFN kernels
 int launch_combine(director_ctx*, int T, const void* yp, const int32_t* inv_row, const float* topk_w,
                    const void* y_shared, void* y, cudaStream_t);
 

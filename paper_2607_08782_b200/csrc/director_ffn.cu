@@ -34,7 +34,7 @@ int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int
                   const DenseFfn* dense, uint64_t max_seg_rows, cudaStream_t st);
 int ffn_small_init(director_ctx* ctx);  // director_ffn_small.cu
 bool ffn_small_applies(const director_ctx* ctx, int T, int Fw);
-int ffn_pass_small(director_ctx* ctx, const void* in, const int32_t* seg_offsets, const int32_t* slot_expert, int G,
+int ffn_pass_small(director_ctx* ctx, const void* in, const int32_t* gather_rows, const int32_t* seg_offsets, const int32_t* slot_expert, int G,
                    const void* w_gate, const void* w_up, const void* w_down, int Fw, void* hidden, void* out, int rows_max,
                    int max_segments, cudaStream_t st);
 int ffn_pair_init(director_ctx* ctx);   // director_ffn_pair.cu
@@ -321,6 +321,14 @@ int ffn_init(director_ctx* ctx) {
     return DIRECTOR_OK;
 }
 
+// True if a batch of T tokens takes the weight-streaming FFN kernels (tile scheme 2 only): the one-call entry points
+// then skip the row copies of the dispatch step, since those kernels stage their rows from x themselves.
+bool ffn_streams_weights(const director_ctx* ctx, int T) {
+    const director_shape& s = ctx->shape;
+    return ctx->ffn_variant == 2 && ctx->ffn_small && ffn_small_applies(ctx, T, s.F) &&
+           (s.S == 0 || ffn_small_applies(ctx, T, s.S * s.F));
+}
+
 // row_token == nullptr: the routed experts read the permuted rows xp.  Otherwise they gather row i as
 // x[row_token[i]] and xp is not used.
 int launch_expert_ffn(director_ctx* ctx, int T, const void* xp, const int32_t* row_token, const int32_t* seg_offsets,
@@ -330,18 +338,19 @@ int launch_expert_ffn(director_ctx* ctx, int T, const void* xp, const int32_t* r
     const director_shape& s = ctx->shape;
     const uint64_t A = (uint64_t)T * s.K;
     const bool shared = s.S > 0 && x != nullptr && y_shared != nullptr;
-    if (ctx->ffn_variant == 2 && ctx->ffn_small && row_token == nullptr && ffn_small_applies(ctx, T, s.F) &&
-        (!shared || ffn_small_applies(ctx, T, s.S * s.F))) {
+    if (ffn_streams_weights(ctx, T)) {
         // decode-sized batch: every segment has at most T rows; stream the touched weights once, feature by feature
-        int rc = ffn_pass_small(ctx, xp, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up, w_down, s.F, ctx->d_hidden,
-                                yp, T, (int)std::min<uint64_t>((uint64_t)ctx->G, A), st);
+        // (with row_token the rows are staged straight from x: x must then be given even without shared experts)
+        if (row_token != nullptr && x == nullptr) return DIRECTOR_ERR_INVALID_ARG;
+        int rc = ffn_pass_small(ctx, row_token ? x : xp, row_token, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up, w_down,
+                                s.F, ctx->d_hidden, yp, T, (int)std::min<uint64_t>((uint64_t)ctx->G, A), st);
         if (rc != DIRECTOR_OK || !shared) return rc;
         {
             LaunchScope scope(ctx, st, "one_segment_kernel");
             one_segment_kernel<<<1, 1, 0, st>>>(ctx->d_one_seg, T);
             if ((rc = cuda_status(cudaGetLastError())) != DIRECTOR_OK) return rc;
         }
-        return ffn_pass_small(ctx, x, ctx->d_one_seg, ctx->d_zero_expert, 1, ws_gate, ws_up, ws_down, s.S * s.F,
+        return ffn_pass_small(ctx, x, nullptr, ctx->d_one_seg, ctx->d_zero_expert, 1, ws_gate, ws_up, ws_down, s.S * s.F,
                               ctx->d_hidden_shared, y_shared, T, 1, st);
     }
     // work-item counters of the (up to four) GEMM launches below

@@ -36,6 +36,7 @@ struct SmallParams {
     const int32_t* slot_expert;   // [G]
     int G;
     const uint16_t* in;           // bf16 [rows, Kdim]
+    const int32_t* gather_rows;   // nullptr, or: row i of the segment table is in[gather_rows[i]] (the un-permuted input)
     const uint16_t* w0;           // MODE 0: gate [E, N, Kdim]; MODE 1: down [E, N, Kdim]
     const uint16_t* w1;           // MODE 0: up   [E, N, Kdim]
     int N;                        // output features per row: F (MODE 0), H (MODE 1)
@@ -181,8 +182,9 @@ small_ffn_kernel(const SmallParams p, const int features_per_cta) {
 
     for (int i = threadIdx.x; i < n * vecs; i += blockDim.x) {
         const int r = i / vecs, c = i - r * vecs;
+        const int src = p.gather_rows ? __ldg(p.gather_rows + row0 + r) : row0 + r;
         *reinterpret_cast<uint4*>(s_rows + (size_t)r * p.Kdim + 8 * c) =
-            __ldg(reinterpret_cast<const uint4*>(p.in + (size_t)(row0 + r) * p.Kdim) + c);
+            __ldg(reinterpret_cast<const uint4*>(p.in + (size_t)src * p.Kdim) + c);
     }
     __syncthreads();
 
@@ -278,15 +280,17 @@ bool ffn_small_applies(const director_ctx* ctx, int T, int Fw) {
 
 // in [rows, H] -> hidden [rows, Fw] -> out [rows, H] over a segment table whose segments hold at most kSmallFfnTokens
 // rows (a batch of at most that many tokens).  max_segments: upper bound of the non-empty segments.
-int ffn_pass_small(director_ctx* ctx, const void* in, const int32_t* seg_offsets, const int32_t* slot_expert, int G,
+// gather_rows != nullptr: `in` is the un-permuted layer input and row i of the segment table is in[gather_rows[i]]
+// (the rows are staged in shared memory once per CTA either way, so the dispatch step needs no row copies).
+int ffn_pass_small(director_ctx* ctx, const void* in, const int32_t* gather_rows, const int32_t* seg_offsets, const int32_t* slot_expert, int G,
                    const void* w_gate, const void* w_up, const void* w_down, int Fw, void* hidden, void* out, int rows_max,
                    int max_segments, cudaStream_t st) {
     const int H = ctx->shape.H;
-    const SmallParams p1{seg_offsets, slot_expert, G, static_cast<const uint16_t*>(in), static_cast<const uint16_t*>(w_gate),
+    const SmallParams p1{seg_offsets, slot_expert, G, static_cast<const uint16_t*>(in), gather_rows, static_cast<const uint16_t*>(w_gate),
                          static_cast<const uint16_t*>(w_up), Fw, H, static_cast<uint16_t*>(hidden), ctx->d_status};
     int rc = launch_small<0>(ctx, "small_ffn_swiglu_kernel", p1, rows_max, max_segments, st);
     if (rc != DIRECTOR_OK) return rc;
-    const SmallParams p2{seg_offsets, slot_expert, G, static_cast<const uint16_t*>(hidden), static_cast<const uint16_t*>(w_down),
+    const SmallParams p2{seg_offsets, slot_expert, G, static_cast<const uint16_t*>(hidden), nullptr, static_cast<const uint16_t*>(w_down),
                          nullptr, H, Fw, static_cast<uint16_t*>(out), ctx->d_status};
     return launch_small<1>(ctx, "small_ffn_down_kernel", p2, rows_max, max_segments, st);
 }

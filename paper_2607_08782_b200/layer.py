@@ -102,7 +102,9 @@ class MoELayer:
         fused: dispatch produces indices only and the expert GEMM gathers its rows from x.  Off by default: the
         weight-stationary GEMM re-reads a token tile once per weight block, so the gather is repeated 2F/256 times
         and costs more than the single row copy it saves."""
-        gather = fused and self.ffn_variant == 2
+        # a batch small enough for the weight-streaming FFN kernels needs no permuted copy either: they stage a
+        # segment's few rows from x themselves
+        gather = (fused and self.ffn_variant == 2) or self.d.batch_streams_weights(T)
         if with_cost:          # front end in one call (a single launch for decode-sized batches)
             self.d.route_dispatch_cost(T, logits, x, self.topk_idx, self.topk_w, None if gather else self.xp,
                                        self.row_token, self.inv_row, self.dest_rank, self.seg_offsets, self.workload,

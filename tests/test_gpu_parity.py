@@ -657,7 +657,22 @@ def test_decode_batches_stream_the_weights_and_match_the_oracle_and_the_tensor_c
     assert case.layer.d.kernel_time("small_ffn")[1] == (4 if S > 0 else 2)        # the streaming kernels ran ...
     assert case.layer.d.kernel_time("grouped_gemm")[1] == 0                       # ... and no tensor-core kernel
     case.layer.d.set_profiling(False)
+    # the whole-layer call skips the row copies for such a batch (the streaming kernels stage their rows from x):
+    # front end, two FFN kernels, combine (+ a helper and two more FFN kernels for shared experts) - and the same bits
+    import torch
+    from paper_2607_08782_b200.layer import tensor_to_bf16_bits
+    L = case.layer
+    assert L.d.batch_streams_weights(T)
+    L.set_placement(X)
+    n1 = L.d.launch_count()
+    y = L.forward(T, case.logits, case.x)
+    torch.cuda.synchronize()
+    assert L.d.last_status() == 0
+    assert L.d.launch_count() - n1 == (7 if S > 0 else 4)
+    assert np.array_equal(tensor_to_bf16_bits(y), g.y)
+    assert np.array_equal(L.workload.cpu().numpy(), g.workload)
     case.layer.d.set_ffn_variant(6)                                               # tensor cores for every batch size
+    assert not L.d.batch_streams_weights(T)
     gt = case.run(X)
     case.layer.d.set_ffn_variant(2)
     a, b = orc.bf16_to_f64(g.y), orc.bf16_to_f64(gt.y)
