@@ -20,6 +20,8 @@
 // winners.  HBM traffic is 4E bytes in and 8K bytes out per token.
 #include "director_common.cuh"
 
+#include <algorithm>
+
 namespace director {
 
 namespace {
@@ -301,20 +303,21 @@ front_small_kernel(const float* __restrict__ logits, int T, int E, int K, int R,
     __shared__ int32_t s_rep_start[kMaxE + 1];        // the placement tables, fetched while the gate runs
     __shared__ int16_t s_rep_slot[kMaxG];
     const int tid = threadIdx.x;
+    const int nthr = blockDim.x;                       // a multiple of 32, at least max(G, T, 4 lanes per token of a pass)
     chain_prologue();
-    for (int i = tid; i <= E; i += kFrontThreads) s_rep_start[i] = __ldg(rep_start + i);
-    for (int i = tid; i < n_replicas; i += kFrontThreads) s_rep_slot[i] = (int16_t)__ldg(rep_slot + i);
+    for (int i = tid; i <= E; i += nthr) s_rep_start[i] = __ldg(rep_start + i);
+    for (int i = tid; i < n_replicas; i += nthr) s_rep_slot[i] = (int16_t)__ldg(rep_slot + i);
 
-    for (int i = tid; i < E * kFrontWarps; i += kFrontThreads) (&mask[0][0])[i] = 0u;
-    for (int i = tid; i <= G; i += kFrontThreads) s_seg[i] = 0;
-    for (int i = tid; i < R * R; i += kFrontThreads) h_rr[i] = 0u;
-    for (int i = tid; i < R; i += kFrontThreads) h_load[i] = 0u;
-    for (int i = tid; i < R * E; i += kFrontThreads) workload[i] = 0ull;
-    for (int i = tid; i < R; i += kFrontThreads) rank_load[i] = 0ull;
-    for (int i = tid; i < R * R; i += kFrontThreads) { dispatch_tokens[i] = 0ull; dispatch_bytes[i] = 0ull; }
+    for (int i = tid; i < E * kFrontWarps; i += nthr) (&mask[0][0])[i] = 0u;
+    for (int i = tid; i <= G; i += nthr) s_seg[i] = 0;
+    for (int i = tid; i < R * R; i += nthr) h_rr[i] = 0u;
+    for (int i = tid; i < R; i += nthr) h_load[i] = 0u;
+    for (int i = tid; i < R * E; i += nthr) workload[i] = 0ull;
+    for (int i = tid; i < R; i += nthr) rank_load[i] = 0ull;
+    for (int i = tid; i < R * R; i += nthr) { dispatch_tokens[i] = 0ull; dispatch_bytes[i] = 0ull; }
 
     // ---- gate (a1) ----
-    for (int t0 = 0; t0 < T; t0 += kFrontThreads / kFrontLpt) {
+    for (int t0 = 0; t0 < T; t0 += nthr / kFrontLpt) {
         const int t_raw = t0 + tid / kFrontLpt, sub = tid % kFrontLpt;
         const bool live = t_raw < T;
         const int t = live ? t_raw : T - 1;
@@ -335,7 +338,7 @@ front_small_kernel(const float* __restrict__ logits, int T, int E, int K, int R,
     if (token_thread)
         for (int s = 0; s < K; ++s) atomicOr(&mask[s_idx[tid][s]][w], 1u << lane);
     __syncthreads();
-    for (int e = tid; e < E; e += kFrontThreads) {
+    for (int e = tid; e < E; e += nthr) {
         int run = 0;
 #pragma unroll
         for (int ww = 0; ww < kFrontWarps; ++ww) { warp_prefix[e][ww] = (uint16_t)run; run += __popc(mask[e][ww]); }
@@ -361,7 +364,7 @@ front_small_kernel(const float* __restrict__ logits, int T, int E, int K, int R,
         if (tid < G) s_seg[tid] = base;
         if (tid == G - 1) s_seg[G] = base + len;
         __syncthreads();
-        for (int g = tid; g <= G; g += kFrontThreads) {
+        for (int g = tid; g <= G; g += nthr) {
             seg_offsets_a[g] = s_seg[g];
             if (seg_offsets_b) seg_offsets_b[g] = s_seg[g];
         }
@@ -387,12 +390,12 @@ front_small_kernel(const float* __restrict__ logits, int T, int E, int K, int R,
         }
     }
     __syncthreads();
-    for (int i = tid; i < R * R; i += kFrontThreads) {
+    for (int i = tid; i < R * R; i += nthr) {
         const unsigned long long c = h_rr[i];
         dispatch_tokens[i] = c;
         dispatch_bytes[i] = c * bytes_per_token;
     }
-    for (int i = tid; i < R; i += kFrontThreads) rank_load[i] = h_load[i];
+    for (int i = tid; i < R; i += nthr) rank_load[i] = h_load[i];
 }
 
 }  // namespace
@@ -408,8 +411,11 @@ int launch_front_small(director_ctx* ctx, int T, const float* logits, int32_t* t
     StageScope stage(ctx, st, "stage_front_small");
     const director_shape& s = ctx->shape;
     LaunchScope scope(ctx, st, "front_small_kernel");
+    // a thread per segment slot (the scan) and per token, four lanes per token in a pass of the gate; no more warps
+    // than that: the kernel is a chain of barriers, and a barrier costs by the warp
+    const int threads = std::min(kFrontThreads, (std::max(std::max(ctx->G, kFrontLpt * T), 128) + 31) / 32 * 32);
 #define FRONT_LAUNCH(VEC, K8)                                                                                          \
-    launch_chained(front_small_kernel<VEC, K8>, dim3(1), dim3(kFrontThreads), 0, st,                                    \
+    launch_chained(front_small_kernel<VEC, K8>, dim3(1), dim3(threads), 0, st,                                          \
         logits, T, (int)s.E, (int)s.K, (int)s.R, (int)s.C_max, ctx->G, ctx->n_replicas, ctx->d_rep_start, ctx->d_rep_slot, topk_idx, topk_w, \
         row_token,                                                                                                     \
         inv_row, dest_rank, seg_offsets, ctx->d_seg_offsets, reinterpret_cast<unsigned long long*>(workload),          \
