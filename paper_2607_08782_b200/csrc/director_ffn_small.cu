@@ -136,14 +136,14 @@ template <int MODE>
 __global__ void __launch_bounds__(kSmallWarps * 32)
 small_ffn_kernel(const SmallParams p, const int features_per_cta) {
     extern __shared__ __align__(16) uint16_t s_rows[];     // [n][Kdim] bf16: the segment's rows
-    __shared__ int s_slot;
+    __shared__ int s_slot, s_lo, s_hi, s_ex;               // the CTA's segment: slot, row range, expert
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     chain_prologue();
 
     // The blockIdx.y-th non-empty segment (slot with an expert and at least one row), found by warp 0: the table is
     // read 256 slots at a time with all loads of a batch in flight together (one round trip to L2 per batch).
     if (warp == 0) {
-        int seen = 0, found = -1;
+        int seen = 0, found = -1, f_lo = 0, f_hi = 0, f_ex = -1;
         for (int b0 = 0; b0 < p.G && found < 0; b0 += 256) {
             int ex[8], lo[8], hi[8];
 #pragma unroll
@@ -161,24 +161,41 @@ small_ffn_kernel(const SmallParams p, const int features_per_cta) {
                 if (found < 0 && seen + here > (int)blockIdx.y) {
                     unsigned mm = m;
                     for (int k = 0; k < (int)blockIdx.y - seen; ++k) mm &= mm - 1;   // drop the lower set bits
-                    found = b0 + 32 * i + __ffs(mm) - 1;
+                    const int src = __ffs(mm) - 1;                  // the lane that holds the segment (warp-uniform)
+                    found = b0 + 32 * i + src;
+                    f_lo = __shfl_sync(0xFFFFFFFFu, lo[i], src);
+                    f_hi = __shfl_sync(0xFFFFFFFFu, hi[i], src);
+                    f_ex = __shfl_sync(0xFFFFFFFFu, ex[i], src);
                 }
                 seen += here;
             }
         }
-        if (lane == 0) s_slot = found;
+        if (lane == 0) { s_slot = found; s_lo = f_lo; s_hi = f_hi; s_ex = f_ex; }
     }
     __syncthreads();
     const int g = s_slot;
     if (g < 0) return;                                      // fewer non-empty segments than grid.y
-    const int row0 = __ldg(p.seg_offsets + g);
-    int n = __ldg(p.seg_offsets + g + 1) - row0;
+    const int row0 = s_lo;
+    int n = s_hi - row0;
     if (n > kRowsMax) {                                     // cannot happen for a batch of at most kRowsMax tokens
         if (threadIdx.x == 0) director_set_status(p.status, DIRECTOR_ERR_BAD_INDEX);
         n = kRowsMax;
     }
-    const int e = __ldg(p.slot_expert + g);
+    const int e = s_ex;
     const int vecs = p.Kdim >> 3;                           // 16-byte vectors per row
+    {
+        // the first weight rows this CTA will stream (one feature per warp, two matrices for MODE 0) are asked into L2
+        // now, so that their first round trip to HBM runs while the segment's rows are being staged below
+        const int f0 = blockIdx.x * features_per_cta;
+        const int n_first = min(kSmallWarps, min((int)(blockIdx.x + 1) * features_per_cta, p.N) - f0);
+        const size_t lines = ((size_t)n_first * p.Kdim * 2 + 127) / 128;            // consecutive rows: one byte range
+        const char* b0 = reinterpret_cast<const char*>(p.w0 + ((size_t)e * p.N + f0) * p.Kdim);
+        const char* b1 = MODE == 0 ? reinterpret_cast<const char*>(p.w1 + ((size_t)e * p.N + f0) * p.Kdim) : nullptr;
+        for (size_t l = threadIdx.x; l < lines; l += blockDim.x) {
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(b0 + 128 * l));
+            if (MODE == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(b1 + 128 * l));
+        }
+    }
 
     for (int i = threadIdx.x; i < n * vecs; i += blockDim.x) {
         const int r = i / vecs, c = i - r * vecs;
