@@ -292,8 +292,9 @@ STAGE_KERNELS = {
     "dispatch": ["dispatch_plan_kernel", "dispatch_count_scan_kernel", "dispatch_index_kernel", "dispatch_scatter_rows_kernel",
                  "dispatch_travel_count_scan_kernel", "dispatch_slot_count_scan_kernel", "dispatch_local_index_kernel"],
     "expert_ffn": ["grouped_gemm_swiglu_kernel", "grouped_gemm_down_kernel", "one_segment_kernel",
-                   "small_ffn_swiglu_kernel", "small_ffn_down_kernel"],
-    "combine": ["combine_kernel"],
+                   "small_ffn_swiglu_kernel", "small_ffn_down_kernel", "grouped_gemm_down_fused_kernel",
+                   "fused_combine_prepare_kernel"],
+    "combine": ["combine_kernel", "fused_combine_finish_kernel"],
     "placement_cost": ["cost_workload_hist_kernel", "cost_from_workload_kernel", "cost_count_scan_kernel", "cost_kernel",
                        "cost_travel_count_scan_kernel", "cost_local_kernel"],
 }
@@ -462,6 +463,9 @@ def main():
     ap.add_argument("--fused", action="store_true",
                     help="index-only dispatch + director_expert_ffn_gather (the GEMM gathers rows from x) instead of the "
                          "materialised permutation")
+    ap.add_argument("--fused-combine", action="store_true",
+                    help="director_expert_ffn_combine: the down projection combines in its epilogue (fp32 atomic adds; "
+                         "opt-in, not bit-reproducible) instead of writing Yp for a separate combine kernel")
     ap.add_argument("--graph", action="store_true",
                     help="replay the device-resident step from a CUDA graph (decode-sized batches); no per-kernel timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -505,7 +509,7 @@ def main():
 
     # ---- device-resident throughput ----
     for _ in range(max(args.warmup, 3)):
-        layer.forward(T, logits, x, fused=args.fused)
+        layer.forward(T, logits, x, fused=args.fused, fused_combine=args.fused_combine)
     torch.cuda.synchronize()
     layer.d.check_device_status()
 
@@ -518,13 +522,13 @@ def main():
             sampler = None
     # keep the GPU busy while the sampler starts so that the first samples see load clocks
     for _ in range(3):
-        layer.forward(T, logits, x, fused=args.fused)
+        layer.forward(T, logits, x, fused=args.fused, fused_combine=args.fused_combine)
     barrier()
     torch.cuda.synchronize()
     graph, launches_per_pass = None, 0
     if args.graph:
         n_c = layer.d.launch_count()
-        graph = layer.capture(T, logits, x, fused=args.fused)
+        graph = layer.capture(T, logits, x, fused=args.fused, fused_combine=args.fused_combine)
         launches_per_pass = (layer.d.launch_count() - n_c) // 2      # capture() runs the pass twice (warm-up + record)
     else:
         # inside the timed region only the dominant kernel is bracketed by events (its live duration is what the
@@ -536,7 +540,7 @@ def main():
     ev0.record()
     for _ in range(args.steps):
         if graph is None:
-            layer.forward(T, logits, x, fused=args.fused)
+            layer.forward(T, logits, x, fused=args.fused, fused_combine=args.fused_combine)
         else:
             graph.replay()
     ev1.record()
@@ -569,7 +573,7 @@ def main():
         layer.d.set_profiling(True)
         wallx0 = time.time()
         for _ in range(extra):
-            layer.forward(T, logits, x, fused=args.fused)
+            layer.forward(T, logits, x, fused=args.fused, fused_combine=args.fused_combine)
         torch.cuda.synchronize()
         wallx1 = time.time()
         for names in STAGE_KERNELS.values():
@@ -583,7 +587,7 @@ def main():
         # kernels pays the bracket once (a pair of events around a microsecond kernel costs as much as the kernel)
         layer.d.set_profiling(2)
         for _ in range(extra):
-            layer.forward(T, logits, x, fused=args.fused)
+            layer.forward(T, logits, x, fused=args.fused, fused_combine=args.fused_combine)
         torch.cuda.synchronize()
         wallx1 = time.time()
         for stage in STAGE_KERNELS:

@@ -182,6 +182,23 @@ int director_expert_ffn_gather(director_ctx* ctx, int32_t T, const void* x, cons
                                const void* w_down, void* yp, const void* ws_gate, const void* ws_up,
                                const void* ws_down, void* y_shared, void* stream);
 
+/* (a3) and (a4) fused, the second half of the survey's "next-2" row: both projections run on the tensor-core
+ * kernels and the down projection combines in its epilogue - every accumulator element, times its row's gating
+ * weight, is added (fp32 atomic add) into an accumulator of y at its row's token, so that Yp is never written and
+ * the combine step (Section II-A: y = sum of the chosen experts' outputs weighted by the gate) shrinks to one
+ * rounding pass.  OPT-IN, for two reasons: the K contributions of a token arrive in no fixed order, so y is
+ * reproducible only to fp32 rounding (the default path is bit-reproducible and placement-invariant); and it is
+ * slower - the atomic traffic costs more than the separate combine kernel saves.
+ * xp, seg_offsets, row_token, inv_row, topk_w: as written by director_dispatch / director_route.  x and ws_*: as for
+ * director_expert_ffn (shared experts run iff the context has S > 0 and x != NULL).  y_acc: dev fp32 [T,H] scratch,
+ * row_weight: dev fp32 [T*K] scratch (caller-owned, contents irrelevant on entry).  y: dev bf16 [T,H] out.
+ * Needs the default tile scheme (director_set_ffn_variant 2), otherwise DIRECTOR_ERR_UNSUPPORTED. */
+int director_expert_ffn_combine(director_ctx* ctx, int32_t T, const void* xp, const int32_t* seg_offsets,
+                                const int32_t* row_token, const int32_t* inv_row, const float* topk_w,
+                                const void* w_gate, const void* w_up, const void* w_down, const void* x,
+                                const void* ws_gate, const void* ws_up, const void* ws_down, float* y_acc,
+                                float* row_weight, void* y, void* stream);
+
 /* (a4) Combine (Section II-A weighted summation; Section II-B second all-to-all):
  *   y[t,:] = bf16( sum_s topk_w[t,s] * yp[inv_row[t,s],:]  (+ y_shared[t,:]) ), fp32 accumulation
  * in slot order.  yp: dev bf16 [T*K,H].  inv_row: dev int32 [T,K].  topk_w: dev fp32 [T,K].

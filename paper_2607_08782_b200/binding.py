@@ -23,7 +23,7 @@ EXPORTED = (
     "director_expert_ffn", "director_combine", "director_placement_cost", "director_layer_forward_host",
     "director_last_status", "director_launch_count", "director_set_profiling", "director_kernel_time",
     "director_status_string", "director_dispatch_index_static", "director_layer_submit_host",
-    "director_layer_wait_host", "director_set_ffn_variant", "director_batch_streams_weights", "director_placement_cost_batch",
+    "director_layer_wait_host", "director_set_ffn_variant", "director_batch_streams_weights", "director_expert_ffn_combine", "director_placement_cost_batch",
     "director_expert_ffn_gather", "director_set_replica_policy", "director_dispatch_src",
     "director_dedup_dispatch_tokens", "director_route_dispatch_cost", "director_layer_forward",
     "director_reserve_placements", "director_select_placement", "director_set_profiling_filter",
@@ -63,6 +63,7 @@ def load_library(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.director_expert_ffn.argtypes = [vp, c_int32] + [vp] * 12
     lib.director_expert_ffn_gather.argtypes = [vp, c_int32] + [vp] * 12
     lib.director_combine.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp]
+    lib.director_expert_ffn_combine.argtypes = [vp, c_int32] + [vp] * 16
     lib.director_placement_cost.argtypes = [vp, c_int32, vp, vp, vp, vp, vp, vp, vp]
     lib.director_layer_forward_host.argtypes = [vp, c_int32] + [vp] * 12
     lib.director_layer_forward.argtypes = [vp, c_int32] + [vp] * 14
@@ -194,6 +195,13 @@ class Director:
                                                    _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(yp), _ptr(ws_gate),
                                                    _ptr(ws_up), _ptr(ws_down), _ptr(y_shared), _stream()),
                "director_expert_ffn_gather")
+
+    def expert_ffn_combine(self, T, xp, seg_offsets, row_token, inv_row, topk_w, w_gate, w_up, w_down, x, ws_gate, ws_up,
+                           ws_down, y_acc, row_weight, y):
+        _check(self.lib.director_expert_ffn_combine(self._ctx, T, _ptr(xp), _ptr(seg_offsets), _ptr(row_token),
+                                                    _ptr(inv_row), _ptr(topk_w), _ptr(w_gate), _ptr(w_up), _ptr(w_down),
+                                                    _ptr(x), _ptr(ws_gate), _ptr(ws_up), _ptr(ws_down), _ptr(y_acc),
+                                                    _ptr(row_weight), _ptr(y), _stream()), "director_expert_ffn_combine")
 
     def combine(self, T, yp, inv_row, topk_w, y_shared, y):
         _check(self.lib.director_combine(self._ctx, T, _ptr(yp), _ptr(inv_row), _ptr(topk_w), _ptr(y_shared),

@@ -412,6 +412,37 @@ int director_expert_ffn_gather(director_ctx* ctx, int32_t T, const void* x, cons
                              shared ? y_shared : nullptr, as_stream(stream));
 }
 
+int director_expert_ffn_combine(director_ctx* ctx, int32_t T, const void* xp, const int32_t* seg_offsets,
+                                const int32_t* row_token, const int32_t* inv_row, const float* topk_w,
+                                const void* w_gate, const void* w_up, const void* w_down, const void* x,
+                                const void* ws_gate, const void* ws_up, const void* ws_down, float* y_acc,
+                                float* row_weight, void* y, void* stream) {
+    REQUIRE_CTX(ctx);
+    REQUIRE_T(ctx, T);
+    REQUIRE_PLACEMENT(ctx);
+    REQUIRE_PTR(xp);
+    REQUIRE_PTR(seg_offsets);
+    REQUIRE_PTR(row_token);
+    REQUIRE_PTR(inv_row);
+    REQUIRE_PTR(topk_w);
+    REQUIRE_PTR(w_gate);
+    REQUIRE_PTR(w_up);
+    REQUIRE_PTR(w_down);
+    REQUIRE_PTR(y_acc);
+    REQUIRE_PTR(row_weight);
+    REQUIRE_PTR(y);
+    const bool shared = ctx->shape.S > 0 && x != nullptr;
+    if (shared) {
+        REQUIRE_PTR(ws_gate);
+        REQUIRE_PTR(ws_up);
+        REQUIRE_PTR(ws_down);
+    }
+    if (ctx->ffn_variant != 2) return DIRECTOR_ERR_UNSUPPORTED;
+    return launch_expert_ffn_combine(ctx, T, xp, seg_offsets, row_token, inv_row, topk_w, w_gate, w_up, w_down,
+                                     shared ? x : nullptr, ws_gate, ws_up, ws_down, y_acc, row_weight, y,
+                                     as_stream(stream));
+}
+
 int director_combine(director_ctx* ctx, int32_t T, const void* yp, const int32_t* inv_row, const float* topk_w,
                      const void* y_shared, void* y, void* stream) {
     REQUIRE_CTX(ctx);

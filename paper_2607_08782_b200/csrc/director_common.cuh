@@ -241,6 +241,17 @@ struct DenseFfn {
     void* hidden;          // bf16 [rows, Fw]
     void* out;             // bf16 [rows, H]
 };
+// The combining form of the down projection (see grouped_gemm_swap_kernel, ALT): per permuted row its token and gating
+// weight, and the fp32 [T, H] accumulator of y (zeroed by the caller).
+struct FusedCombine {
+    const int32_t* row_token;
+    const float* row_weight;
+    float* y_acc;
+};
+int launch_expert_ffn_combine(director_ctx*, int T, const void* xp, const int32_t* seg_offsets, const int32_t* row_token,
+                              const int32_t* inv_row, const float* topk_w, const void* w_gate, const void* w_up,
+                              const void* w_down, const void* x, const void* ws_gate, const void* ws_up,
+                              const void* ws_down, float* y_acc, float* row_weight, void* y, cudaStream_t);
 int launch_expert_ffn(director_ctx*, int T, const void* xp, const int32_t* row_token, const int32_t* seg_offsets,
                       const void* w_gate, const void* w_up, const void* w_down, void* yp, const void* x,
                       const void* ws_gate, const void* ws_up, const void* ws_down, void* y_shared, cudaStream_t);

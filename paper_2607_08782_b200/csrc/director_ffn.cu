@@ -23,6 +23,8 @@
 #include "director_common.cuh"
 #include "director_umma.cuh"
 
+#include <cuda_bf16.h>
+
 #include <algorithm>
 
 namespace director {
@@ -31,7 +33,7 @@ int ffn_swap_init(director_ctx* ctx);   // director_ffn_swap.cu
 int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int32_t* gather_rows, uint64_t rows,
                   const int32_t* seg_offsets, const int32_t* slot_expert, int G, const void* w_gate, const void* w_up,
                   const void* w_down, uint64_t n_experts, int Fw, void* hidden, void* out, unsigned int* counters,
-                  const DenseFfn* dense, uint64_t max_seg_rows, cudaStream_t st);
+                  const DenseFfn* dense, uint64_t max_seg_rows, const FusedCombine* fc, cudaStream_t st);
 int ffn_small_init(director_ctx* ctx);  // director_ffn_small.cu
 bool ffn_small_applies(const director_ctx* ctx, int T, int Fw);
 int ffn_pass_small(director_ctx* ctx, const void* in, const int32_t* gather_rows, const int32_t* seg_offsets, const int32_t* slot_expert, int G,
@@ -288,7 +290,7 @@ int ffn_pass(director_ctx* ctx, const void* in, uint64_t in_rows, const int32_t*
              uint64_t max_seg_rows, cudaStream_t st) {
     if (ctx->ffn_variant == 2) {
         const int rc = ffn_pass_swap(ctx, in, in_rows, gather_rows, rows, seg_offsets, slot_expert, G, w_gate, w_up, w_down,
-                                     n_experts, Fw, hidden, out, counters, nullptr, max_seg_rows, st);
+                                     n_experts, Fw, hidden, out, counters, nullptr, max_seg_rows, nullptr, st);
         if (rc != DIRECTOR_ERR_UNSUPPORTED) return rc;   // weight arrays not expressible as one map: tile scheme 0
     }
     if (gather_rows != nullptr) return DIRECTOR_ERR_UNSUPPORTED;   // only the weight-stationary scheme gathers
@@ -359,7 +361,7 @@ int launch_expert_ffn(director_ctx* ctx, int T, const void* xp, const int32_t* r
         // routed and shared experts in the same two launches: the shared experts' work items follow the routed ones
         const DenseFfn dense{x, (uint64_t)T, ws_gate, ws_up, ws_down, s.S * s.F, ctx->d_hidden_shared, y_shared};
         const int rc = ffn_pass_swap(ctx, xp, A, nullptr, A, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up, w_down,
-                                     s.E, s.F, ctx->d_hidden, yp, ctx->d_sched, &dense, (uint64_t)T, st);
+                                     s.E, s.F, ctx->d_hidden, yp, ctx->d_sched, &dense, (uint64_t)T, nullptr, st);
         if (rc != DIRECTOR_ERR_UNSUPPORTED) return rc;    // a weight pair not expressible as one map: separate passes
     }
     int rc = row_token ? ffn_pass(ctx, x, (uint64_t)T, row_token, A, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up,
@@ -375,6 +377,81 @@ int launch_expert_ffn(director_ctx* ctx, int T, const void* xp, const int32_t* r
     // The S shared experts as one FFN of width S*F over all T rows of x (a single segment, "expert" 0).
     return ffn_pass(ctx, x, (uint64_t)T, nullptr, (uint64_t)T, ctx->d_one_seg, ctx->d_zero_expert, 1, ws_gate, ws_up,
                     ws_down, 1, s.S * s.F, ctx->d_hidden_shared, y_shared, ctx->d_sched + 2, (uint64_t)T, st);
+}
+
+namespace {
+
+// Zeroes the fp32 accumulator of y and writes every permuted row's gating weight (row_weight[inv_row[t,s]] = w[t,s]).
+__global__ void __launch_bounds__(256)
+combine_prepare_kernel(float4* __restrict__ y_acc, long long n_vec, const int32_t* __restrict__ inv_row,
+                       const float* __restrict__ topk_w, float* __restrict__ row_weight, long long A) {
+    chain_prologue();
+    const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x, stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = i0; i < n_vec; i += stride) y_acc[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    for (long long i = i0; i < A; i += stride) {
+        const int row = __ldg(inv_row + i);
+        if (row >= 0) row_weight[row] = __ldg(topk_w + i);
+    }
+}
+
+// y = bf16(y_acc + y_shared): the one rounding of the combining form.
+__global__ void __launch_bounds__(256)
+combine_finish_kernel(const float4* __restrict__ y_acc, const uint2* __restrict__ y_shared, uint2* __restrict__ y,
+                      long long n_vec) {
+    chain_prologue();
+    const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x, stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = i0; i < n_vec; i += stride) {
+        float4 a = __ldcs(y_acc + i);
+        if (y_shared != nullptr) {
+            const uint2 sh = __ldg(y_shared + i);
+            a.x += __uint_as_float(sh.x << 16);
+            a.y += __uint_as_float(sh.x & 0xFFFF0000u);
+            a.z += __uint_as_float(sh.y << 16);
+            a.w += __uint_as_float(sh.y & 0xFFFF0000u);
+        }
+        uint2 o;
+        o.x = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(a.x)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(a.y)) << 16);
+        o.y = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(a.z)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(a.w)) << 16);
+        y[i] = o;
+    }
+}
+
+}  // namespace
+
+// (a3) and (a4) in one: both projections on the tensor-core kernels, the down projection combining in its epilogue.
+// y_acc: fp32 [T, H] scratch, row_weight: fp32 [T*K] scratch (both caller-owned).  Tile scheme 2 only.
+int launch_expert_ffn_combine(director_ctx* ctx, int T, const void* xp, const int32_t* seg_offsets, const int32_t* row_token,
+                              const int32_t* inv_row, const float* topk_w, const void* w_gate, const void* w_up,
+                              const void* w_down, const void* x, const void* ws_gate, const void* ws_up,
+                              const void* ws_down, float* y_acc, float* row_weight, void* y, cudaStream_t st) {
+    if (ctx->ffn_variant != 2) return DIRECTOR_ERR_UNSUPPORTED;
+    const director_shape& s = ctx->shape;
+    const uint64_t A = (uint64_t)T * s.K;
+    const bool shared = s.S > 0 && x != nullptr;
+    const long long n_vec = (long long)T * s.H / 4;
+    const unsigned grid = (unsigned)std::min<long long>((n_vec + 255) / 256, 8LL * ctx->sm_count);
+    {
+        StageScope stage(ctx, st, "stage_expert_ffn");
+        {
+            LaunchScope scope(ctx, st, "fused_combine_prepare_kernel");
+            int rc = cuda_status(launch_chained(combine_prepare_kernel, dim3(grid), dim3(256), 0, st,
+                                                reinterpret_cast<float4*>(y_acc), n_vec, inv_row, topk_w, row_weight, (long long)A));
+            if (rc != DIRECTOR_OK) return rc;
+        }
+        if (cudaMemsetAsync(ctx->d_sched, 0, 4 * sizeof(unsigned int), st) != cudaSuccess) return DIRECTOR_ERR_CUDA;
+        const FusedCombine fc{row_token, row_weight, y_acc};
+        const DenseFfn dense{x, (uint64_t)T, ws_gate, ws_up, ws_down, s.S * s.F, ctx->d_hidden_shared, ctx->e_y_shared};
+        const int rc = ffn_pass_swap(ctx, xp, A, nullptr, A, seg_offsets, ctx->d_slot_expert, ctx->G, w_gate, w_up, w_down,
+                                     s.E, s.F, ctx->d_hidden, nullptr, ctx->d_sched, shared ? &dense : nullptr, (uint64_t)T,
+                                     &fc, st);
+        if (rc != DIRECTOR_OK) return rc;
+    }
+    StageScope stage(ctx, st, "stage_combine");
+    LaunchScope scope(ctx, st, "fused_combine_finish_kernel");
+    return cuda_status(launch_chained(combine_finish_kernel, dim3(grid), dim3(256), 0, st,
+                                      reinterpret_cast<const float4*>(y_acc),
+                                      shared ? static_cast<const uint2*>(ctx->e_y_shared) : static_cast<const uint2*>(nullptr),
+                                      static_cast<uint2*>(y), n_vec));
 }
 
 }  // namespace director

@@ -193,7 +193,8 @@ struct SwapParams {
     void* out;
     int32_t* status;
     unsigned int* counter;     // next unclaimed work item of this launch (zero when the kernel starts)
-    const int32_t* row_token;  // GATHER only: token of every permuted row (the tokens operand is gathered from x)
+    const int32_t* row_token;  // GATHER / combining epilogue: token of every permuted row
+    const float* row_weight;   // combining epilogue only: gating weight of every permuted row
     // Optional second problem of the same launch: one dense segment of `dense_rows` rows against a single weight
     // set (the shared experts run as one wide FFN over all tokens).  Its items follow the grouped problem's in the
     // work-item order, so the two share the launch, its prologue and its tail.  dense_rows == 0: absent.
@@ -270,14 +271,21 @@ struct SwapWalker {
 };
 
 // MODE 0: gate/up + SwiGLU (A from the 3-D interleaving map).  MODE 1: down projection (A from a 2-D map).
-// GATHER (GEMM-1 only): the token rows are not read from a permuted copy but gathered straight from the layer
+// ALT selects the alternative form of a launch.  GEMM-2 (MODE 1): the combining epilogue - instead of storing the
+// bf16 rows of Yp, every accumulator element is multiplied by its row's gating weight and added (red.global.add.f32)
+// into an fp32 [tokens, H] accumulator of y at its row's token, so the un-permute / combine step shrinks to one
+// rounding pass.  The K contributions of a token arrive in no fixed order: results are reproducible to fp32
+// rounding only, which is why this form is opt-in.  The dense problem (shared experts) stores bf16 as usual.
+// GEMM-1 (MODE 0), GATHER: the token rows are not read from a permuted copy but gathered straight from the layer
 // input x through row_token - tm_x then describes x with a one-row box and the whole producer warp issues the
 // loads, four rows per lane - so the dispatch step needs no row copies at all.
-template <int MODE, int EPI_GROUPS, bool GATHER, int S_STAGES>
+template <int MODE, int EPI_GROUPS, bool ALT, int S_STAGES>
 __global__ void __launch_bounds__(96 + 128 * EPI_GROUPS, 1)
 grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
                          const __grid_constant__ CUtensorMap tm_w2 /* dense problem */,
                          const __grid_constant__ CUtensorMap tm_x2, const SwapParams p) {
+    constexpr bool GATHER = ALT && MODE == 0;               // token rows gathered from x
+    constexpr bool COMBINE = ALT && MODE == 1;              // combining epilogue
     extern __shared__ uint8_t smem_raw[];
     chain_prologue();
     const uint32_t raw = smem_u32(smem_raw);
@@ -645,6 +653,27 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 }
             } else {
                 const int h_col = t.wb * 256 + (int)rank * 128 + lane_row;
+                if (COMBINE && !t.prob) {
+                    // lane j of the warp fetches token and gating weight of the chunk's j-th row; every lane then adds
+                    // its own feature of that row into the token's accumulator (32 lanes = 128 contiguous bytes)
+                    float* const acc_y = static_cast<float*>(p.out) + h_col;
+#pragma unroll 1
+                    for (int c = c_first; c < t.n; c += CSTEP) {
+                        uint32_t v[32];
+                        tmem_ld32(taddr + c, v);
+                        const int rem = t.valid - c;
+                        const int row = t.row0 + c + lane;
+                        const int tok = lane < rem ? __ldg(p.row_token + row) : 0;
+                        const float wgt = lane < rem ? __ldg(p.row_weight + row) : 0.0f;
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const int tj = __shfl_sync(0xFFFFFFFFu, tok, j);
+                            const float wj = __shfl_sync(0xFFFFFFFFu, wgt, j);
+                            if (j < rem) atomicAdd(acc_y + (size_t)tj * out_pitch, wj * __uint_as_float(v[j]));
+                        }
+                    }
+                } else {
                 uint16_t* ocol = out + (size_t)t.row0 * out_pitch + h_col;
 #pragma unroll 1
                 for (int c = c_first; c < t.n; c += CSTEP) {
@@ -658,6 +687,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                         if (j < rem) *ptr = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[j])));
                         ptr += out_pitch;
                     }
+                }
                 }
             }
             tc_fence_before();
@@ -783,7 +813,7 @@ bool swap_opt_in() {
 
 int ffn_swap_init(director_ctx*) {
     if (!swap_opt_in<0, EPI_GROUPS_GEMM1, false>() || !swap_opt_in<0, EPI_GROUPS_GEMM1, true>() ||
-        !swap_opt_in<1, EPI_GROUPS_GEMM2, false>())
+        !swap_opt_in<1, EPI_GROUPS_GEMM2, false>() || !swap_opt_in<1, EPI_GROUPS_GEMM2, true>())
         return DIRECTOR_ERR_CUDA;
     return DIRECTOR_OK;
 }
@@ -796,15 +826,17 @@ int ffn_swap_init(director_ctx*) {
 // max_seg_rows: an upper bound on the length of any segment of the table (`rows` if nothing better is known); with a
 // bound of at most 64 the launches use the small-batch ring (see S_SMALL_STAGES) - correct for any table, since that
 // ring also tiles the tokens by 64.
+// fc (optional, not with gather_rows): the down projection combines in its epilogue - `out` is not written; every
+// element of a routed row goes, times the row's gating weight, into fc->y_acc at the row's token (see the kernel's ALT).
 // Returns DIRECTOR_ERR_UNSUPPORTED if a pair of weight arrays cannot be described by one interleaving map.
 int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int32_t* gather_rows, uint64_t rows,
                   const int32_t* seg_offsets, const int32_t* slot_expert, int G, const void* w_gate, const void* w_up,
                   const void* w_down, uint64_t n_experts, int Fw, void* hidden, void* out,
                   unsigned int* counters /* 2 zeroed work-item counters */, const DenseFfn* dense, uint64_t max_seg_rows,
-                  cudaStream_t st) {
+                  const FusedCombine* fc, cudaStream_t st) {
     const int H = ctx->shape.H;
     // small-batch ring (tiles of 64 tokens, ten stages): when no segment, routed or dense, can be longer than a tile
-    const bool small = !gather_rows && max_seg_rows <= 2u * swap_tok_rows(S_SMALL_STAGES) &&
+    const bool small = !gather_rows && !fc && max_seg_rows <= 2u * swap_tok_rows(S_SMALL_STAGES) &&
                        (!dense || dense->rows <= 2u * swap_tok_rows(S_SMALL_STAGES));
     const uint32_t tok_box = small ? swap_tok_rows(S_SMALL_STAGES) : 128;
     struct Interleave { bool ok; bool gate_first; const void* first; uint64_t delta; };
@@ -816,7 +848,7 @@ int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int
     };
     const Interleave ia = interleave(w_gate, w_up);
     if (!ia.ok) return DIRECTOR_ERR_UNSUPPORTED;
-    if (dense && gather_rows) return DIRECTOR_ERR_INVALID_ARG;
+    if ((dense || fc) && gather_rows) return DIRECTOR_ERR_INVALID_ARG;
     CUtensorMap m_in, m_gu, m_h, m_d;
     if (!map_2d(ctx, &m_in, in, in_rows, H, gather_rows ? 1 : tok_box) || !map_2d(ctx, &m_h, hidden, rows, Fw, tok_box) ||
         !map_2d(ctx, &m_d, w_down, n_experts * H, Fw))
@@ -839,14 +871,17 @@ int ffn_pass_swap(director_ctx* ctx, const void* in, uint64_t in_rows, const int
     const int32_t* order = (slot_expert == ctx->d_slot_expert && G == ctx->G && swap_can_order(G)) ? slot_expert + G : nullptr;
     unsigned long long* const clk = ctx->gemm_stats ? ctx->d_gemm_clock : nullptr;
     SwapParams p1{seg_offsets, slot_expert, order, G, Fw / 128, H / BLOCK_K, Fw, Fw, ia.gate_first ? 1 : 0, hidden, ctx->d_status,
-                  counters, gather_rows, d_rows, d_Fw / 128, H / BLOCK_K, d_Fw, id.gate_first ? 1 : 0,
+                  counters, gather_rows, nullptr, d_rows, d_Fw / 128, H / BLOCK_K, d_Fw, id.gate_first ? 1 : 0,
                   dense ? dense->hidden : nullptr, clk};
     int rc = gather_rows ? launch_swap<0, EPI_GROUPS_GEMM1, true>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, d_gu, d_in, p1, false, st)
                          : launch_swap<0, EPI_GROUPS_GEMM1, false>(ctx, "grouped_gemm_swiglu_kernel", m_gu, m_in, d_gu, d_in, p1, small, st);
     if (rc != DIRECTOR_OK) return rc;
-    SwapParams p2{seg_offsets, slot_expert, order, G, H / 256, Fw / BLOCK_K, H, H, 1, out, ctx->d_status, counters + 1, nullptr,
+    // with fc the routed experts' output is not Yp but the fp32 accumulator of y (pitch H floats), see the kernel's ALT
+    SwapParams p2{seg_offsets, slot_expert, order, G, H / 256, Fw / BLOCK_K, H, H, 1, fc ? static_cast<void*>(fc->y_acc) : out,
+                  ctx->d_status, counters + 1, fc ? fc->row_token : nullptr, fc ? fc->row_weight : nullptr,
                   d_rows, H / 256, d_Fw / BLOCK_K, H, 1, dense ? dense->out : nullptr,
                   clk ? clk + (size_t)kGemmClockWords * kGemmClockCtas : nullptr};
+    if (fc) return launch_swap<1, EPI_GROUPS_GEMM2, true>(ctx, "grouped_gemm_down_fused_kernel", m_d, m_h, d_d, d_h, p2, false, st);
     return launch_swap<1, EPI_GROUPS_GEMM2, false>(ctx, "grouped_gemm_down_kernel", m_d, m_h, d_d, d_h, p2, small, st);
 }
 

@@ -93,18 +93,31 @@ class MoELayer:
     def combine(self, T):
         self.d.combine(T, self.yp, self.inv_row, self.topk_w, self.y_shared, self.y)
 
+    def expert_ffn_combine(self, T, x=None):
+        """Expert FFN with the combine fused into the down projection's epilogue (fp32 atomic adds into an accumulator
+        of y: not bit-reproducible, and slower than the two separate steps - see director_expert_ffn_combine)."""
+        d = self.dims
+        if getattr(self, "y_acc", None) is None:
+            dev = self.y.device
+            self.y_acc = torch.empty((d["T_max"], d["H"]), dtype=torch.float32, device=dev)
+            self.row_weight = torch.empty((d["T_max"] * d["K"],), dtype=torch.float32, device=dev)
+        S = d["S"]
+        self.d.expert_ffn_combine(T, self.xp, self.seg_offsets, self.row_token, self.inv_row, self.topk_w, *self.w,
+                                  x if S > 0 else None, *(self.ws if S > 0 else (None, None, None)), self.y_acc,
+                                  self.row_weight, self.y)
+
     def placement_cost(self, T, token_src_rank=None):
         self.d.placement_cost(T, self.topk_idx, token_src_rank, self.workload, self.rank_load,
                               self.dispatch_tokens, self.dispatch_bytes)
 
-    def forward(self, T, logits, x, with_cost=True, fused=False):
+    def forward(self, T, logits, x, with_cost=True, fused=False, fused_combine=False):
         """One pass of the whole layer on device tensors; returns y[:T] (a view of the owned buffer).
         fused: dispatch produces indices only and the expert GEMM gathers its rows from x.  Off by default: the
         weight-stationary GEMM re-reads a token tile once per weight block, so the gather is repeated 2F/256 times
         and costs more than the single row copy it saves."""
         # a batch small enough for the weight-streaming FFN kernels needs no permuted copy either: they stage a
         # segment's few rows from x themselves
-        gather = (fused and self.ffn_variant == 2) or self.d.batch_streams_weights(T)
+        gather = (fused and self.ffn_variant == 2) or (self.d.batch_streams_weights(T) and not fused_combine)
         if with_cost:          # front end in one call (a single launch for decode-sized batches)
             self.d.route_dispatch_cost(T, logits, x, self.topk_idx, self.topk_w, None if gather else self.xp,
                                        self.row_token, self.inv_row, self.dest_rank, self.seg_offsets, self.workload,
@@ -112,6 +125,9 @@ class MoELayer:
         else:
             self.route(T, logits)
             self.dispatch(T, x, indices_only=gather)
+        if fused_combine and not gather:          # combine inside the down projection (opt-in, see expert_ffn_combine)
+            self.expert_ffn_combine(T, x)
+            return self.y[:T]
         if gather:
             self.expert_ffn_gather(T, x)
         else:
@@ -119,16 +135,16 @@ class MoELayer:
         self.combine(T)
         return self.y[:T]
 
-    def capture(self, T, logits, x, with_cost=True, fused=False):
+    def capture(self, T, logits, x, with_cost=True, fused=False, fused_combine=False):
         """Records one pass of the layer (fixed T, fixed input and output buffers) into a CUDA graph and returns it;
         `graph.replay()` re-runs the pass with a single launch, which matters for decode-sized batches where the
         handful of kernel launches cost more than the kernels.  Per-kernel profiling must be off while capturing."""
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):                      # first pass outside the capture: lazy module loading
-            self.forward(T, logits, x, with_cost, fused)
+            self.forward(T, logits, x, with_cost, fused, fused_combine)
         torch.cuda.current_stream().wait_stream(side)
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
-            self.forward(T, logits, x, with_cost, fused)
+            self.forward(T, logits, x, with_cost, fused, fused_combine)
         return graph

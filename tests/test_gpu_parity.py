@@ -738,3 +738,46 @@ def test_small_batch_ring_gives_the_same_bits_as_the_ordinary_one(seed, H, E, K,
         idx, w, w64, d, c = _oracle_front(shape, logits[:T], x[:T], X, C)
         sT = synth.Shape(shape.name, T, H, E, K, F, S, R, C, shape.zipf_s, shape.seed)
         _check_outputs(sT, g, x[:T], weights, idx, w, w64, d, c, np.arange(T), f"small_ring{seed}_T{T}")
+
+
+@pytest.mark.parametrize("seed,T,H,E,K,F,S,R,C,extra", [
+    (141, 777, 256, 12, 3, 384, 0, 4, 4, 4),       # several tiles and ragged tails, replicas
+    (142, 1000, 512, 60, 4, 256, 2, 8, 8, 4),      # shared experts: the dense problem still stores bf16
+    (143, 33, 256, 5, 5, 128, 1, 2, 5, 5),         # K == E, a small batch (tensor-core kernels all the same)
+    (144, 3, 256, 8, 2, 128, 0, 4, 2, 0),          # a batch the default path would stream
+])
+def test_combining_down_projection_matches_the_oracle_and_the_two_step_path(seed, T, H, E, K, F, S, R, C, extra):
+    """director_expert_ffn_combine: the down projection adds w * value into an fp32 accumulator of y in its epilogue.
+    Same mathematics as expert_ffn + combine, another rounding (Yp is never rounded to bf16) and no fixed order of
+    the K contributions: compared within the layer's tolerance, against the oracle on every token and against the
+    two-step path."""
+    import torch
+    from paper_2607_08782_b200.layer import tensor_to_bf16_bits
+    shape, logits, x, weights = _custom(seed, T, H, E, K, F, S, R, C)
+    X = _random_placement(seed, E, R, C, extra)
+    case = GpuCase(shape, logits, x, weights)
+    g = case.run(X)                                        # route, dispatch, expert_ffn, combine
+    L = case.layer
+    y_two_step = g.y.copy()
+    L.y.zero_()
+    n0 = L.d.launch_count()
+    L.expert_ffn_combine(T, case.x)                        # on the tables the run above left in place
+    torch.cuda.synchronize()
+    assert L.d.last_status() == 0
+    assert L.d.launch_count() - n0 == 4                    # prepare, gate|up, down + combine, rounding pass
+    y_fused = tensor_to_bf16_bits(L.y[:T])
+    idx, w, w64, d, c = _oracle_front(shape, logits, x, X, C)
+    y_o, rows, yp_o, ysh_o = oracle_layer_tokens(shape, x, weights, idx, w64, d, np.arange(T))
+    a = orc.bf16_to_f64(y_fused)
+    assert rel_l2(a, y_o) <= REL_L2_TOL and max_abs(a, y_o) <= MAX_ABS_TOL
+    b = orc.bf16_to_f64(y_two_step)
+    assert rel_l2(a, b) <= REL_L2_TOL and max_abs(a, b) <= MAX_ABS_TOL
+    y1 = L.forward(T, case.logits, case.x, fused_combine=True)           # whole layer with the fused step
+    torch.cuda.synchronize()
+    a1 = orc.bf16_to_f64(tensor_to_bf16_bits(y1))
+    assert rel_l2(a1, y_o) <= REL_L2_TOL and max_abs(a1, y_o) <= MAX_ABS_TOL
+    case.layer.d.set_ffn_variant(0)                         # the other tile schemes have no combining epilogue
+    from paper_2607_08782_b200.binding import DirectorError
+    with pytest.raises(DirectorError):
+        L.expert_ffn_combine(T, case.x)
+    case.layer.d.set_ffn_variant(2)
