@@ -3,7 +3,8 @@
  *   - the segment table ends at T*K and every assignment's row points back at its token,
  *   - the per-rank loads of Eq. 1 sum to T*K and the workload matrix sums to T*K,
  *   - dispatch followed by combine with identity experts (yp := xp) returns x bit for bit,
- *   - the stage calls in order and director_layer_forward give the same bits (y and all histograms).
+ *   - the stage calls in order and director_layer_forward give the same bits (y and all histograms),
+ *   - the combining down projection (director_expert_ffn_combine) agrees with expert_ffn + combine to bf16 rounding.
  * Exit code 0 = pass.  Built and run by tests/test_gpu_c_abi.py. */
 #include <cuda_runtime_api.h>
 #include <stdio.h>
@@ -151,8 +152,34 @@ int main(void) {
     const int layer_ok = memcmp(y2, y, 2 * T * H) == 0 && memcmp(cost2, cost, sizeof cost) == 0;
     if (!layer_ok) ++bad;
 
-    printf("layer_from_c: %d tokens, %d assignments, identity %s, one-call layer %s, %d mismatches\n", T, A,
-           identity_ok ? "exact" : "DIFFERS", layer_ok ? "identical" : "DIFFERS", bad);
+    /* ---- which FFN kernels a batch takes: the streaming ones up to 4 tokens ---- */
+    if (director_batch_streams_weights(ctx, T) != 0 || director_batch_streams_weights(ctx, 2) != 1 ||
+        director_batch_streams_weights(ctx, 0) >= 0 || director_batch_streams_weights(NULL, 1) >= 0)
+        ++bad;
+
+    /* ---- the combining down projection agrees with expert_ffn + combine to a bf16 unit or two ---- */
+    float* d_yacc = (float*)dev_copy(NULL, sizeof(float) * T * H);
+    float* d_rw = (float*)dev_copy(NULL, sizeof(float) * A);
+    if (!d_yacc || !d_rw) return 3;
+    CHECK(cudaMemset(d_y2, 0, 2 * T * H));
+    CHECK(director_expert_ffn_combine(ctx, T, d_xp, d_seg, d_row_token, d_inv_row, d_w, d_wg, d_wu, d_wd, NULL, NULL, NULL,
+                                      NULL, d_yacc, d_rw, d_y2, NULL));
+    CHECK(cudaDeviceSynchronize());
+    CHECK(director_last_status(ctx, NULL));
+    CHECK(cudaMemcpy(y2, d_y2, 2 * T * H, cudaMemcpyDeviceToHost));
+    int fused_far = 0;
+    for (int i = 0; i < T * H; ++i) {
+        uint32_t ua = (uint32_t)y[i] << 16, ub = (uint32_t)y2[i] << 16;
+        float a, b;
+        memcpy(&a, &ua, 4);
+        memcpy(&b, &ub, 4);
+        const float d = a > b ? a - b : b - a, m = (a < 0 ? -a : a) > (b < 0 ? -b : b) ? (a < 0 ? -a : a) : (b < 0 ? -b : b);
+        if (d > m / 64.0f + 1e-3f) ++fused_far;
+    }
+    if (fused_far) ++bad;
+
+    printf("layer_from_c: %d tokens, %d assignments, identity %s, one-call layer %s, fused combine %d far, %d mismatches\n",
+           T, A, identity_ok ? "exact" : "DIFFERS", layer_ok ? "identical" : "DIFFERS", fused_far, bad);
     CHECK(director_destroy(ctx));
     return bad ? 1 : 0;
 }
