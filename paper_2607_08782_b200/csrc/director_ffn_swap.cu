@@ -389,9 +389,9 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     SwapTile t;
 
     // Work items (segment, weight block, token tile) are handed out dynamically, in their natural order, from a
-    // global counter.  A scheduler thread - lane 0 of a warp of its own in the leader CTA, next to the MMA thread that
+    // global counter.  A scheduler thread - lane 0 of a warp of its own in the leader CTA, next to the MMA warp that
     // reads its ring most urgently - claims items and publishes them through a small ring in both CTAs' shared
-    // memory, already decoded into tile coordinates; every other role (both producers, the MMA thread, all epilogue
+    // memory, already decoded into tile coordinates; every other role (both producers, the MMA warp, all epilogue
     // warps) reads the ring.  Claiming and publishing take ~2000 cycles per item (a global atomic, a remote
     // store and a remote arrive with cluster-scope release); on a thread of its own that latency is off the load
     // path.  Tail tiles are cheaper than full ones, so fixed assignments leave 6-15 % of imbalance between clusters;
