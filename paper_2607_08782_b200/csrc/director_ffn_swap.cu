@@ -218,6 +218,7 @@ struct SwapTile {
     int n;         // valid rounded up to a multiple of 32: N of the MMA
     int w_row;     // first weight row of the pair's block (f index for GEMM-1, W_down row for GEMM-2)
     int wb;
+    int tail;      // 1: the tile follows full tiles of its segment (its ragged end), 0: the segment's first tile
 };
 
 // Work items in their hand-out order.  Consecutive segments of the walk that hold the same expert (the replicas of
@@ -262,6 +263,7 @@ struct SwapWalker {
             local -= tt_start[g] - tt_start[gs];
         }
         t.prob = 0;
+        t.tail = local > 0 ? 1 : 0;
         t.row0 = seg_off[g] + local * tile_rows;
         t.valid = min(tile_rows, seg_end[g] - t.row0);
         t.n = (t.valid + TOKEN_STEP - 1) / TOKEN_STEP * TOKEN_STEP;
@@ -414,7 +416,8 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
             tile.valid = v.y;
             tile.n = (v.y + TOKEN_STEP - 1) / TOKEN_STEP * TOKEN_STEP;
             tile.w_row = v.z;
-            tile.wb = v.w & 0x3FFFFFFF;
+            tile.wb = v.w & 0x1FFFFFFF;
+            tile.tail = (v.w >> 29) & 1;
             tile.prob = (v.w >> 30) & 1;
         }
         return ok;
@@ -434,6 +437,7 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
         tile.w_row = __shfl_sync(0xFFFFFFFFu, tile.w_row, 0);
         tile.wb = __shfl_sync(0xFFFFFFFFu, tile.wb, 0);
         tile.prob = __shfl_sync(0xFFFFFFFFu, tile.prob, 0);
+        tile.tail = __shfl_sync(0xFFFFFFFFu, tile.tail, 0);
         return ok;
     };
     const uint32_t abort_addr = smem_u32(const_cast<const int*>(abort_flag));
@@ -536,6 +540,14 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 const uint32_t idesc = S_IDESC_BASE | ((uint32_t)(t.n >> 3) << 17);
                 const int k_steps = t.prob ? p.dense_k_steps : p.k_steps;
                 const uint32_t c_loop = stats ? (uint32_t)clock() : 0u;
+                // The ragged end of a segment that also has full tiles, in a LONG contraction, is paced to a full tile's
+                // speed (512 cycles per k-step).  Finishing early buys nothing there - items are few and long, the part
+                // is power-limited - while a cluster that runs ahead of the clusters it shares its weight block with,
+                // and then starts its next item out of step with its neighbours, stops meeting them in L2: with unpaced
+                // ragged tiles a Mixtral-shaped down projection read 2.19 GB from DRAM instead of 1.59 GB, and the
+                // layer step was 2.8 % slower.  Segments without a full tile (small batches) are never paced.
+                const bool paced = MODE == 1 && S_STAGES <= 8 && k_steps >= 128 && t.tail && t.n < TOKEN_TILE;
+                const uint32_t c_pace = (uint32_t)clock();
                 stat_a += c_loop - c_item;                  // waited for the accumulator buffer
                 stat_c += (uint32_t)k_steps;
                 stat_d += 1;
@@ -545,6 +557,9 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                     bad = mbar_wait_conv(full_bar(stage), phase, abort_addr, bad, lead_lane);
                     tc_fence_after();
                     if (lead_lane && !bad) {
+                        if (paced) {                       // see `paced` above: no k-step before its full-tile slot
+                            while ((uint32_t)clock() - c_pace < 512u * (uint32_t)kb) {}
+                        }
 #pragma unroll
                         for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
                             umma_pair_n(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
@@ -585,12 +600,13 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 int4 item = make_int4(0, 0, 0, 0);
                 if (w < walker.total) {
                     walker.get(w, t);
-                    item = make_int4(t.row0, t.valid, t.w_row, t.wb);
+                    item = make_int4(t.row0, t.valid, t.w_row, t.wb | (t.tail << 29));
                     pub_k += p.k_steps;
                 } else if (w < total_items) {          // dense problem: (weight block, token tile) over one segment
                     const int local = w - walker.total;
                     const int wb = local / dense_tiles, row0 = (local - wb * dense_tiles) * TILE_ROWS;
-                    item = make_int4(row0, min(TILE_ROWS, p.dense_rows - row0), wb * ROWS_PER_BLOCK, wb | (1 << 30));
+                    item = make_int4(row0, min(TILE_ROWS, p.dense_rows - row0), wb * ROWS_PER_BLOCK,
+                                     wb | ((row0 > 0 ? 1 : 0) << 29) | (1 << 30));
                     pub_k += p.dense_k_steps;
                 }
                 sched_item[q] = item;
