@@ -37,8 +37,8 @@ UNIT = "tokens/s"
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from the
 # committed ncu summary of that kernel on that workload (None until a capture for the workload exists).
 NCU_TRAFFIC_BYTES = {
-    # gate||up GEMM, full-size workload: 1 954 545 920 B read + 229 700 608 B written
-    "c2_mixtral": 2184246528,
+    # gate||up GEMM, full-size workload: 1 955 644 416 B read + 229 357 568 B written
+    "c2_mixtral": 2185001984,
 }
 
 
