@@ -603,8 +603,16 @@ grouped_gemm_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                     item = make_int4(t.row0, t.valid, t.w_row, t.wb | (t.tail << 29));
                     pub_k += p.k_steps;
                 } else if (w < total_items) {          // dense problem: (weight block, token tile) over one segment
+                    // Chunks of token tiles, inside a chunk weight block first, the chunk sized so that all weight
+                    // blocks of its tiles are in flight together (clusters / weight blocks tiles): a token tile is then
+                    // read from HBM once, by the clusters that work on it at the same k, instead of once per weight block
+                    // (a dense segment's activations need not fit in L2: four Qwen1.5-shaped shared experts' hidden
+                    // activations are 185 MB, and weight-block-major order read them eight times).
                     const int local = w - walker.total;
-                    const int wb = local / dense_tiles, row0 = (local - wb * dense_tiles) * TILE_ROWS;
+                    const int chunk = max(1, (int)(gridDim.x >> 1) / p.dense_w_blocks);
+                    const int ch = local / (chunk * p.dense_w_blocks), r = local - ch * chunk * p.dense_w_blocks;
+                    const int in_chunk = min(chunk, dense_tiles - ch * chunk);
+                    const int wb = r / in_chunk, row0 = (ch * chunk + r - wb * in_chunk) * TILE_ROWS;
                     item = make_int4(row0, min(TILE_ROWS, p.dense_rows - row0), wb * ROWS_PER_BLOCK,
                                      wb | ((row0 > 0 ? 1 : 0) << 29) | (1 << 30));
                     pub_k += p.dense_k_steps;
